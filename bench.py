@@ -1,0 +1,316 @@
+#!/usr/bin/env python
+"""Benchmark of the convolution-forward hot path on B200.
+
+A "step" is one forward pass of the AlexNet-shaped, ungrouped conv stack at batch 20
+(conv1 pool conv2 pool conv3 conv4 conv5 pool; 43.07 GFLOP of convolution) on synthetic seeded
+inputs.  With N GPUs every rank runs its own replica of the step on its own batch (batch items are
+independent, so the path shards over images with no collective): weak scaling.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+
+Prints ONE JSON line (rank 0).  `value` is conv GFLOP/s with inputs resident in HBM; `e2e` is the
+same metric with the image batch copied from pinned host memory and the result copied back inside
+the timed region.  `--impl reference` times the fp64 CPU oracle on the host cores instead.
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+if ROOT not in sys.path:
+    sys.path.insert(0, ROOT)
+
+METRIC = "conv_forward_gflops_alexnet_conv_stack"
+UNIT = "GFLOP/s"
+BATCH = 20
+L2_FLUSH_BYTES = 512 << 20
+
+
+def _peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        p = json.load(open(path))
+        return {"hbm_gbs": float(p["hbm_gbs"]), "bf16_tflops": float(p["bf16_tflops"]),
+                "bf16_tflops_sustained": float(p.get("bf16_tflops_sustained", p["bf16_tflops"])),
+                "sm_max_mhz": float(p.get("sm_max_mhz", 1965.0)), "source": "measured"}
+    return {"hbm_gbs": 6650.0, "bf16_tflops": 1590.0, "bf16_tflops_sustained": 1400.0, "sm_max_mhz": 1965.0,
+            "source": "fallback"}
+
+
+class ClockSampler:
+    """Samples SM clock and throttle reasons of one GPU with nvidia-smi while the timed region runs."""
+    FIELDS = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.hw_slowdown,"
+              "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+              "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index = gpu_index
+        self.samples = []
+        self.proc = None
+        self.thread = None
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(
+                ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
+                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+        except OSError:
+            self.proc = None
+            return
+        self.thread = threading.Thread(target=self._read, daemon=True)
+        self.thread.start()
+
+    def _read(self):
+        for line in self.proc.stdout:
+            parts = [p.strip() for p in line.split(",")]
+            if len(parts) >= 7:
+                self.samples.append(parts)
+
+    def stop(self):
+        if self.proc is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        self.proc.terminate()          # the exact child started above
+        try:
+            self.proc.wait(timeout=5)
+        except subprocess.TimeoutExpired:
+            self.proc.kill()
+        if self.thread is not None:
+            self.thread.join(timeout=2)
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for s in self.samples:
+            try:
+                sm.append(float(s[0]))
+                mx.append(float(s[1]))
+            except ValueError:
+                continue
+            for name, val in zip(names, s[3:7]):
+                if val.lower().startswith("active"):
+                    reasons.add(name)
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": max(mx) if mx else None,
+                "samples": len(sm), "reasons": sorted(reasons)}
+
+
+def _oracle_stack(x, params, ops, orc):
+    import numpy as np
+    a = x.astype(np.float64)
+    i = 0
+    for op in ops:
+        if op.kind == "conv":
+            w, b = params[i]
+            i += 1
+            s = op.shape
+            a = orc.conv_fwd(a, w, b, stride=s.stride, pad=s.pad, relu=True)
+        else:
+            a = orc.maxpool_fwd(a, op.ksz, op.stride)
+    return a
+
+
+def time_oracle(batch: int, reps: int):
+    """Times the fp64 oracle, as it stands, on the whole stack at the given batch on the host cores."""
+    from oracle import conv_oracle as orc
+    from paper_1606_00094_b200 import workloads as wl
+    x, params = wl.stack_tensors(batch)
+    ops = wl.alexnet_stack(batch)
+    best = float("inf")
+    for _ in range(reps):
+        t0 = time.perf_counter()
+        _oracle_stack(x, params, ops, orc)
+        best = min(best, time.perf_counter() - t0)
+    return wl.stack_flops(batch) / best / 1e9, best, orc.num_threads()
+
+
+def run_reference(args):
+    rank = int(os.environ.get("RANK", "0"))
+    if rank != 0:
+        return
+    from paper_1606_00094_b200 import workloads as wl
+    sample_batch = 4                      # bounded sample of the batch-20 workload: 4 of its 20 images
+    for _ in range(args.warmup):
+        time_oracle(1, 1)
+    times = []
+    threads = 1
+    for _ in range(args.steps):
+        _, t, threads = time_oracle(sample_batch, 1)
+        times.append(t)
+    ms = 1e3 * sum(times) / len(times)
+    value = wl.stack_flops(sample_batch) / (ms * 1e-3) / 1e9
+    sample = f"{sample_batch} of the {BATCH} images of the stack per step (fp64 7-loop oracle, OpenMP over (n,k))"
+    line = {
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": args.gpus, "steps": args.steps,
+        "warmup": args.warmup, "ms_per_step": ms, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": f"alexnet_conv_stack_ungrouped_N{BATCH}", "global_batch": BATCH, "sample": sample},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+        "gpu_launches": 0,
+    }
+    print(json.dumps(line))
+
+
+def run_ours(args):
+    import numpy as np
+    import torch
+    import torch.distributed as dist
+
+    from paper_1606_00094_b200 import binding as B
+    from paper_1606_00094_b200 import workloads as wl
+    from paper_1606_00094_b200.stack import ConvStack
+
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    rank = int(os.environ.get("RANK", "0"))
+    local_rank = int(os.environ.get("LOCAL_RANK", "0"))
+    torch.cuda.set_device(local_rank)
+    if world > 1:
+        os.environ.setdefault("MASTER_ADDR", "127.0.0.1")
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local_rank))
+
+    def barrier():
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    peaks = _peaks()
+    ops = wl.alexnet_stack(BATCH)
+    x_np, params = wl.stack_tensors(BATCH)
+    stack = ConvStack(ops, params, math=B.BODA_MATH_AUTO, tune=1 if args.tune else 0)
+    x_dev = torch.from_numpy(x_np).cuda()
+    x_pin = torch.from_numpy(x_np).pin_memory()
+    out_pin = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+    flush = torch.empty(L2_FLUSH_BYTES // 4, dtype=torch.float32, device="cuda")
+    flops_step = wl.stack_flops(BATCH)
+    n_ops = len(ops)
+
+    def step_events():
+        return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_ops)]
+
+    for _ in range(max(args.warmup, 3)):
+        flush.zero_()
+        stack.forward(x_dev)
+    barrier()
+    assert B.boda_query_status() == 0, "device status word set during warm-up"
+
+    # ---------------- timed region 1: inputs resident in HBM
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    launches0 = B.boda_kernel_launch_count()
+    barrier()
+    step_ev, layer_ev = [], []
+    for _ in range(args.steps):
+        flush.zero_()                                   # evict the 126 MB L2 between steps (not timed)
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        evs = step_events()
+        e0.record()
+        stack.forward(x_dev, events=evs)
+        e1.record()
+        step_ev.append((e0, e1))
+        layer_ev.append(evs)
+    barrier()
+    launches = B.boda_kernel_launch_count() - launches0
+    ms_steps = [a.elapsed_time(b) for a, b in step_ev]
+    total_ms = sum(ms_steps)
+    layer_ms = [sum(layer_ev[s][i][0].elapsed_time(layer_ev[s][i][1]) for s in range(args.steps)) / args.steps
+                for i in range(n_ops)]
+
+    # ---------------- timed region 2: end to end from pinned host buffers
+    for _ in range(2):
+        stack.forward_host(x_pin, out_pin)
+    barrier()
+    e2e_ev = []
+    for _ in range(args.steps):
+        flush.zero_()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        stack.forward_host(x_pin, out_pin)
+        e1.record()
+        e2e_ev.append((e0, e1))
+    barrier()
+    clocks = sampler.stop()
+    e2e_total_ms = sum(a.elapsed_time(b) for a, b in e2e_ev)
+    status = B.boda_query_status()
+    assert status == 0, f"device status word {status}"
+
+    t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device="cuda")
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    total_ms, e2e_total_ms = float(t[0]), float(t[1])
+    ms_per_step = total_ms / args.steps
+    value = world * flops_step / (ms_per_step * 1e-3) / 1e9
+    e2e_value = world * flops_step / (e2e_total_ms / args.steps * 1e-3) / 1e9
+
+    if rank == 0:
+        descs = stack.describe()
+        layers = []
+        for i, op in enumerate(ops):
+            if op.kind == "conv":
+                gf = op.shape.flops / (layer_ms[i] * 1e-3) / 1e9
+                layers.append({"op": f"conv{len([l for l in layers if l['op'].startswith('conv')]) + 1}",
+                               "ms": round(layer_ms[i], 5), "gflops": round(gf, 1), "plan": descs[i]})
+            else:
+                layers.append({"op": "pool", "ms": round(layer_ms[i], 5)})
+        # dominant kernel: the conv layer that takes the most time in the step
+        conv_idx = [i for i, op in enumerate(ops) if op.kind == "conv"]
+        dom = max(conv_idx, key=lambda i: layer_ms[i])
+        dom_tf = ops[dom].shape.flops / (layer_ms[dom] * 1e-3) / 1e12
+        tensor_path = "variant=direct" not in descs[dom]
+        if tensor_path:
+            peak = 0.5 * peaks["bf16_tflops"]      # dense TF32 = half the bf16 rate; measured bf16 burst
+            bound, peak_note = "tensor", f"0.5 x bf16 burst ({peaks['source']})"
+        else:
+            peak = 148 * 128 * 2 * peaks["sm_max_mhz"] * 1e6 / 1e12     # FP32 FMA lanes x 2 x max SM clock
+            bound, peak_note = "alu", "148 SM x 128 FMA/clk x 2 x max SM clock (derived)"
+        traffic = None
+        tpath = os.path.join(ROOT, "profiles", "dominant_kernel_traffic.json")
+        if os.path.exists(tpath):
+            traffic = json.load(open(tpath)).get("dram_bytes_per_launch")
+        roofline = {"bound": bound, "achieved": round(dom_tf, 3), "peak": round(peak, 2), "unit": "TFLOP/s",
+                    "frac": round(dom_tf / peak, 4), "traffic": traffic, "kernel": layers[dom]["op"] + ": " + descs[dom],
+                    "peak_source": peak_note, "launch_ms": round(layer_ms[dom], 5)}
+        cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
+        line = {
+            "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
+            "scaling": "weak", "vs_baseline": None, "dtype": "tf32" if tensor_path else "f32", "data": "synthetic",
+            "config": {"workload": f"alexnet_conv_stack_ungrouped_N{BATCH}", "global_batch": BATCH * world,
+                       "parallelism": f"replicas{world}", "l2": "flushed between steps (512 MiB write)",
+                       "flops_per_step": flops_step},
+            "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(x_np.nbytes),
+                    "d2h_bytes_per_step": int(np.prod(stack.out_shape)) * 4},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roofline,
+            "cpu_baseline": {"value": round(cpu_v, 2) if cpu_v else None, "unit": UNIT, "cores": cpu_threads,
+                             "kind": "oracle", "sample": f"the whole batch-{BATCH} stack, best of 2 ({cpu_t:.2f} s)" if cpu_t else "skipped"},
+            "layers": layers,
+            "frac_of_tf32_peak_whole_step": round(value / 1e3 / (0.5 * peaks["bf16_tflops"]) / world, 4),
+        }
+        print(json.dumps(line))
+    stack.close()
+    if world > 1:
+        dist.destroy_process_group()
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--tune", type=int, default=1, help="time candidate tiles when planning (default on)")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

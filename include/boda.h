@@ -1,0 +1,181 @@
+/*
+ * boda.h - C ABI of the B200 (sm_100a) convolution-forward library.
+ *
+ * The library computes the forward pass of one CNN convolution layer,
+ *
+ *     out[n][k][p][q] = act( bias[k] + sum_{c,r,s} in[n][c][p*stride+r-pad][q*stride+s-pad]
+ *                                                  * filt[k][c][r][s] )
+ *
+ * with zero padding, P = (H + 2*pad - R)/stride + 1 (floor; Q likewise) and act = ReLU or identity.
+ * This is the operation out = conv(in, filts) of Section 2 of the Boda-RTC paper (arXiv 1606.00094):
+ * the window of `in` for an output point starts at (oy*stride, ox*stride) of the (padded) input and
+ * spans all input channels; the output is the sum of the element-wise product of that window and
+ * the filter slice of the output channel (a cross-correlation, no flip); ReLU = max(0, x) is fused
+ * into the operation.  The bias, which the paper sets aside, is a per-output-channel constant added
+ * before the activation.
+ *
+ * Conventions that hold for every entry point unless stated otherwise
+ *   - Tensor pointers are DEVICE pointers to dense, row-major fp32 arrays owned by the caller:
+ *       in [N][C][H][W], filt [K][C][R][S], bias [K] (NULL means no bias), out [N][K][P][Q].
+ *     They must be at least 16-byte aligned; `out` must not overlap any input.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the default stream).  Calls enqueue work
+ *     and return; they do not synchronise unless the comment says so.
+ *   - Every function returns a boda_status (0 = success).  Nothing throws across the ABI.
+ *   - The library keeps per-device caches (plans made by boda_conv_fwd, packed operands); they are
+ *     protected by one mutex, so calls may come from several host threads.
+ *   - Not supported, and reported as an error rather than silently mis-computed: groups, dilation,
+ *     different stride or padding per spatial dimension (the paper restricts itself to scalar
+ *     kernel size and stride; R != S is accepted).
+ */
+#ifndef BODA_H_
+#define BODA_H_
+
+#include <stddef.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum boda_status {
+    BODA_OK = 0,
+    BODA_ERR_INVALID_ARG = 1,    /* NULL pointer, non-positive extent, stride < 1, pad < 0, window larger than padded input */
+    BODA_ERR_UNSUPPORTED = 2,    /* device is not sm_100, or a forced variant / tile is illegal for the shape */
+    BODA_ERR_CUDA = 3,           /* a CUDA runtime or driver call failed; boda_last_error_string() has the text */
+    BODA_ERR_DEVICE_TIMEOUT = 4, /* a bounded wait inside a kernel expired (reported by boda_query_status) */
+    BODA_ERR_NOMEM = 5,          /* device or host allocation failed, or the workspace given is too small */
+    BODA_ERR_TOO_LARGE = 6       /* a size exceeds a fixed capacity stated by the entry point */
+} boda_status;
+
+/* Kernel variants.  The names follow Section 5 of the paper: `conv` (implicit-GEMM fallback, here an
+ * FP32 CUDA-core kernel called DIRECT), `k1conv` (kernel size 1: a plain GEMM over input channels)
+ * and `tconv` (tiled convolution for kernel sizes 2..11).  K1CONV and TCONV run on the tcgen05
+ * tensor cores in TF32 with fp32 accumulation. */
+enum { BODA_VARIANT_AUTO = -1, BODA_VARIANT_DIRECT = 0, BODA_VARIANT_K1CONV = 1, BODA_VARIANT_TCONV = 2 };
+
+/* Arithmetic the plan may use. */
+enum { BODA_MATH_AUTO = 0,       /* TF32 tensor cores where a tensor-core variant applies */
+       BODA_MATH_FP32 = 1,       /* FP32 FMA only (DIRECT); relative L2 error vs fp64 <= 1e-5 */
+       BODA_MATH_TF32 = 2 };     /* TF32 operands, fp32 accumulate; relative L2 error <= 5e-3 */
+
+typedef struct boda_conv_shape {
+    int N, C, H, W;              /* input  [N][C][H][W] */
+    int K, R, S;                 /* filters [K][C][R][S] */
+    int stride, pad;             /* same in both spatial dimensions; zero padding */
+    int relu;                    /* 0: identity, otherwise max(0, x) */
+} boda_conv_shape;
+
+typedef struct boda_plan_opts {
+    int math;                    /* BODA_MATH_* */
+    int tune;                    /* 0: pick variant and tile by rule; 1: time the candidates on the device (synchronises) */
+    int variant;                 /* BODA_VARIANT_AUTO or a forced variant (used by tests) */
+    int tile_id;                 /* -1: automatic; otherwise index into the variant's tile table */
+    int split_k;                 /* 0: automatic; otherwise the number of reduction splits of a tensor-core variant */
+    int device;                  /* CUDA device ordinal; -1: the current device */
+} boda_plan_opts;
+
+typedef struct boda_conv_plan boda_conv_plan;   /* opaque; created and destroyed by the library */
+
+/* Output extent of one spatial dimension, 1 + (in + 2*pad - ksz)/stride with floor division
+ * (Section 2: out_X = 1 + (in_X - KSZ)/stride on the padded input).  Returns 0 if the window does
+ * not fit.  Host-only helper. */
+int boda_conv_out_dim(int in_dim, int ksz, int stride, int pad);
+
+/* Fill *opts with the defaults (automatic everything, current device). */
+void boda_plan_opts_default(boda_plan_opts* opts);
+
+/*
+ * Variant selection and blocking for one layer shape: the analogue of the paper's flow
+ * "operation -> variant -> blocking constants" (Section 4, Figure "codegen", and the variant rules
+ * of Section 5: k1conv for kernel size 1, tconv for kernel sizes 2..11, conv otherwise).  With
+ * opts->tune != 0 the legal candidates are timed on scratch buffers and the fastest is kept (the
+ * automated tuning the paper names as future work); this synchronises the device.
+ * `opts` may be NULL (defaults).  On success *plan owns device memory (index tables, packed filter
+ * storage, workspace); destroy it with boda_conv_plan_destroy.
+ * Errors: INVALID_ARG (bad shape), UNSUPPORTED (forced variant illegal, device not sm_100), CUDA, NOMEM.
+ */
+int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* opts, boda_conv_plan** plan);
+
+/* Frees everything the plan owns.  The caller must make sure no launch that uses it is in flight. */
+int boda_conv_plan_destroy(boda_conv_plan* plan);
+
+/* Writes a NUL-terminated one-line description (variant, tile, split, math, workspace) into buf. */
+int boda_conv_plan_describe(const boda_conv_plan* plan, char* buf, size_t buf_bytes);
+
+/* Bytes of caller-provided scratch that boda_conv_fwd_planned needs (0 if none).  The scratch holds
+ * the re-laid-out input (the "input transformation" that the paper's k1conv and tconv apply, Section 5)
+ * and split-reduction partial sums. */
+size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* plan);
+
+/*
+ * Optional: pre-pack the filters (and remember the bias pointer's contents are NOT copied) for a
+ * tensor-core plan, so that boda_conv_fwd_planned can skip the per-call filter re-layout.  Weights
+ * are constants at deployment time (Section 2 speaks of deployment / inference).  After binding,
+ * the `filt` argument of boda_conv_fwd_planned is ignored when it equals the bound pointer; passing
+ * a different pointer re-packs on that call.  Enqueues on `stream`.
+ */
+int boda_conv_plan_bind_filters(boda_conv_plan* plan, const float* filt, void* stream);
+
+/*
+ * The forward pass with an explicit plan.  `workspace` must point to at least
+ * boda_conv_plan_workspace_bytes(plan) bytes of device memory, 256-byte aligned (NULL if 0 bytes);
+ * it may be shared between plans whose launches are ordered on one stream.  No allocation and no
+ * synchronisation happen here.  The same plan must not be used from two streams at once.
+ * Errors: INVALID_ARG (NULL tensor), CUDA (launch failure).
+ */
+int boda_conv_fwd_planned(boda_conv_plan* plan, const float* in, const float* filt, const float* bias,
+                          float* out, void* workspace, void* stream);
+
+/*
+ * The forward pass in one call (the signature named by the build's specification).  Looks up, or
+ * creates with default options, a plan for the shape on the current device and an internal
+ * workspace, then launches on `stream`.  The first call for a shape allocates; later calls do not.
+ */
+int boda_conv_fwd(const float* in, const float* filt, const float* bias, float* out,
+                  int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int relu,
+                  void* stream);
+
+/*
+ * Same operation with HOST pointers: copies in / filt / bias to device staging buffers kept by the
+ * library, runs the planned kernel(s) and copies `out` back, all on `stream`, then synchronises the
+ * stream so that `out` is valid on return.  Pinned host memory makes the copies asynchronous.
+ */
+int boda_conv_fwd_host(const float* in_host, const float* filt_host, const float* bias_host, float* out_host,
+                       int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int relu,
+                       void* stream);
+
+/*
+ * Max-pooling, ksz x ksz window, given stride, no padding, floor output extent; the pooling that
+ * sits between the convolutions of the AlexNet-shaped stack (the paper lists pooling among the
+ * deployment operations, Section 2, without analysing it).  in [N][C][H][W] -> out [N][C][P][Q],
+ * device pointers.
+ */
+int boda_maxpool_fwd(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,
+                     void* stream);
+
+/*
+ * Reads the device-side status word of the current device: kernels never trap or spin for ever;
+ * a bounded wait that expires records BODA_ERR_DEVICE_TIMEOUT there and the kernel returns.
+ * Synchronises `stream`, copies the word to *device_status (BODA_OK if nothing was recorded) and
+ * clears it.
+ */
+int boda_query_status(void* stream, int* device_status);
+
+/* Releases the per-device caches made by boda_conv_fwd / boda_conv_fwd_host (plans, workspaces). */
+int boda_clear_caches(void);
+
+const char* boda_status_string(int status);
+
+/* Text of the last CUDA error seen by the calling thread ("" if none). */
+const char* boda_last_error_string(void);
+
+/* Number of kernels this library has launched in this process so far (all devices, all threads).
+ * A counter for benchmarks and tests that want to state how much of the work ran in these kernels. */
+unsigned long long boda_kernel_launch_count(void);
+
+/* Library version, e.g. 100 for 0.1.0. */
+int boda_version(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* BODA_H_ */

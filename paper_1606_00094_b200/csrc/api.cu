@@ -1,0 +1,466 @@
+// C ABI: plans (variant selection + blocking), the forward entry points, caches and status.
+#include <atomic>
+#include <cstdio>
+#include <cstring>
+#include <map>
+#include <mutex>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "boda_internal.h"
+#include "igemm_tf32.h"
+
+namespace boda {
+
+static thread_local std::string t_last_error;
+static std::atomic<unsigned long long> g_launches{0};
+
+void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
+unsigned long long launch_count() { return g_launches.load(std::memory_order_relaxed); }
+
+int record_cuda_error(cudaError_t e, const char* what)
+{
+    t_last_error = std::string(cudaGetErrorName(e)) + ": " + cudaGetErrorString(e) + " in " + what;
+    (void)cudaGetLastError();   // clear the sticky-less error state
+    return BODA_ERR_CUDA;
+}
+
+namespace {
+
+struct DeviceCtx {
+    int device = -1;
+    int cc_major = 0;
+    int* d_status = nullptr;          // STATUS_WORDS ints
+};
+
+struct ShapeKey {
+    int v[11];
+    bool operator<(const ShapeKey& o) const { return std::memcmp(v, o.v, sizeof(v)) < 0; }
+};
+
+struct CachedEntry {
+    boda_conv_plan* plan = nullptr;
+    void* workspace = nullptr;
+    // device staging for the host-pointer entry point
+    float *s_in = nullptr, *s_filt = nullptr, *s_bias = nullptr, *s_out = nullptr;
+};
+
+std::mutex g_mutex;
+std::map<int, DeviceCtx> g_ctx;
+std::map<ShapeKey, CachedEntry> g_cache;
+
+int get_ctx(int device, DeviceCtx** out)
+{
+    if (device < 0) BODA_CUDA_TRY(cudaGetDevice(&device));
+    auto it = g_ctx.find(device);
+    if (it == g_ctx.end()) {
+        DeviceCtx c;
+        c.device = device;
+        int major = 0;
+        BODA_CUDA_TRY(cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, device));
+        c.cc_major = major;
+        int prev = 0;
+        BODA_CUDA_TRY(cudaGetDevice(&prev));
+        BODA_CUDA_TRY(cudaSetDevice(device));
+        cudaError_t e = cudaMalloc(&c.d_status, STATUS_WORDS * sizeof(int));
+        if (e == cudaSuccess) e = cudaMemset(c.d_status, 0, STATUS_WORDS * sizeof(int));
+        (void)cudaSetDevice(prev);
+        if (e != cudaSuccess) return record_cuda_error(e, "status word allocation");
+        it = g_ctx.emplace(device, c).first;
+    }
+    *out = &it->second;
+    return BODA_OK;
+}
+
+bool shape_ok(const boda_conv_shape& s)
+{
+    if (s.N <= 0 || s.C <= 0 || s.H <= 0 || s.W <= 0 || s.K <= 0 || s.R <= 0 || s.S <= 0) return false;
+    if (s.stride < 1 || s.pad < 0) return false;
+    if (s.R >= 0x4000 || s.S >= 0x4000) return false;
+    if (boda_conv_out_dim(s.H, s.R, s.stride, s.pad) <= 0) return false;
+    if (boda_conv_out_dim(s.W, s.S, s.stride, s.pad) <= 0) return false;
+    const long long lim = 0x7fffffffLL;
+    const long long P = boda_conv_out_dim(s.H, s.R, s.stride, s.pad), Q = boda_conv_out_dim(s.W, s.S, s.stride, s.pad);
+    if ((long long)s.N * s.C * s.H * s.W > lim) return false;
+    if ((long long)s.K * s.C * s.R * s.S > lim) return false;
+    if ((long long)s.N * s.K * P * Q > lim) return false;
+    return true;
+}
+
+}  // namespace
+}  // namespace boda
+
+using namespace boda;
+
+struct boda_conv_plan {
+    boda_conv_shape shape;
+    ConvDims d;
+    int device = 0;
+    int variant = BODA_VARIANT_DIRECT;
+    int tile_id = 0;
+    int math = BODA_MATH_FP32;
+    int* d_status = nullptr;
+    DirectTapEntry* d_tab = nullptr;     // DIRECT
+    IgemmPlan* ig = nullptr;             // K1CONV / TCONV
+    size_t ws_bytes = 0;
+};
+
+extern "C" {
+
+int boda_conv_out_dim(int in_dim, int ksz, int stride, int pad)
+{
+    if (in_dim <= 0 || ksz <= 0 || stride <= 0 || pad < 0) return 0;
+    const long long padded = (long long)in_dim + 2LL * pad;
+    if (padded < ksz) return 0;
+    return (int)((padded - ksz) / stride + 1);
+}
+
+void boda_plan_opts_default(boda_plan_opts* o)
+{
+    if (!o) return;
+    o->math = BODA_MATH_AUTO;
+    o->tune = 0;
+    o->variant = BODA_VARIANT_AUTO;
+    o->tile_id = -1;
+    o->split_k = 0;
+    o->device = -1;
+}
+
+int boda_conv_plan_destroy(boda_conv_plan* plan)
+{
+    if (!plan) return BODA_OK;
+    int prev = 0;
+    (void)cudaGetDevice(&prev);
+    (void)cudaSetDevice(plan->device);
+    if (plan->d_tab) (void)cudaFree(plan->d_tab);
+    if (plan->ig) igemm_plan_destroy(plan->ig);
+    (void)cudaSetDevice(prev);
+    delete plan;
+    return BODA_OK;
+}
+
+static int plan_time_ms(boda_conv_plan* plan, float* ms_out);
+
+static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, DeviceCtx* ctx, int variant,
+                      int tile_id, int split_k, boda_conv_plan** out)
+{
+    boda_conv_plan* p = new (std::nothrow) boda_conv_plan();
+    if (!p) return BODA_ERR_NOMEM;
+    p->shape = shape;
+    p->d = make_dims(shape);
+    p->device = ctx->device;
+    p->d_status = ctx->d_status;
+    p->variant = variant;
+    int rc = BODA_OK;
+    if (variant == BODA_VARIANT_DIRECT) {
+        p->math = BODA_MATH_FP32;
+        if (tile_id >= direct_num_tiles()) { delete p; return BODA_ERR_UNSUPPORTED; }
+        p->tile_id = tile_id >= 0 ? tile_id : direct_pick_tile(p->d);
+        const int len = direct_table_len(p->d);
+        std::vector<DirectTapEntry> tab(len);
+        direct_build_table(p->d, tab.data());
+        cudaError_t e = cudaMalloc(&p->d_tab, len * sizeof(DirectTapEntry));
+        if (e == cudaSuccess)
+            e = cudaMemcpy(p->d_tab, tab.data(), len * sizeof(DirectTapEntry), cudaMemcpyHostToDevice);
+        if (e != cudaSuccess) rc = record_cuda_error(e, "tap table upload");
+        p->ws_bytes = 0;
+    } else {
+        p->math = BODA_MATH_TF32;
+        rc = igemm_plan_create(p->d, variant, tile_id, split_k, ctx->d_status, &p->ig);
+        if (rc == BODA_OK) { p->tile_id = igemm_plan_tile(p->ig); p->ws_bytes = igemm_plan_workspace_bytes(p->ig); }
+    }
+    if (rc != BODA_OK) { boda_conv_plan_destroy(p); return rc; }
+    *out = p;
+    (void)o;
+    return BODA_OK;
+}
+
+int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* opts, boda_conv_plan** plan)
+{
+    if (!shape || !plan) return BODA_ERR_INVALID_ARG;
+    *plan = nullptr;
+    if (!shape_ok(*shape)) return BODA_ERR_INVALID_ARG;
+    boda_plan_opts o;
+    boda_plan_opts_default(&o);
+    if (opts) o = *opts;
+    if (o.math < BODA_MATH_AUTO || o.math > BODA_MATH_TF32) return BODA_ERR_INVALID_ARG;
+    if (o.variant < BODA_VARIANT_AUTO || o.variant > BODA_VARIANT_TCONV) return BODA_ERR_INVALID_ARG;
+
+    std::lock_guard<std::mutex> lock(g_mutex);
+    DeviceCtx* ctx = nullptr;
+    int rc = get_ctx(o.device, &ctx);
+    if (rc != BODA_OK) return rc;
+    if (ctx->cc_major != 10) return BODA_ERR_UNSUPPORTED;
+    int prev = 0;
+    BODA_CUDA_TRY(cudaGetDevice(&prev));
+    BODA_CUDA_TRY(cudaSetDevice(ctx->device));
+
+    const ConvDims d = make_dims(*shape);
+    // Variant rules of Section 5: kernel size 1 -> k1conv; kernel sizes 2..11 -> tconv; else conv.
+    const bool k1_legal = igemm_variant_legal(d, BODA_VARIANT_K1CONV);
+    const bool t_legal = igemm_variant_legal(d, BODA_VARIANT_TCONV);
+    int variant = o.variant;
+    if (variant == BODA_VARIANT_AUTO) {
+        if (o.math == BODA_MATH_FP32) variant = BODA_VARIANT_DIRECT;
+        else if (k1_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_K1CONV;
+        else if (t_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_TCONV;
+        else variant = BODA_VARIANT_DIRECT;
+    }
+    if ((variant == BODA_VARIANT_K1CONV && !k1_legal) || (variant == BODA_VARIANT_TCONV && !t_legal) ||
+        (variant != BODA_VARIANT_DIRECT && o.math == BODA_MATH_FP32)) {
+        (void)cudaSetDevice(prev);
+        return BODA_ERR_UNSUPPORTED;
+    }
+
+    if (!o.tune || o.tile_id >= 0) {
+        rc = plan_build(*shape, o, ctx, variant, o.tile_id, o.split_k, plan);
+    } else {
+        // Automated tuning: time every tile (and split) of the chosen variant, keep the fastest.
+        boda_conv_plan* best = nullptr;
+        float best_ms = 1e30f;
+        const int ntiles = variant == BODA_VARIANT_DIRECT ? direct_num_tiles() : igemm_num_tiles();
+        for (int t = 0; t < ntiles; ++t) {
+            const int nsplit = variant == BODA_VARIANT_DIRECT ? 1 : igemm_num_split_candidates();
+            for (int si = 0; si < nsplit; ++si) {
+                const int split = variant == BODA_VARIANT_DIRECT ? 0 : igemm_split_candidate(si);
+                if (o.split_k > 0 && split != o.split_k) continue;
+                boda_conv_plan* cand = nullptr;
+                if (plan_build(*shape, o, ctx, variant, t, split, &cand) != BODA_OK) continue;
+                float ms = 0.f;
+                if (plan_time_ms(cand, &ms) == BODA_OK && ms < best_ms) {
+                    if (best) boda_conv_plan_destroy(best);
+                    best = cand;
+                    best_ms = ms;
+                } else {
+                    boda_conv_plan_destroy(cand);
+                }
+            }
+        }
+        if (best) { *plan = best; rc = BODA_OK; }
+        else rc = plan_build(*shape, o, ctx, variant, -1, o.split_k, plan);
+    }
+    (void)cudaSetDevice(prev);
+    return rc;
+}
+
+int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
+{
+    if (!p || !buf || n == 0) return BODA_ERR_INVALID_ARG;
+    static const char* vn[] = {"direct", "k1conv", "tconv"};
+    if (p->variant == BODA_VARIANT_DIRECT) {
+        std::snprintf(buf, n, "variant=%s tile=%s(id %d) math=fp32 split_k=1 workspace=%zu", vn[p->variant],
+                      direct_tile_name(p->tile_id), p->tile_id, p->ws_bytes);
+    } else {
+        char tmp[160];
+        igemm_plan_describe(p->ig, tmp, sizeof(tmp));
+        std::snprintf(buf, n, "variant=%s %s math=tf32 workspace=%zu", vn[p->variant], tmp, p->ws_bytes);
+    }
+    return BODA_OK;
+}
+
+size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* p) { return p ? p->ws_bytes : 0; }
+
+int boda_conv_plan_bind_filters(boda_conv_plan* p, const float* filt, void* stream)
+{
+    if (!p || !filt) return BODA_ERR_INVALID_ARG;
+    if (p->variant == BODA_VARIANT_DIRECT) return BODA_OK;   // reads KCRS in place
+    return igemm_bind_filters(p->ig, filt, (cudaStream_t)stream);
+}
+
+int boda_conv_fwd_planned(boda_conv_plan* p, const float* in, const float* filt, const float* bias, float* out,
+                          void* workspace, void* stream)
+{
+    if (!p || !in || !out) return BODA_ERR_INVALID_ARG;
+    if (p->variant == BODA_VARIANT_DIRECT) {
+        if (!filt) return BODA_ERR_INVALID_ARG;
+        return direct_launch(p->d, p->tile_id, in, filt, bias, out, p->d_tab, (cudaStream_t)stream);
+    }
+    if (p->ws_bytes && !workspace) return BODA_ERR_NOMEM;
+    return igemm_launch(p->ig, in, filt, bias, out, workspace, (cudaStream_t)stream);
+}
+
+}  // extern "C"
+
+// Times one plan on scratch buffers (used by the tuner).  Synchronises.
+static int plan_time_ms(boda_conv_plan* p, float* ms_out)
+{
+    const ConvDims& d = p->d;
+    const size_t n_in = (size_t)d.N * d.C * d.H * d.W, n_f = (size_t)d.K * d.Kred, n_out = (size_t)d.M * d.K;
+    float *in = nullptr, *f = nullptr, *b = nullptr, *out = nullptr;
+    void* ws = nullptr;
+    int rc = BODA_OK;
+    cudaEvent_t e0 = nullptr, e1 = nullptr;
+    auto cleanup = [&]() {
+        if (in) cudaFree(in); if (f) cudaFree(f); if (b) cudaFree(b); if (out) cudaFree(out); if (ws) cudaFree(ws);
+        if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1);
+    };
+#define TRY_T(x) do { cudaError_t _e = (x); if (_e != cudaSuccess) { rc = record_cuda_error(_e, #x); cleanup(); return rc; } } while (0)
+    TRY_T(cudaMalloc(&in, n_in * 4)); TRY_T(cudaMalloc(&f, n_f * 4)); TRY_T(cudaMalloc(&b, d.K * 4));
+    TRY_T(cudaMalloc(&out, n_out * 4));
+    if (p->ws_bytes) TRY_T(cudaMalloc(&ws, p->ws_bytes));
+    TRY_T(cudaMemset(in, 0, n_in * 4)); TRY_T(cudaMemset(f, 0, n_f * 4)); TRY_T(cudaMemset(b, 0, d.K * 4));
+    TRY_T(cudaEventCreate(&e0)); TRY_T(cudaEventCreate(&e1));
+    if (p->variant != BODA_VARIANT_DIRECT) { rc = igemm_bind_filters(p->ig, f, 0); if (rc) { cleanup(); return rc; } }
+    for (int i = 0; i < 2; ++i) { rc = boda_conv_fwd_planned(p, in, f, b, out, ws, nullptr); if (rc) { cleanup(); return rc; } }
+    TRY_T(cudaStreamSynchronize(0));
+    const int iters = 10;
+    TRY_T(cudaEventRecord(e0, 0));
+    for (int i = 0; i < iters; ++i) { rc = boda_conv_fwd_planned(p, in, f, b, out, ws, nullptr); if (rc) { cleanup(); return rc; } }
+    TRY_T(cudaEventRecord(e1, 0));
+    TRY_T(cudaEventSynchronize(e1));
+    float ms = 0.f;
+    TRY_T(cudaEventElapsedTime(&ms, e0, e1));
+    int st[STATUS_WORDS] = {0, 0, 0, 0};
+    TRY_T(cudaMemcpy(st, p->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+    if (st[0] != 0) { (void)cudaMemset(p->d_status, 0, sizeof(st)); cleanup(); return st[0]; }
+    if (p->variant != BODA_VARIANT_DIRECT) igemm_unbind_filters(p->ig);
+#undef TRY_T
+    cleanup();
+    *ms_out = ms / iters;
+    return BODA_OK;
+}
+
+extern "C" {
+
+static int cache_lookup(const boda_conv_shape& s, bool need_staging, CachedEntry** out)
+{
+    int device = 0;
+    BODA_CUDA_TRY(cudaGetDevice(&device));
+    ShapeKey key;
+    const int vals[11] = {device, s.N, s.C, s.H, s.W, s.K, s.R, s.S, s.stride, s.pad, s.relu ? 1 : 0};
+    std::memcpy(key.v, vals, sizeof(vals));
+    CachedEntry* e = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto it = g_cache.find(key);
+        if (it != g_cache.end()) e = &it->second;
+    }
+    if (!e) {
+        boda_conv_plan* plan = nullptr;
+        int rc = boda_conv_plan_create(&s, nullptr, &plan);
+        if (rc != BODA_OK) return rc;
+        CachedEntry ne;
+        ne.plan = plan;
+        if (plan->ws_bytes) {
+            cudaError_t ce = cudaMalloc(&ne.workspace, plan->ws_bytes);
+            if (ce != cudaSuccess) { boda_conv_plan_destroy(plan); return record_cuda_error(ce, "workspace allocation"); }
+        }
+        std::lock_guard<std::mutex> lock(g_mutex);
+        auto ins = g_cache.emplace(key, ne);
+        if (!ins.second) {   // another thread won the race
+            if (ne.workspace) cudaFree(ne.workspace);
+            boda_conv_plan_destroy(plan);
+        }
+        e = &ins.first->second;
+    }
+    if (need_staging && !e->s_in) {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        if (!e->s_in) {
+            const ConvDims& d = e->plan->d;
+            BODA_CUDA_TRY(cudaMalloc(&e->s_in, (size_t)d.N * d.C * d.H * d.W * 4));
+            BODA_CUDA_TRY(cudaMalloc(&e->s_filt, (size_t)d.K * d.Kred * 4));
+            BODA_CUDA_TRY(cudaMalloc(&e->s_bias, (size_t)d.K * 4));
+            BODA_CUDA_TRY(cudaMalloc(&e->s_out, (size_t)d.M * d.K * 4));
+        }
+    }
+    *out = e;
+    return BODA_OK;
+}
+
+int boda_conv_fwd(const float* in, const float* filt, const float* bias, float* out, int N, int C, int H, int W,
+                  int K, int R, int S, int stride, int pad, int relu, void* stream)
+{
+    if (!in || !filt || !out) return BODA_ERR_INVALID_ARG;
+    const boda_conv_shape s = {N, C, H, W, K, R, S, stride, pad, relu};
+    if (!shape_ok(s)) return BODA_ERR_INVALID_ARG;
+    CachedEntry* e = nullptr;
+    int rc = cache_lookup(s, false, &e);
+    if (rc != BODA_OK) return rc;
+    return boda_conv_fwd_planned(e->plan, in, filt, bias, out, e->workspace, stream);
+}
+
+int boda_conv_fwd_host(const float* in, const float* filt, const float* bias, float* out, int N, int C, int H,
+                       int W, int K, int R, int S, int stride, int pad, int relu, void* stream)
+{
+    if (!in || !filt || !out) return BODA_ERR_INVALID_ARG;
+    const boda_conv_shape s = {N, C, H, W, K, R, S, stride, pad, relu};
+    if (!shape_ok(s)) return BODA_ERR_INVALID_ARG;
+    CachedEntry* e = nullptr;
+    int rc = cache_lookup(s, true, &e);
+    if (rc != BODA_OK) return rc;
+    const ConvDims& d = e->plan->d;
+    cudaStream_t st = (cudaStream_t)stream;
+    BODA_CUDA_TRY(cudaMemcpyAsync(e->s_in, in, (size_t)d.N * d.C * d.H * d.W * 4, cudaMemcpyHostToDevice, st));
+    BODA_CUDA_TRY(cudaMemcpyAsync(e->s_filt, filt, (size_t)d.K * d.Kred * 4, cudaMemcpyHostToDevice, st));
+    if (bias) BODA_CUDA_TRY(cudaMemcpyAsync(e->s_bias, bias, (size_t)d.K * 4, cudaMemcpyHostToDevice, st));
+    if (e->plan->ig) igemm_unbind_filters(e->plan->ig);   // the staged filters may have changed
+    rc = boda_conv_fwd_planned(e->plan, e->s_in, e->s_filt, bias ? e->s_bias : nullptr, e->s_out, e->workspace, stream);
+    if (rc != BODA_OK) return rc;
+    BODA_CUDA_TRY(cudaMemcpyAsync(out, e->s_out, (size_t)d.M * d.K * 4, cudaMemcpyDeviceToHost, st));
+    BODA_CUDA_TRY(cudaStreamSynchronize(st));
+    return BODA_OK;
+}
+
+int boda_maxpool_fwd(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride, void* stream)
+{
+    if (!in || !out || N <= 0 || C <= 0 || ksz <= 0 || stride <= 0) return BODA_ERR_INVALID_ARG;
+    if (boda_conv_out_dim(H, ksz, stride, 0) <= 0 || boda_conv_out_dim(W, ksz, stride, 0) <= 0)
+        return BODA_ERR_INVALID_ARG;
+    return maxpool_launch(in, out, N, C, H, W, ksz, stride, (cudaStream_t)stream);
+}
+
+int boda_query_status(void* stream, int* device_status)
+{
+    if (!device_status) return BODA_ERR_INVALID_ARG;
+    DeviceCtx* ctx = nullptr;
+    {
+        std::lock_guard<std::mutex> lock(g_mutex);
+        int rc = get_ctx(-1, &ctx);
+        if (rc != BODA_OK) return rc;
+    }
+    BODA_CUDA_TRY(cudaStreamSynchronize((cudaStream_t)stream));
+    int st[STATUS_WORDS] = {0, 0, 0, 0};
+    BODA_CUDA_TRY(cudaMemcpy(st, ctx->d_status, sizeof(st), cudaMemcpyDeviceToHost));
+    if (st[0] != 0) BODA_CUDA_TRY(cudaMemset(ctx->d_status, 0, sizeof(st)));
+    *device_status = st[0];
+    return BODA_OK;
+}
+
+int boda_clear_caches(void)
+{
+    std::lock_guard<std::mutex> lock(g_mutex);
+    for (auto& kv : g_cache) {
+        CachedEntry& e = kv.second;
+        if (e.workspace) cudaFree(e.workspace);
+        if (e.s_in) cudaFree(e.s_in);
+        if (e.s_filt) cudaFree(e.s_filt);
+        if (e.s_bias) cudaFree(e.s_bias);
+        if (e.s_out) cudaFree(e.s_out);
+        boda_conv_plan_destroy(e.plan);
+    }
+    g_cache.clear();
+    return BODA_OK;
+}
+
+const char* boda_status_string(int s)
+{
+    switch (s) {
+        case BODA_OK: return "ok";
+        case BODA_ERR_INVALID_ARG: return "invalid argument";
+        case BODA_ERR_UNSUPPORTED: return "unsupported (device is not sm_100, or variant illegal for the shape)";
+        case BODA_ERR_CUDA: return "CUDA error";
+        case BODA_ERR_DEVICE_TIMEOUT: return "a bounded wait inside a kernel expired";
+        case BODA_ERR_NOMEM: return "out of memory or workspace missing";
+        case BODA_ERR_TOO_LARGE: return "size exceeds a fixed capacity";
+        default: return "unknown status";
+    }
+}
+
+const char* boda_last_error_string(void) { return t_last_error.c_str(); }
+
+unsigned long long boda_kernel_launch_count(void) { return boda::launch_count(); }
+
+int boda_version(void) { return 100; }
+
+}  // extern "C"

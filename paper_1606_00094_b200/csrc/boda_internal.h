@@ -1,0 +1,65 @@
+// Internal declarations shared by the translation units of the library (not part of the ABI).
+#pragma once
+
+#include <cuda_runtime.h>
+#include <stddef.h>
+#include <stdint.h>
+
+#include "boda.h"
+
+namespace boda {
+
+// Device status word layout (int[4]): [0] status code, [1] where (kernel id), [2] block, [3] detail.
+enum { STATUS_WORDS = 4 };
+enum { KERNEL_ID_DIRECT = 1, KERNEL_ID_IGEMM = 2, KERNEL_ID_PACK = 3 };
+
+struct ConvDims {
+    int N, C, H, W, K, R, S, stride, pad, relu;
+    int P, Q;
+    int M;        // N*P*Q output points per channel ("pixels")
+    int Kred;     // C*R*S reduction length
+};
+
+inline ConvDims make_dims(const boda_conv_shape& s) {
+    ConvDims d;
+    d.N = s.N; d.C = s.C; d.H = s.H; d.W = s.W; d.K = s.K; d.R = s.R; d.S = s.S;
+    d.stride = s.stride; d.pad = s.pad; d.relu = s.relu ? 1 : 0;
+    d.P = boda_conv_out_dim(s.H, s.R, s.stride, s.pad);
+    d.Q = boda_conv_out_dim(s.W, s.S, s.stride, s.pad);
+    d.M = s.N * d.P * d.Q;
+    d.Kred = s.C * s.R * s.S;
+    return d;
+}
+
+// Bumps the process-wide count of kernels launched by the library.
+void count_launch(int n = 1);
+
+// Records the last CUDA error text for boda_last_error_string(); returns BODA_ERR_CUDA.
+int record_cuda_error(cudaError_t e, const char* what);
+
+#define BODA_CUDA_TRY(expr)                                                  \
+    do {                                                                     \
+        cudaError_t _e = (expr);                                             \
+        if (_e != cudaSuccess) return ::boda::record_cuda_error(_e, #expr);  \
+    } while (0)
+
+// ---- DIRECT (FP32 CUDA-core) variant -----------------------------------------------------------
+// Reduction-index table entry: for flattened reduction index j = (c*R + r)*S + s the element offset
+// c*H*W + r*W + s inside one image and the tap (r, s); entries past C*R*S have r = 0x4000 so that
+// the bounds test fails and the element counts as padding.
+struct DirectTapEntry { int offset; int rs; };
+
+int direct_num_tiles();
+const char* direct_tile_name(int tile_id);
+int direct_pick_tile(const ConvDims& d);
+// Length (entries) of the table the tile needs; build it on the host into `host_tab`.
+int direct_table_len(const ConvDims& d);
+void direct_build_table(const ConvDims& d, DirectTapEntry* host_tab);
+int direct_launch(const ConvDims& d, int tile_id, const float* in, const float* filt, const float* bias,
+                  float* out, const DirectTapEntry* dev_tab, cudaStream_t stream);
+
+// ---- pooling -------------------------------------------------------------------------------------
+int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,
+                   cudaStream_t stream);
+
+}  // namespace boda

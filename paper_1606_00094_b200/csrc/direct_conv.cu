@@ -1,0 +1,259 @@
+// DIRECT variant: FP32 CUDA-core convolution, the general fallback (the paper's `conv`, Section 5:
+// SGEMM blocking with im2col folded into the shared-memory load) and the small-input-channel path.
+//
+// Blocking follows the paper's SGEMM template (Section 4, Listing 1 and the parameter list after
+// it): each thread owns a register tile of Mt x Nt outputs (here TM pixels x TN output channels),
+// a thread block of 256 threads owns Mb*Mt x Nb*Nt = (16*TM) x (16*TN) outputs, the reduction is
+// walked in chunks of Kb = 8, operands of a chunk are staged in shared memory and the inner loop
+// is fully unrolled.  The gather that im2col would do is a table lookup: entry j of the table
+// gives, for reduction index j = (c, r, s), the element offset inside an image and the tap, so the
+// load needs no division.  Bias and ReLU are applied in registers before the store.
+#include "boda_internal.h"
+
+namespace boda {
+namespace {
+
+constexpr int kThreads = 256;
+constexpr int BK = 8;
+
+template <int TM, int TN>
+__global__ void __launch_bounds__(kThreads)
+direct_conv_kernel(const ConvDims d, const float* __restrict__ in, const float* __restrict__ filt,
+                   const float* __restrict__ bias, float* __restrict__ out,
+                   const DirectTapEntry* __restrict__ tab)
+{
+    constexpr int BM = 16 * TM;
+    constexpr int BN = 16 * TN;
+    constexpr int BNP = BN + 4;                       // padded pitch: conflict-free transposed store
+    constexpr int A_PER_THREAD = (BK * BM + kThreads - 1) / kThreads;
+    constexpr int B_PER_THREAD = (BK * BN + kThreads - 1) / kThreads;
+    static_assert(kThreads % BM == 0 || BM % kThreads == 0, "a thread keeps one pixel for all its A loads");
+
+    __shared__ __align__(16) float As[2][BK][BM];
+    __shared__ __align__(16) float Bs[2][BK][BNP];
+
+    const int tid = threadIdx.x;
+    const int tx = tid & 15;                          // pixel group
+    const int ty = tid >> 4;                          // channel group
+    const int m0 = blockIdx.x * BM;
+    const int k0 = blockIdx.y * BN;
+    const int PQ = d.P * d.Q;
+    const int HW = d.H * d.W;
+
+    // ---- per-thread constants of the A (input) gather: this thread always loads pixel a_m
+    const int a_ml = tid % BM;
+    const int a_kk0 = tid / BM;                       // first chunk row this thread loads
+    constexpr int A_KK_STEP = (kThreads >= BM) ? kThreads / BM : 1;
+    int a_y0 = 0, a_x0 = 0;
+    long long a_base = 0;
+    bool a_ok = false;
+    {
+        const int m = m0 + a_ml;
+        if (m < d.M) {
+            const int n = m / PQ;
+            const int pq = m - n * PQ;
+            const int p = pq / d.Q;
+            const int q = pq - p * d.Q;
+            a_y0 = p * d.stride - d.pad;
+            a_x0 = q * d.stride - d.pad;
+            a_base = (long long)n * d.C * HW + (long long)a_y0 * d.W + a_x0;
+            a_ok = true;
+        }
+    }
+    // ---- per-thread constants of the B (filter) load
+    const int b_kk = tid & (BK - 1);
+    const int b_n0 = tid >> 3;                        // 0..31
+
+    float a_pre[A_PER_THREAD];
+    float b_pre[B_PER_THREAD];
+
+    auto load_global = [&](int kred0) {
+#pragma unroll
+        for (int i = 0; i < A_PER_THREAD; ++i) {
+            const int kk = a_kk0 + i * A_KK_STEP;
+            float v = 0.f;
+            if (kk < BK) {
+                const DirectTapEntry e = tab[kred0 + kk];
+                const int y = a_y0 + (e.rs >> 16);
+                const int x = a_x0 + (e.rs & 0xffff);
+                if (a_ok && (unsigned)y < (unsigned)d.H && (unsigned)x < (unsigned)d.W)
+                    v = __ldg(in + a_base + e.offset);
+            }
+            a_pre[i] = v;
+        }
+#pragma unroll
+        for (int i = 0; i < B_PER_THREAD; ++i) {
+            const int nl = b_n0 + i * 32;
+            const int k = k0 + nl;
+            const int j = kred0 + b_kk;
+            float v = 0.f;
+            if (nl < BN && k < d.K && j < d.Kred) v = __ldg(filt + (size_t)k * d.Kred + j);
+            b_pre[i] = v;
+        }
+    };
+    auto store_shared = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < A_PER_THREAD; ++i) {
+            const int kk = a_kk0 + i * A_KK_STEP;
+            if (kk < BK) As[buf][kk][a_ml] = a_pre[i];
+        }
+#pragma unroll
+        for (int i = 0; i < B_PER_THREAD; ++i) {
+            const int nl = b_n0 + i * 32;
+            if (nl < BN) Bs[buf][b_kk][nl] = b_pre[i];
+        }
+    };
+
+    float acc[TM][TN];
+#pragma unroll
+    for (int i = 0; i < TM; ++i)
+#pragma unroll
+        for (int j = 0; j < TN; ++j) acc[i][j] = 0.f;
+
+    const int chunks = (d.Kred + BK - 1) / BK;
+    load_global(0);
+    store_shared(0);
+    __syncthreads();
+
+    for (int t = 0; t < chunks; ++t) {
+        const int buf = t & 1;
+        if (t + 1 < chunks) load_global((t + 1) * BK);
+#pragma unroll
+        for (int kk = 0; kk < BK; ++kk) {
+            float a[TM], b[TN];
+            // pixels of this thread: groups of 4 (or TM if smaller) consecutive, 64 apart
+            if constexpr (TM % 4 == 0) {
+#pragma unroll
+                for (int g = 0; g < TM / 4; ++g) {
+                    const float4 v = *reinterpret_cast<const float4*>(&As[buf][kk][g * 64 + tx * 4]);
+                    a[4 * g + 0] = v.x; a[4 * g + 1] = v.y; a[4 * g + 2] = v.z; a[4 * g + 3] = v.w;
+                }
+            } else {
+#pragma unroll
+                for (int i = 0; i < TM; ++i) a[i] = As[buf][kk][tx * TM + i];
+            }
+            if constexpr (TN % 4 == 0) {
+#pragma unroll
+                for (int g = 0; g < TN / 4; ++g) {
+                    const float4 v = *reinterpret_cast<const float4*>(&Bs[buf][kk][ty * TN + 4 * g]);
+                    b[4 * g + 0] = v.x; b[4 * g + 1] = v.y; b[4 * g + 2] = v.z; b[4 * g + 3] = v.w;
+                }
+            } else if constexpr (TN % 2 == 0) {
+#pragma unroll
+                for (int g = 0; g < TN / 2; ++g) {
+                    const float2 v = *reinterpret_cast<const float2*>(&Bs[buf][kk][ty * TN + 2 * g]);
+                    b[2 * g + 0] = v.x; b[2 * g + 1] = v.y;
+                }
+            } else {
+#pragma unroll
+                for (int j = 0; j < TN; ++j) b[j] = Bs[buf][kk][ty * TN + j];
+            }
+#pragma unroll
+            for (int i = 0; i < TM; ++i)
+#pragma unroll
+                for (int j = 0; j < TN; ++j) acc[i][j] = fmaf(a[i], b[j], acc[i][j]);
+        }
+        if (t + 1 < chunks) store_shared(buf ^ 1);
+        __syncthreads();
+    }
+
+    // ---- epilogue: bias, ReLU, NCHW store
+#pragma unroll
+    for (int i = 0; i < TM; ++i) {
+        const int ml = (TM % 4 == 0) ? ((i >> 2) * 64 + tx * 4 + (i & 3)) : (tx * TM + i);
+        const int m = m0 + ml;
+        if (m >= d.M) continue;
+        const int n = m / PQ;
+        const int pq = m - n * PQ;
+        float* o = out + ((size_t)n * d.K) * PQ + pq;
+#pragma unroll
+        for (int j = 0; j < TN; ++j) {
+            const int k = k0 + ty * TN + j;
+            if (k < d.K) {
+                float v = acc[i][j] + (bias ? __ldg(bias + k) : 0.f);
+                if (d.relu) v = fmaxf(v, 0.f);
+                o[(size_t)k * PQ] = v;
+            }
+        }
+    }
+}
+
+struct TileInfo { int TM, TN; const char* name; };
+constexpr TileInfo kTiles[] = {
+    {8, 8, "direct_128x128"}, {8, 6, "direct_128x96"}, {8, 4, "direct_128x64"}, {8, 2, "direct_128x32"},
+    {4, 4, "direct_64x64"},   {4, 2, "direct_64x32"},  {4, 1, "direct_64x16"},  {2, 2, "direct_32x32"},
+    {2, 1, "direct_32x16"},
+};
+constexpr int kNumTiles = sizeof(kTiles) / sizeof(kTiles[0]);
+
+template <int TM, int TN>
+int launch_tile(const ConvDims& d, const float* in, const float* filt, const float* bias, float* out,
+                const DirectTapEntry* tab, cudaStream_t stream)
+{
+    constexpr int BM = 16 * TM, BN = 16 * TN;
+    dim3 grid((d.M + BM - 1) / BM, (d.K + BN - 1) / BN);
+    direct_conv_kernel<TM, TN><<<grid, kThreads, 0, stream>>>(d, in, filt, bias, out, tab);
+    count_launch();
+    BODA_CUDA_TRY(cudaGetLastError());
+    return BODA_OK;
+}
+
+}  // namespace
+
+int direct_num_tiles() { return kNumTiles; }
+const char* direct_tile_name(int id) { return (id >= 0 && id < kNumTiles) ? kTiles[id].name : "?"; }
+
+int direct_pick_tile(const ConvDims& d)
+{
+    // Rule of thumb in the spirit of Section 4: the widest channel tile that K fills without much
+    // waste, then the tallest pixel tile that still yields about two blocks per SM.
+    int best = kNumTiles - 1;
+    double best_cost = 1e300;
+    for (int t = 0; t < kNumTiles; ++t) {
+        const int BM = 16 * kTiles[t].TM, BN = 16 * kTiles[t].TN;
+        const long long gm = (d.M + BM - 1) / BM, gn = (d.K + BN - 1) / BN;
+        const double padded = (double)gm * BM * gn * BN;             // FMAs issued per reduction step
+        const double blocks = (double)gm * gn;
+        const double waves = blocks / (148.0 * 2.0);
+        const double fill = waves < 1.0 ? 1.0 / waves : (double)(long long)(waves + 0.999) / waves;
+        // small register tiles pay more shared-memory traffic per FMA
+        const double ldst = 1.0 + 0.5 * (1.0 / kTiles[t].TM + 1.0 / kTiles[t].TN);
+        const double cost = padded * fill * ldst;
+        if (cost < best_cost) { best_cost = cost; best = t; }
+    }
+    return best;
+}
+
+int direct_table_len(const ConvDims& d) { return ((d.Kred + BK - 1) / BK) * BK; }
+
+void direct_build_table(const ConvDims& d, DirectTapEntry* tab)
+{
+    const int len = direct_table_len(d);
+    int j = 0;
+    for (int c = 0; c < d.C; ++c)
+        for (int r = 0; r < d.R; ++r)
+            for (int s = 0; s < d.S; ++s, ++j) {
+                tab[j].offset = c * d.H * d.W + r * d.W + s;
+                tab[j].rs = (r << 16) | s;
+            }
+    for (; j < len; ++j) { tab[j].offset = 0; tab[j].rs = (0x4000 << 16); }
+}
+
+int direct_launch(const ConvDims& d, int tile_id, const float* in, const float* filt, const float* bias,
+                  float* out, const DirectTapEntry* tab, cudaStream_t stream)
+{
+    switch (tile_id) {
+        case 0: return launch_tile<8, 8>(d, in, filt, bias, out, tab, stream);
+        case 1: return launch_tile<8, 6>(d, in, filt, bias, out, tab, stream);
+        case 2: return launch_tile<8, 4>(d, in, filt, bias, out, tab, stream);
+        case 3: return launch_tile<8, 2>(d, in, filt, bias, out, tab, stream);
+        case 4: return launch_tile<4, 4>(d, in, filt, bias, out, tab, stream);
+        case 5: return launch_tile<4, 2>(d, in, filt, bias, out, tab, stream);
+        case 6: return launch_tile<4, 1>(d, in, filt, bias, out, tab, stream);
+        case 7: return launch_tile<2, 2>(d, in, filt, bias, out, tab, stream);
+        case 8: return launch_tile<2, 1>(d, in, filt, bias, out, tab, stream);
+        default: return BODA_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace boda

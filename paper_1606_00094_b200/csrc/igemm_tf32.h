@@ -1,0 +1,27 @@
+// Tensor-core (tcgen05, TF32) implicit-GEMM variants K1CONV and TCONV: host-side interface.
+#pragma once
+
+#include "boda_internal.h"
+
+namespace boda {
+
+struct IgemmPlan;
+
+bool igemm_variant_legal(const ConvDims& d, int variant);
+// Rule used by automatic selection: is the tensor-core path expected to beat DIRECT for this shape?
+bool igemm_variant_profitable(const ConvDims& d);
+int igemm_num_tiles();
+int igemm_num_split_candidates();
+int igemm_split_candidate(int i);
+
+int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int* d_status, IgemmPlan** out);
+void igemm_plan_destroy(IgemmPlan* p);
+int igemm_plan_tile(const IgemmPlan* p);
+size_t igemm_plan_workspace_bytes(const IgemmPlan* p);
+void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n);
+int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream);
+void igemm_unbind_filters(IgemmPlan* p);
+int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
+                 cudaStream_t stream);
+
+}  // namespace boda
