@@ -1,16 +1,686 @@
+// K1CONV and TCONV: implicit-GEMM convolution on the sm_100a tensor cores (tcgen05, TF32 operands,
+// fp32 accumulation in tensor memory).
+//
+// GEMM view (Section 3 of the paper: out = inmat * filtsmat, with inmat never materialised, Section 5):
+//   M = N*P*Q output points ("pixels"), N_gemm = K output channels, reduction = (r, s, c).
+// One CTA owns a 128-pixel x BN-channel output tile.  The reduction is walked tap by tap and, inside a
+// tap, in chunks of 32 input channels (one 128-byte swizzled shared-memory row per pixel / channel):
+//   A tile  [128 pixels][32 channels]  <- TMA im2col-mode load from the NHWC re-laid-out input; the
+//            hardware walks the 128 consecutive output points of the tile across rows and images, adds
+//            the tap offset (s, r) and fills out-of-image pixels with zeros (= the padding);
+//   B tile  [BN channels][32 channels] <- TMA tiled load from tap-major filters [R*S][K][C].
+// k1conv (kernel size 1) is the same kernel with a single tap: a plain GEMM over C.
+// Roles inside the CTA (192 threads): warp 0 = TMA producer (one elected lane), warp 1 = TMEM owner and
+// MMA issuer (one elected lane issues tcgen05.mma, tcgen05.commit releases shared-memory stages),
+// warps 2..5 = epilogue (tcgen05.ld of the accumulator, bias, ReLU, store).  This is Listing 1's
+// "load block / fma block / store block" loop with hardware pipelines in place of barriers.
+// Every wait is bounded (two seconds): on expiry the kernel records BODA_ERR_DEVICE_TIMEOUT in the
+// status word, all roles leave their loops, tensor memory is released and the CTA returns.
+#include <cuda.h>
+
+#include <algorithm>
+#include <cstdio>
+#include <cstring>
+#include <new>
+
 #include "igemm_tf32.h"
+
 namespace boda {
-bool igemm_variant_legal(const ConvDims&, int) { return false; }
-bool igemm_variant_profitable(const ConvDims&) { return false; }
-int igemm_num_tiles() { return 0; }
-int igemm_num_split_candidates() { return 0; }
-int igemm_split_candidate(int) { return 1; }
-int igemm_plan_create(const ConvDims&, int, int, int, int*, IgemmPlan**) { return BODA_ERR_UNSUPPORTED; }
-void igemm_plan_destroy(IgemmPlan*) {}
-int igemm_plan_tile(const IgemmPlan*) { return 0; }
-size_t igemm_plan_workspace_bytes(const IgemmPlan*) { return 0; }
-void igemm_plan_describe(const IgemmPlan*, char* b, size_t n) { if (n) b[0] = 0; }
-int igemm_bind_filters(IgemmPlan*, const float*, cudaStream_t) { return BODA_ERR_UNSUPPORTED; }
-void igemm_unbind_filters(IgemmPlan*) {}
-int igemm_launch(IgemmPlan*, const float*, const float*, const float*, float*, void*, cudaStream_t) { return BODA_ERR_UNSUPPORTED; }
+namespace {
+
+constexpr int BM = 128;          // pixels per CTA tile (UMMA M)
+constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of fp32)
+constexpr int A_STAGE_BYTES = BM * BKC * 4;
+constexpr int kIgemmThreads = 192;
+constexpr unsigned long long kWaitLimitNs = 2000000000ull;
+
+struct IgemmParams {
+    int M, K, PQ, Q, stride, pad, S;
+    int cchunks;                 // Cp / 32
+    int iters_total;             // taps * cchunks
+    int iters_per_split;
+    int splits;
+    int relu;
+    const float* bias;
+    float* out;
+    float* partials;             // [tile][split][BN][128], splits > 1 only
+    int* counters;               // [tile], zero between launches
+    int* status;
+};
+
+// ------------------------------------------------------------------------------------------------
+// PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
+{
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
 }
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
+{
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
+{
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
+    return ok != 0;
+}
+__device__ __forceinline__ unsigned long long global_timer_ns()
+{
+    unsigned long long t;
+    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
+    return t;
+}
+
+// Bounded wait.  Returns false if the CTA is aborting or the limit expired (then it raises the abort flag
+// and records where it gave up).
+__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
+{
+    if (mbar_try_wait(bar, parity)) return true;
+    const unsigned long long t0 = global_timer_ns();
+    for (uint32_t spin = 1;; ++spin) {
+        if (mbar_try_wait(bar, parity)) return true;
+        if ((spin & 63u) == 0u) {
+            if (*abort_flag) return false;
+            if (global_timer_ns() - t0 > kWaitLimitNs) {
+                *abort_flag = 1;
+                if (atomicCAS(status, 0, (int)BODA_ERR_DEVICE_TIMEOUT) == 0) {
+                    status[1] = KERNEL_ID_IGEMM;
+                    status[2] = (int)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));
+                    status[3] = where;
+                }
+                return false;
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w,
+                                                   int h, int n, uint16_t off_w, uint16_t off_h)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
+        :: "r"(dst), "l"((uint64_t)map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
+        : "memory");
+}
+__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z)
+{
+    asm volatile(
+        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
+        " [%0], [%1, {%3, %4, %5}], [%2];"
+        :: "r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
+}
+__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map)
+{
+    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)map) : "memory");
+}
+
+__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
+{
+    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tmem_relinquish()
+{
+    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+}
+__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
+{
+    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
+}
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar)
+{
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+// D[tmem] (+)= A[smem] * B[smem], TF32 operands, 128 x N x 8 per instruction
+__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&v)[32])
+{
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
+        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
+        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
+        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
+          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
+          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
+          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
+        : "r"(taddr) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled, with
+// 8-row groups 1024 bytes apart (the layout both TMA loads above produce).
+__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr)
+{
+    return (uint64_t)((addr & 0x3FFFFu) >> 4)      // start address, 16-byte units
+         | (1ull << 16)                            // leading byte offset (unused for swizzled K-major)
+         | ((uint64_t)(1024 >> 4) << 32)           // stride byte offset: next 8-row group
+         | (1ull << 46)                            // descriptor version of sm_100
+         | (2ull << 61);                           // 128-byte swizzle
+}
+
+template <int BN>
+__host__ __device__ constexpr uint32_t instr_desc_tf32()
+{
+    return (1u << 4)                   // accumulator format: fp32
+         | (2u << 7) | (2u << 10)      // A and B format: TF32
+         | (0u << 15) | (0u << 16)     // A and B are K-major
+         | ((uint32_t)(BN >> 3) << 17) // N
+         | ((uint32_t)(BM >> 4) << 24);// M
+}
+
+template <int BN> struct TileCfg {
+    static constexpr int B_STAGE_BYTES = BN * BKC * 4;
+    static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+    static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
+    static constexpr int TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+    static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
+};
+
+// ------------------------------------------------------------------------------------------------
+template <int BN>
+__global__ void __launch_bounds__(kIgemmThreads, 1)
+igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const IgemmParams p)
+{
+    using Cfg = TileCfg<BN>;
+    constexpr int STAGES = Cfg::STAGES;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;       // swizzle atoms need 1024-byte alignment
+    const uint32_t smem_a = smem_base;
+    const uint32_t smem_b = smem_base + STAGES * A_STAGE_BYTES;
+    const uint32_t bars = smem_base + STAGES * Cfg::STAGE_BYTES;
+    const uint32_t full_bar = bars;                    // STAGES x 8 bytes
+    const uint32_t empty_bar = bars + 8 * STAGES;
+    const uint32_t accum_bar = bars + 16 * STAGES;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ volatile int s_abort;
+    __shared__ int s_is_last;
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int m0 = blockIdx.x * BM;
+    const int k0 = blockIdx.y * BN;
+    const int it_begin = blockIdx.z * p.iters_per_split;
+    const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
+    const int my_iters = it_end - it_begin;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&s_tmem_base), Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = s_tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer
+            const int n0 = m0 / p.PQ;
+            const int rem = m0 - n0 * p.PQ;
+            const int p0 = rem / p.Q;
+            const int q0 = rem - p0 * p.Q;
+            const int w0 = q0 * p.stride - p.pad;
+            const int h0 = p0 * p.stride - p.pad;
+            int tap = it_begin / p.cchunks;
+            int cc = it_begin - tap * p.cchunks;
+            int r = tap / p.S;
+            int s = tap - r * p.S;
+            for (int i = 0; i < my_iters; ++i) {
+                const int stage = i % STAGES;
+                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+                if (!mbar_wait(empty_bar + 8 * stage, ph ^ 1u, &s_abort, p.status, 1)) break;
+                const uint32_t fb = full_bar + 8 * stage;
+                mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+                tma_load_im2col_4d(smem_a + stage * A_STAGE_BYTES, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                tma_load_3d(smem_b + stage * Cfg::B_STAGE_BYTES, &map_b, fb, cc * BKC, k0, tap);
+                if (++cc == p.cchunks) { cc = 0; ++tap; if (++s == p.S) { s = 0; ++r; } }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            constexpr uint32_t idesc = instr_desc_tf32<BN>();
+            bool ok = true;
+            for (int i = 0; i < my_iters && ok; ++i) {
+                const int stage = i % STAGES;
+                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
+                ok = mbar_wait(full_bar + 8 * stage, ph, &s_abort, p.status, 2);
+                if (!ok) break;
+                tc_fence_after();
+                const uint64_t da = smem_desc_k_sw128(smem_a + stage * A_STAGE_BYTES);
+                const uint64_t db = smem_desc_k_sw128(smem_b + stage * Cfg::B_STAGE_BYTES);
+#pragma unroll
+                for (int k = 0; k < BKC / 8; ++k)       // 8 TF32 values = 32 bytes = 2 descriptor units per step
+                    umma_tf32(tmem_acc, da + 2 * k, db + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
+                tc_commit(empty_bar + 8 * stage);       // frees the stage once these MMAs have read it
+            }
+            tc_commit(accum_bar);                       // accumulator complete (or: everything issued so far has drained)
+            if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
+        }
+    } else {
+        // ---------------- epilogue: 4 warps, warp w reads TMEM lanes 32*(w%4) .. +31
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const int m = m0 + row;
+        const bool ok = mbar_wait(accum_bar, 0, &s_abort, p.status, 4);
+        tc_fence_after();
+        const bool m_ok = m < p.M;
+        int n = 0, pq = 0;
+        if (m_ok) { n = m / p.PQ; pq = m - n * p.PQ; }
+        const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+        const int tile_lin = blockIdx.y * gridDim.x + blockIdx.x;
+        if (ok && p.splits == 1) {
+            float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
+#pragma unroll 1
+            for (int j0 = 0; j0 < BN; j0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32cols(trow + j0, v);
+                tmem_ld_wait();
+                if (m_ok) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        const int k = k0 + j0 + j;
+                        if (k < p.K) {
+                            float y = __uint_as_float(v[j]) + (p.bias ? __ldg(p.bias + k) : 0.f);
+                            if (p.relu) y = fmaxf(y, 0.f);
+                            o[(size_t)k * p.PQ] = y;
+                        }
+                    }
+                }
+            }
+        } else if (ok) {
+            // split reduction: park the partial tile, the CTA that arrives last sums all partials in split order
+            float* part = p.partials + ((size_t)tile_lin * p.splits + blockIdx.z) * (BN * BM);
+#pragma unroll 1
+            for (int j0 = 0; j0 < BN; j0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32cols(trow + j0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(j0 + j) * BM + row, __uint_as_float(v[j]));
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) {
+                const int old = atomicAdd(p.counters + tile_lin, 1);
+                s_is_last = (old == p.splits - 1);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (s_is_last) {
+                __threadfence();
+                const float* base = p.partials + (size_t)tile_lin * p.splits * (BN * BM);
+                if (m_ok) {
+                    float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
+#pragma unroll 1
+                    for (int j = 0; j < BN; ++j) {
+                        const int k = k0 + j;
+                        if (k >= p.K) break;
+                        float acc = p.bias ? __ldg(p.bias + k) : 0.f;
+                        for (int z = 0; z < p.splits; ++z) acc += __ldcg(base + ((size_t)z * BN + j) * BM + row);
+                        if (p.relu) acc = fmaxf(acc, 0.f);
+                        o[(size_t)k * p.PQ] = acc;
+                    }
+                }
+                if (threadIdx.x == 64) p.counters[tile_lin] = 0;
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_acc, Cfg::TMEM_COLS);
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Operand staging ("input transformation", Section 5): NCHW -> NHWC with channels padded to a multiple of
+// 32 and values rounded to TF32 (round to nearest, ties away), so that the tensor core's truncation of the
+// low mantissa bits is exact.
+__device__ __forceinline__ float round_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+__global__ void __launch_bounds__(256)
+pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int C, int Cp, int HW)
+{
+    __shared__ float tile[32][33];
+    const int n = blockIdx.z;
+    const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8
+    const float* src = in + (size_t)n * C * HW;
+    float* dst = xp + (size_t)n * HW * Cp;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i, hw = hw0 + tx;
+        tile[ty + 8 * i][tx] = (c < C && hw < HW) ? __ldg(src + (size_t)c * HW + hw) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int hw = hw0 + ty + 8 * i, c = c0 + tx;
+        if (hw < HW) dst[(size_t)hw * Cp + c] = round_tf32(tile[tx][ty + 8 * i]);
+    }
+}
+
+// filters KCRS -> [R*S][K][Cp], TF32-rounded, zero in the padded channels
+__global__ void __launch_bounds__(256)
+pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int Cp, int RS)
+{
+    const long long total = (long long)RS * K * Cp;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % Cp);
+        const long long t = idx / Cp;
+        const int k = (int)(t % K);
+        const int tap = (int)(t / K);
+        wp[idx] = c < C ? round_tf32(__ldg(filt + ((size_t)k * C + c) * RS + tap)) : 0.f;
+    }
+}
+
+// ------------------------------------------------------------------------------------------------
+// Host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+typedef CUresult (*EncodeIm2colFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                   const cuuint64_t*, const int*, const int*, cuuint32_t, cuuint32_t, const cuuint32_t*,
+                                   CUtensorMapInterleave, CUtensorMapSwizzle, CUtensorMapL2promotion,
+                                   CUtensorMapFloatOOBfill);
+EncodeTiledFn g_encode_tiled = nullptr;
+EncodeIm2colFn g_encode_im2col = nullptr;
+
+int load_driver_entry_points()
+{
+    if (g_encode_tiled && g_encode_im2col) return BODA_OK;
+    void* f1 = nullptr;
+    void* f2 = nullptr;
+    cudaDriverEntryPointQueryResult q1, q2;
+    BODA_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &f1, cudaEnableDefault, &q1));
+    BODA_CUDA_TRY(cudaGetDriverEntryPoint("cuTensorMapEncodeIm2col", &f2, cudaEnableDefault, &q2));
+    if (!f1 || !f2 || q1 != cudaDriverEntryPointSuccess || q2 != cudaDriverEntryPointSuccess) return BODA_ERR_UNSUPPORTED;
+    g_encode_tiled = (EncodeTiledFn)f1;
+    g_encode_im2col = (EncodeIm2colFn)f2;
+    return BODA_OK;
+}
+
+constexpr int kTileBN[] = {64, 96, 128, 192, 256};
+constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
+constexpr int kSplitCandidates[] = {1, 2, 3, 4, 6, 8};
+
+}  // namespace
+
+struct IgemmPlan {
+    ConvDims d;
+    int variant = 0;
+    int tile_id = 0;
+    int BN = 128;
+    int Cp = 0;
+    int splits = 1;
+    int iters_total = 0, iters_per_split = 0;
+    int tiles_m = 0, tiles_n = 0;
+    int* d_status = nullptr;
+    float* d_wp = nullptr;           // packed filters [RS][K][Cp]
+    int* d_counters = nullptr;       // [tiles_m * tiles_n]
+    const float* bound_filt = nullptr;
+    size_t xp_bytes = 0, partial_bytes = 0;
+    CUtensorMap map_b;
+    CUtensorMap map_a;
+    const void* map_a_base = nullptr;
+};
+
+bool igemm_variant_legal(const ConvDims& d, int variant)
+{
+    if (d.R > 11 || d.S > 11 || d.stride > 8 || d.pad > 100) return false;
+    if (d.P <= 0 || d.Q <= 0) return false;
+    if (variant == BODA_VARIANT_K1CONV) return d.R == 1 && d.S == 1;
+    if (variant == BODA_VARIANT_TCONV) return d.R * d.S >= 2;
+    return false;
+}
+
+bool igemm_variant_profitable(const ConvDims& d)
+{
+    // Channels are padded to 32 per reduction chunk and pixels to 128 per tile: tiny C (first layers) and tiny
+    // layers stay on the FP32 kernel.
+    return d.C >= 16 && d.K >= 16 && (long long)d.M * d.K >= 128 * 64;
+}
+
+int igemm_num_tiles() { return kNumIgemmTiles; }
+int igemm_num_split_candidates() { return (int)(sizeof(kSplitCandidates) / sizeof(int)); }
+int igemm_split_candidate(int i) { return kSplitCandidates[i]; }
+
+namespace {
+
+// Rough cost model (clocks) used when the plan is not tuned by timing: MMA issue versus operand bytes from L2.
+double model_cost(const ConvDims& d, int Cp, int BN, int splits)
+{
+    const int taps = d.R * d.S;
+    const int iters = taps * (Cp / BKC);
+    const int ips = (iters + splits - 1) / splits;
+    const long long tm = (d.M + BM - 1) / BM, tn = (d.K + BN - 1) / BN;
+    const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
+    const double waves = (double)(long long)((ctas + 147) / 148);
+    const double mma_clk = BN * 2.0;                                     // 128 x BN x 32 MACs at 2048 MAC/clk
+    const double feed_clk = (A_STAGE_BYTES + BN * 128.0) / 48.0;         // about 48 B/clk/SM from L2
+    const double per_iter = std::max(mma_clk, feed_clk);
+    const double epilogue = BN * 6.0 * (splits > 1 ? 2.0 + 0.6 * splits : 1.0) + 1500.0;
+    return waves * (ips * per_iter + epilogue);
+}
+
+template <int BN>
+int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
+{
+    using Cfg = TileCfg<BN>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        BODA_CUDA_TRY(cudaFuncSetAttribute(igemm_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+        attr_set = true;
+    }
+    dim3 grid(p->tiles_m, p->tiles_n, p->splits);
+    igemm_tf32_kernel<BN><<<grid, kIgemmThreads, Cfg::SMEM_BYTES, stream>>>(p->map_a, p->map_b, prm);
+    BODA_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BODA_OK;
+}
+
+int encode_map_a(IgemmPlan* p, const void* xp)
+{
+    const ConvDims& d = p->d;
+    const cuuint64_t dims[4] = {(cuuint64_t)p->Cp, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
+    const cuuint64_t strides[3] = {(cuuint64_t)p->Cp * 4, (cuuint64_t)d.W * p->Cp * 4, (cuuint64_t)d.H * d.W * p->Cp * 4};
+    const int lower[2] = {-d.pad, -d.pad};                                 // W, H
+    const int upper[2] = {d.pad - (d.S - 1), d.pad - (d.R - 1)};
+    const cuuint32_t estr[4] = {1, (cuuint32_t)d.stride, (cuuint32_t)d.stride, 1};
+    CUresult r = g_encode_im2col(&p->map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(xp), dims, strides,
+                                 lower, upper, BKC, BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeIm2col failed with CUresult %d", (int)r);
+        return record_cuda_error(cudaErrorInvalidValue, msg);
+    }
+    p->map_a_base = xp;
+    return BODA_OK;
+}
+
+int encode_map_b(IgemmPlan* p)
+{
+    const ConvDims& d = p->d;
+    const cuuint64_t dims[3] = {(cuuint64_t)p->Cp, (cuuint64_t)d.K, (cuuint64_t)(d.R * d.S)};
+    const cuuint64_t strides[2] = {(cuuint64_t)p->Cp * 4, (cuuint64_t)d.K * p->Cp * 4};
+    const cuuint32_t box[3] = {BKC, (cuuint32_t)p->BN, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    CUresult r = g_encode_tiled(&p->map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled failed with CUresult %d", (int)r);
+        return record_cuda_error(cudaErrorInvalidValue, msg);
+    }
+    return BODA_OK;
+}
+
+}  // namespace
+
+int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int* d_status, IgemmPlan** out)
+{
+    if (!igemm_variant_legal(d, variant)) return BODA_ERR_UNSUPPORTED;
+    if (tile_id >= kNumIgemmTiles) return BODA_ERR_UNSUPPORTED;
+    if (split_k < 0 || split_k > 64) return BODA_ERR_INVALID_ARG;
+    int rc = load_driver_entry_points();
+    if (rc != BODA_OK) return rc;
+    IgemmPlan* p = new (std::nothrow) IgemmPlan();
+    if (!p) return BODA_ERR_NOMEM;
+    p->d = d;
+    p->variant = variant;
+    p->d_status = d_status;
+    p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
+    p->iters_total = d.R * d.S * (p->Cp / BKC);
+    // tile and split: forced, or the minimum of the cost model
+    double best = 1e300;
+    int best_t = 2, best_s = 1;
+    for (int t = 0; t < kNumIgemmTiles; ++t) {
+        if (tile_id >= 0 && t != tile_id) continue;
+        for (int s : kSplitCandidates) {
+            if (split_k > 0 && s != split_k) continue;
+            if (s > p->iters_total) continue;
+            const double c = model_cost(d, p->Cp, kTileBN[t], s);
+            if (c < best) { best = c; best_t = t; best_s = s; }
+        }
+    }
+    if (split_k > 0) best_s = std::min(split_k, p->iters_total);
+    if (tile_id >= 0) best_t = tile_id;
+    p->tile_id = best_t;
+    p->BN = kTileBN[best_t];
+    p->iters_per_split = (p->iters_total + best_s - 1) / best_s;
+    p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;   // no empty split
+    p->tiles_m = (d.M + BM - 1) / BM;
+    p->tiles_n = (d.K + p->BN - 1) / p->BN;
+    p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
+    p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * BM * 4 : 0;
+
+    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cp * 4);
+    if (e == cudaSuccess) e = cudaMalloc(&p->d_counters, (size_t)p->tiles_m * p->tiles_n * sizeof(int));
+    if (e == cudaSuccess) e = cudaMemset(p->d_counters, 0, (size_t)p->tiles_m * p->tiles_n * sizeof(int));
+    if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
+    rc = encode_map_b(p);
+    if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
+    *out = p;
+    return BODA_OK;
+}
+
+void igemm_plan_destroy(IgemmPlan* p)
+{
+    if (!p) return;
+    if (p->d_wp) cudaFree(p->d_wp);
+    if (p->d_counters) cudaFree(p->d_counters);
+    delete p;
+}
+
+int igemm_plan_tile(const IgemmPlan* p) { return p->tile_id; }
+size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->partial_bytes; }
+
+void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
+{
+    std::snprintf(buf, n, "tile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", p->BN, p->tile_id,
+                  p->BN == 64 ? TileCfg<64>::STAGES : p->BN == 96 ? TileCfg<96>::STAGES : p->BN == 128 ? TileCfg<128>::STAGES
+                  : p->BN == 192 ? TileCfg<192>::STAGES : TileCfg<256>::STAGES,
+                  p->splits, p->tiles_m, p->tiles_n, p->splits);
+}
+
+static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
+{
+    const ConvDims& d = p->d;
+    const long long total = (long long)d.R * d.S * d.K * p->Cp;
+    const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
+    pack_filters_kernel<<<blocks, 256, 0, stream>>>(filt, p->d_wp, d.K, d.C, p->Cp, d.R * d.S);
+    BODA_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BODA_OK;
+}
+
+int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
+{
+    int rc = pack_filters(p, filt, stream);
+    if (rc == BODA_OK) p->bound_filt = filt;
+    return rc;
+}
+
+void igemm_unbind_filters(IgemmPlan* p) { p->bound_filt = nullptr; }
+
+int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
+                 cudaStream_t stream)
+{
+    const ConvDims& d = p->d;
+    if (!workspace) return BODA_ERR_NOMEM;
+    if (((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
+    float* xp = (float*)workspace;
+    float* partials = (float*)((char*)workspace + p->xp_bytes);
+    if (filt != p->bound_filt || !filt) {
+        if (!filt) return BODA_ERR_INVALID_ARG;
+        int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
+        if (rc != BODA_OK) return rc;
+    }
+    {
+        const int HW = d.H * d.W;
+        dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
+        pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
+        BODA_CUDA_TRY(cudaGetLastError());
+        count_launch();
+    }
+    if (p->map_a_base != xp) {
+        int rc = encode_map_a(p, xp);
+        if (rc != BODA_OK) return rc;
+    }
+    IgemmParams prm;
+    prm.M = d.M; prm.K = d.K; prm.PQ = d.P * d.Q; prm.Q = d.Q; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
+    prm.cchunks = p->Cp / BKC;
+    prm.iters_total = p->iters_total;
+    prm.iters_per_split = p->iters_per_split;
+    prm.splits = p->splits;
+    prm.relu = d.relu;
+    prm.bias = bias;
+    prm.out = out;
+    prm.partials = partials;
+    prm.counters = p->d_counters;
+    prm.status = p->d_status;
+    switch (p->BN) {
+        case 64: return launch_bn<64>(p, prm, stream);
+        case 96: return launch_bn<96>(p, prm, stream);
+        case 128: return launch_bn<128>(p, prm, stream);
+        case 192: return launch_bn<192>(p, prm, stream);
+        case 256: return launch_bn<256>(p, prm, stream);
+        default: return BODA_ERR_UNSUPPORTED;
+    }
+}
+
+}  // namespace boda
