@@ -286,7 +286,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int m = m0 + row;
-        const bool ok = mbar_wait(accum_bar, 0, &s_abort, p.status, 4);
+        (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 4);
+        // All 128 epilogue threads meet here whatever their wait returned, then take one common decision:
+        // a failed wait has raised the abort flag before returning.
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const bool ok = (s_abort == 0);
         tc_fence_after();
         const bool m_ok = m < p.M;
         int n = 0, pq = 0;

@@ -1,0 +1,104 @@
+"""GPU parity of the tensor-core variants (K1CONV, TCONV: tcgen05 TF32 implicit GEMM) against the fp64 oracle."""
+import numpy as np
+import pytest
+
+from paper_1606_00094_b200 import workloads as wl
+from helpers import TF32_TOL, assert_parity, oracle_out, run_planned
+
+pytestmark = pytest.mark.gpu
+
+K1, TC = 1, 2
+
+
+def _int_tensors(shape, seed):
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    return wl.integers(seed, (N, C, H, W)), wl.integers(seed + 1, (K, C, R, S)), wl.integers(seed + 2, (K,))
+
+
+def _real_tensors(shape, seed):
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    return (wl.half_normal(seed, (N, C, H, W)), wl.normal(seed + 1, (K, C, R, S), 0, (2.0 / (C * R * S)) ** 0.5),
+            wl.normal(seed + 2, (K,), 0, 0.01))
+
+
+# integer-valued inputs in [-8, 8] are exact in TF32 and every partial sum is exact in fp32, so the
+# tensor-core path must reproduce the oracle bit for bit: an indexing test that no tolerance can blur.
+EXACT_CASES = [
+    # shape, variant
+    ((1, 32, 8, 8, 16, 1, 1, 1, 0, 0), K1),            # single tile, single chunk
+    ((2, 64, 14, 14, 48, 1, 1, 1, 0, 1), K1),          # several pixel tiles, ragged last tile (392 = 3*128 + 8)
+    ((5, 40, 7, 9, 200, 1, 1, 1, 0, 0), K1),           # C not a multiple of 32, K ragged against every tile
+    ((1, 32, 6, 6, 16, 3, 3, 1, 1, 0), TC),            # one image, padding on all sides
+    ((3, 64, 13, 13, 80, 3, 3, 1, 1, 1), TC),          # tiles straddle rows and images
+    ((2, 96, 27, 27, 72, 5, 5, 1, 2, 1), TC),          # conv2-like
+    ((2, 20, 15, 17, 24, 3, 5, 2, 1, 0), TC),          # stride 2, R != S, C padded
+    ((1, 36, 23, 23, 40, 11, 11, 4, 0, 1), TC),        # conv1-like window and stride
+    ((2, 32, 9, 9, 16, 2, 2, 1, 0, 1), TC),            # even window, no padding
+    ((1, 32, 5, 5, 16, 3, 3, 1, 3, 0), TC),            # pad >= window: border outputs are pure bias
+    ((2, 33, 10, 12, 300, 3, 3, 3, 2, 1), TC),         # stride 3, floor in the output extent
+]
+
+
+@pytest.mark.parametrize("shape,variant", EXACT_CASES)
+def test_exact_on_small_integers(shape, variant):
+    x, w, b = _int_tensors(shape, 500)
+    got, desc = run_planned(shape, x, w, b, variant=variant)
+    ref = oracle_out(shape, x, w, b)
+    assert np.abs(ref).max() < 2 ** 24
+    np.testing.assert_array_equal(got.astype(np.float64), ref, err_msg=desc)
+
+
+@pytest.mark.parametrize("tile", range(5))
+@pytest.mark.parametrize("split", [1, 2, 3, 8])
+def test_every_tile_and_split_exact(tile, split):
+    shape = (3, 64, 13, 13, 272, 3, 3, 1, 1, 1)
+    x, w, b = _int_tensors(shape, 600)
+    got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile, split_k=split)
+    import re
+    eff = int(re.search(r"split_k=(\d+)", desc).group(1))      # splits that would be empty are dropped
+    assert f"id {tile}" in desc and (eff == split or (split == 8 and eff == 6))
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_k1conv_is_the_matrix_product():
+    # Section 5 of the paper: for kernel size 1 the per-image im2col is the identity
+    shape = (2, 64, 6, 5, 32, 1, 1, 1, 0, 0)
+    x, w, _ = _int_tensors(shape, 700)
+    got, _ = run_planned(shape, x, w, None, variant=K1)
+    for n in range(2):
+        ref = w.reshape(32, 64).astype(np.float64) @ x[n].reshape(64, 30).astype(np.float64)
+        np.testing.assert_array_equal(got[n].reshape(32, 30).astype(np.float64), ref)
+
+
+@pytest.mark.parametrize("shape,variant", [
+    ((5, 480, 14, 14, 192, 1, 1, 1, 0, 1), K1),
+    ((4, 256, 13, 13, 384, 3, 3, 1, 1, 1), TC),
+    ((2, 96, 27, 27, 256, 5, 5, 1, 2, 1), TC),
+    ((3, 50, 20, 20, 70, 3, 3, 2, 1, 0), TC),
+])
+def test_tf32_tolerance_on_real_values(shape, variant):
+    x, w, b = _real_tensors(shape, 800)
+    ref = oracle_out(shape, x, w, b)
+    for bind in (False, True):
+        got, desc = run_planned(shape, x, w, b, variant=variant, bind=bind)
+        err = assert_parity(got, ref, TF32_TOL, desc)
+        assert err > 1e-7      # it really ran in reduced precision (an fp32 path would be ~1e-7)
+
+
+@pytest.mark.parametrize("cfg", [3, 4])
+def test_baseline_configs_tf32(cfg):
+    c = wl.CONFIGS[cfg]
+    x, w, b = c.tensors()
+    got, desc = run_planned(c.shape.as_tuple(), x, w, b)
+    assert ("k1conv" if cfg == 3 else "tconv") in desc
+    assert_parity(got, oracle_out(c.shape.as_tuple(), x, w, b), TF32_TOL, f"cfg{cfg} {desc}")
+
+
+def test_same_result_twice_bitwise_and_tuned_plan():
+    shape = (4, 128, 13, 13, 200, 3, 3, 1, 1, 1)
+    x, w, b = _real_tensors(shape, 900)
+    a, _ = run_planned(shape, x, w, b, variant=TC, split_k=3)
+    c, _ = run_planned(shape, x, w, b, variant=TC, split_k=3)
+    np.testing.assert_array_equal(a, c)          # split reduction is summed in split order: deterministic
+    t, desc = run_planned(shape, x, w, b, tune=1)
+    assert_parity(t, oracle_out(shape, x, w, b), TF32_TOL, desc)
