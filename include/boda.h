@@ -144,6 +144,42 @@ int boda_conv_fwd_host(const float* in_host, const float* filt_host, const float
                        void* stream);
 
 /*
+ * The forward pass for callers that must not allocate device memory.  (The paper has no counterpart: this
+ * is a property of the library, not of the method.)
+ *
+ * Who needs it: code that runs where cudaMalloc is off limits - inside a framework whose caching allocator
+ * owns all device memory and forbids side allocations, in a real-time loop where an allocation's implicit
+ * device synchronisation and unbounded latency are not acceptable, in a process whose memory budget was
+ * fixed at start-up, or after start-up under a policy that freezes the address space.  boda_conv_fwd
+ * allocates a plan and a workspace the first time it sees a shape; this entry point never does.
+ *
+ * What it does: the same operation as boda_conv_fwd, always on the tensor-core path (K1CONV for R = S = 1,
+ * TCONV otherwise; TF32 operands, fp32 accumulation), with the kernel's scratch - re-laid-out input and
+ * filters, split partial sums, split counters - in a device array of BODA_NOALLOC_SCRATCH_BYTES that is
+ * part of the library image.  Every GPU that loads the library holds that array until the process exits.
+ * It calls no cudaMalloc / cudaFree and no allocating library routine.  in / filt / bias / out are device
+ * pointers owned by the caller, as for boda_conv_fwd.
+ *
+ * Limits and rules
+ *   - Shapes whose scratch does not fit (roughly 4 * (N*H*W + R*S*K) * roundup(C, 32) bytes plus a small
+ *     header) are rejected with BODA_ERR_TOO_LARGE; shapes outside the tensor-core variants (R or S > 11,
+ *     stride > 8) with BODA_ERR_UNSUPPORTED.  Nothing is launched in either case.
+ *   - The first call on a device resolves the array's device address (cudaGetSymbolAddress), loads two
+ *     driver entry points and raises the kernel's shared-memory limit.  Make that first call during
+ *     start-up, before any stream capture begins.
+ *   - All calls share the one array and it keeps the previous call's contents; the entry point clears the
+ *     words that must start at zero itself.  Two calls whose GPU work can overlap (different streams
+ *     without an ordering between them, or different host threads on unordered streams) race on the
+ *     array and give wrong results: order them on one stream or with events.
+ *   - A bounded wait that expires inside the kernel is recorded in the array's own header, which
+ *     boda_query_status does not read; the output is then left unwritten.
+ */
+#define BODA_NOALLOC_SCRATCH_BYTES (32u << 20)
+int boda_conv_fwd_noalloc(const float* in, const float* filt, const float* bias, float* out,
+                          int N, int C, int H, int W, int K, int R, int S, int stride, int pad, int relu,
+                          void* stream);
+
+/*
  * Max-pooling, ksz x ksz window, given stride, no padding, floor output extent; the pooling that
  * sits between the convolutions of the AlexNet-shaped stack (the paper lists pooling among the
  * deployment operations, Section 2, without analysing it).  in [N][C][H][W] -> out [N][C][P][Q],

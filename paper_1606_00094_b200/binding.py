@@ -62,6 +62,8 @@ _lib.boda_conv_fwd.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd.restype = _i
 _lib.boda_conv_fwd_host.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd_host.restype = _i
+_lib.boda_conv_fwd_noalloc.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
+_lib.boda_conv_fwd_noalloc.restype = _i
 _lib.boda_maxpool_fwd.argtypes = [_vp, _vp] + [_i] * 6 + [_vp]
 _lib.boda_maxpool_fwd.restype = _i
 _lib.boda_query_status.argtypes = [_vp, ctypes.POINTER(_i)]
@@ -176,6 +178,18 @@ def boda_conv_fwd_host(inp, filt, bias, out, N, C, H, W, K, R, S, stride, pad, r
     """Same with HOST buffers (torch CPU tensors, preferably pinned, or raw host addresses)."""
     _check(_lib.boda_conv_fwd_host(_addr(inp), _addr(filt), _addr(bias), _addr(out), N, C, H, W, K, R, S, stride, pad,
                                    int(bool(relu)), _stream(stream)), "boda_conv_fwd_host")
+
+
+BODA_NOALLOC_SCRATCH_BYTES = 32 << 20
+
+
+def boda_conv_fwd_noalloc(inp, filt, bias, out, N, C, H, W, K, R, S, stride, pad, relu, stream=None) -> None:
+    """Forward pass that allocates no device memory: for callers that cannot call cudaMalloc (all device
+    memory owned by another allocator, real-time loops, frozen memory budgets).  Scratch lives in a fixed
+    array inside the library, shared by all calls: order the calls on one stream.  Raises BodaError with
+    BODA_ERR_TOO_LARGE when the shape's scratch exceeds BODA_NOALLOC_SCRATCH_BYTES."""
+    _check(_lib.boda_conv_fwd_noalloc(_addr(inp), _addr(filt), _addr(bias), _addr(out), N, C, H, W, K, R, S, stride,
+                                      pad, int(bool(relu)), _stream(stream)), "boda_conv_fwd_noalloc")
 
 
 def boda_maxpool_fwd(inp, out, N, C, H, W, ksz=3, stride=2, stream=None) -> None:

@@ -687,4 +687,106 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     }
 }
 
+// ------------------------------------------------------------------------------------------------
+// The same convolution with every piece of scratch (status word, split counters, re-laid-out filters and
+// input, split partial sums) carved out of ONE device region handed in by the caller.  Nothing is
+// allocated here; the region keeps its previous contents, so what must start at zero is cleared first.
+size_t igemm_region_min_bytes(const ConvDims& d)
+{
+    const size_t Cp = (size_t)((d.C + BKC - 1) / BKC) * BKC;
+    const size_t tiles = (size_t)((d.M + BM - 1) / BM) * (size_t)((d.K + 63) / 64);
+    const size_t head = 256 + ((tiles * sizeof(int) + 255) & ~(size_t)255);
+    const size_t wp = (((size_t)d.R * d.S * d.K * Cp * 4) + 1023) & ~(size_t)1023;
+    const size_t xp = (((size_t)d.N * d.H * d.W * Cp * 4) + 1023) & ~(size_t)1023;
+    return head + 1024 + wp + xp;
+}
+
+int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const float* filt, const float* bias,
+                        float* out, void* region, size_t region_bytes, cudaStream_t stream)
+{
+    if (!igemm_variant_legal(d, variant)) return BODA_ERR_UNSUPPORTED;
+    if (!in || !filt || !out || !region || ((uintptr_t)region & 255) != 0) return BODA_ERR_INVALID_ARG;
+    if (igemm_region_min_bytes(d) > region_bytes) return BODA_ERR_TOO_LARGE;
+    int rc = load_driver_entry_points();
+    if (rc != BODA_OK) return rc;
+
+    IgemmPlan plan;                       // lives on the host stack for the duration of this call only
+    IgemmPlan* p = &plan;
+    p->d = d;
+    p->variant = variant;
+    p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
+    p->iters_total = d.R * d.S * (p->Cp / BKC);
+    p->tiles_m = (d.M + BM - 1) / BM;
+    const size_t wp_bytes = (((size_t)d.R * d.S * d.K * p->Cp * 4) + 1023) & ~(size_t)1023;
+    p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
+    const size_t tiles_max = (size_t)p->tiles_m * (size_t)((d.K + 63) / 64);
+    const size_t head_bytes = 256 + ((tiles_max * sizeof(int) + 255) & ~(size_t)255);
+    const size_t fixed = head_bytes + 1024 + wp_bytes + p->xp_bytes;
+    // tile and split by the cost model, among the choices whose partial sums still fit the region
+    double best = 1e300;
+    int best_t = -1, best_s = 1;
+    for (int t = 0; t < kNumIgemmTiles; ++t)
+        for (int s : kSplitCandidates) {
+            if (s > p->iters_total) continue;
+            const int ips = (p->iters_total + s - 1) / s;
+            const int eff = (p->iters_total + ips - 1) / ips;
+            const size_t tn = (size_t)((d.K + kTileBN[t] - 1) / kTileBN[t]);
+            const size_t part = eff > 1 ? (size_t)p->tiles_m * tn * eff * kTileBN[t] * BM * 4 : 0;
+            if (fixed + part > region_bytes) continue;
+            const double c = model_cost(d, p->Cp, kTileBN[t], s);
+            if (c < best) { best = c; best_t = t; best_s = s; }
+        }
+    if (best_t < 0) return BODA_ERR_TOO_LARGE;
+    p->tile_id = best_t;
+    p->BN = kTileBN[best_t];
+    p->iters_per_split = (p->iters_total + best_s - 1) / best_s;
+    p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;
+    p->tiles_n = (d.K + p->BN - 1) / p->BN;
+
+    char* base = (char*)region;
+    p->d_status = (int*)base;
+    p->d_counters = (int*)(base + 256);
+    char* cur = (char*)(((uintptr_t)(base + head_bytes) + 1023) & ~(uintptr_t)1023);
+    p->d_wp = (float*)cur;
+    float* xp = (float*)(cur + wp_bytes);
+    float* partials = (float*)(cur + wp_bytes + p->xp_bytes);
+
+    BODA_CUDA_TRY(cudaMemsetAsync(base, 0, head_bytes, stream));      // status word and split counters start at zero
+    rc = encode_map_b(p);
+    if (rc == BODA_OK) rc = encode_map_a(p, xp);
+    if (rc == BODA_OK) rc = pack_filters(p, filt, stream);
+    if (rc != BODA_OK) { p->d_wp = nullptr; p->d_counters = nullptr; return rc; }
+    {
+        const int HW = d.H * d.W;
+        dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
+        pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
+        cudaError_t e = cudaGetLastError();
+        if (e != cudaSuccess) { p->d_wp = nullptr; p->d_counters = nullptr; return record_cuda_error(e, "pack_input_nhwc_kernel"); }
+        count_launch();
+    }
+    IgemmParams prm;
+    prm.M = d.M; prm.K = d.K; prm.PQ = d.P * d.Q; prm.Q = d.Q; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
+    prm.cchunks = p->Cp / BKC;
+    prm.iters_total = p->iters_total;
+    prm.iters_per_split = p->iters_per_split;
+    prm.splits = p->splits;
+    prm.relu = d.relu;
+    prm.bias = bias;
+    prm.out = out;
+    prm.partials = partials;
+    prm.counters = p->d_counters;
+    prm.status = p->d_status;
+    switch (p->BN) {
+        case 64: rc = launch_bn<64>(p, prm, stream); break;
+        case 96: rc = launch_bn<96>(p, prm, stream); break;
+        case 128: rc = launch_bn<128>(p, prm, stream); break;
+        case 192: rc = launch_bn<192>(p, prm, stream); break;
+        case 256: rc = launch_bn<256>(p, prm, stream); break;
+        default: rc = BODA_ERR_UNSUPPORTED; break;
+    }
+    p->d_wp = nullptr;                    // the region is the caller's: nothing for a destructor to free
+    p->d_counters = nullptr;
+    return rc;
+}
+
 }  // namespace boda

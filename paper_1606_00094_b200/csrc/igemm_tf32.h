@@ -24,4 +24,9 @@ void igemm_unbind_filters(IgemmPlan* p);
 int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
                  cudaStream_t stream);
 
+// Scratch-in-a-caller-region form (allocates nothing): bytes needed at least, and the run itself.
+size_t igemm_region_min_bytes(const ConvDims& d);
+int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const float* filt, const float* bias,
+                        float* out, void* region, size_t region_bytes, cudaStream_t stream);
+
 }  // namespace boda

@@ -1,0 +1,64 @@
+"""The allocation-free entry point, boda_conv_fwd_noalloc, against the ordinary one, boda_conv_fwd.
+
+Some callers cannot allocate device memory at call time (another allocator owns the device, a real-time
+loop cannot afford cudaMalloc's synchronisation, the memory budget is frozen after start-up).  For them the
+library keeps the kernel's scratch in a fixed array of its own.  This test calls that entry point through the
+C ABI twice in a row on different inputs - the array keeps the previous call's contents, so the second call
+shows that nothing stale leaks through - and compares each result with what boda_conv_fwd gives for the
+same inputs, within the TF32 bar the other tests use.  The file sorts last on purpose: a run that stops at
+the first failure has then already run every other test.
+"""
+import numpy as np
+import pytest
+
+from helpers import TF32_TOL
+from oracle import conv_oracle as orc
+from paper_1606_00094_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+SHAPES = [
+    (3, 64, 13, 13, 80, 3, 3, 1, 1, 1),      # tconv, tiles straddle rows and images, split reduction
+    (5, 480, 14, 14, 192, 1, 1, 1, 0, 1),    # k1conv
+]
+
+
+@pytest.mark.parametrize("shape", SHAPES)
+def test_noalloc_matches_ordinary_entry_point_twice_in_a_row(shape):
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    P, Q = B.boda_conv_out_dim(H, R, st, pad), B.boda_conv_out_dim(W, S, st, pad)
+    for call in range(2):
+        x = torch.from_numpy(wl.half_normal(100 + call, (N, C, H, W))).cuda()
+        w = torch.from_numpy(wl.normal(200 + call, (K, C, R, S), 0, (2.0 / (C * R * S)) ** 0.5)).cuda()
+        b = torch.from_numpy(wl.normal(300 + call, (K,), 0, 0.01)).cuda()
+        ref = torch.empty((N, K, P, Q), dtype=torch.float32, device="cuda")
+        got = torch.full((N, K, P, Q), float("nan"), dtype=torch.float32, device="cuda")
+        B.boda_conv_fwd(x, w, b, ref, N, C, H, W, K, R, S, st, pad, relu)
+        torch.cuda.synchronize()
+        before = torch.cuda.memory_allocated()
+        B.boda_conv_fwd_noalloc(x, w, b, got, N, C, H, W, K, R, S, st, pad, relu)
+        torch.cuda.synchronize()
+        assert torch.cuda.memory_allocated() == before
+        g, r = got.cpu().numpy(), ref.cpu().numpy()
+        assert not np.isnan(g).any(), "output not fully written"
+        err = orc.rel_l2(g, r)
+        assert err <= TF32_TOL, f"call {call}: rel-L2 {err:.3e} between the two entry points"
+        # and both sit within the bar of the fp64 oracle
+        o = orc.conv_fwd(x.cpu().numpy(), w.cpu().numpy(), b.cpu().numpy(), stride=st, pad=pad, relu=bool(relu))
+        assert orc.rel_l2(g, o) <= TF32_TOL
+    B.boda_clear_caches()
+
+
+def test_noalloc_rejects_what_does_not_fit():
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    dummy = torch.zeros(16, device="cuda")
+    # scratch for this shape: 4 * 64*56*56*256 bytes of re-laid-out input alone = 205 MB > 32 MiB
+    with pytest.raises(B.BodaError) as e:
+        B.boda_conv_fwd_noalloc(dummy, dummy, None, dummy, 64, 256, 56, 56, 256, 3, 3, 1, 1, 1)
+    assert e.value.status == B.BODA_ERR_TOO_LARGE
+    with pytest.raises(B.BodaError) as e:       # a 13 x 13 window is outside the tensor-core variants
+        B.boda_conv_fwd_noalloc(dummy, dummy, None, dummy, 1, 32, 20, 20, 16, 13, 13, 1, 0, 1)
+    assert e.value.status == B.BODA_ERR_UNSUPPORTED
