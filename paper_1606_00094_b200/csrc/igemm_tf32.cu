@@ -14,16 +14,20 @@
 // MMA issuer (one elected lane issues tcgen05.mma, tcgen05.commit releases shared-memory stages),
 // warps 2..5 = epilogue (tcgen05.ld of the accumulator, bias, ReLU, store).  This is Listing 1's
 // "load block / fma block / store block" loop with hardware pipelines in place of barriers.
-// Every wait is bounded (two seconds): on expiry the kernel records BODA_ERR_DEVICE_TIMEOUT in the
+// Every wait is bounded (4e9 SM cycles, about two seconds): on expiry the kernel records BODA_ERR_DEVICE_TIMEOUT in the
 // status word, all roles leave their loops, tensor memory is released and the CTA returns.
 #include <cuda.h>
 
 #include <algorithm>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
+#include <vector>
 
 #include "igemm_tf32.h"
+#include "tc_ptx.cuh"
+#include "tconv_halo.cuh"
 
 namespace boda {
 namespace {
@@ -32,7 +36,6 @@ constexpr int BM = 128;          // pixels per CTA tile (UMMA M)
 constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of fp32)
 constexpr int A_STAGE_BYTES = BM * BKC * 4;
 constexpr int kIgemmThreads = 192;
-constexpr unsigned long long kWaitLimitNs = 2000000000ull;
 
 struct IgemmParams {
     int M, K, PQ, Q, stride, pad, S;
@@ -48,140 +51,7 @@ struct IgemmParams {
     int* status;
 };
 
-// ------------------------------------------------------------------------------------------------
-// PTX wrappers
-__device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
-
-__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count)
-{
-    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
-}
-__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes)
-{
-    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
-}
-__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity)
-{
-    uint32_t ok;
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
-        "selp.u32 %0, 1, 0, p;\n\t}"
-        : "=r"(ok) : "r"(bar), "r"(parity) : "memory");
-    return ok != 0;
-}
-__device__ __forceinline__ unsigned long long global_timer_ns()
-{
-    unsigned long long t;
-    asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t));
-    return t;
-}
-
-// Bounded wait.  Returns false if the CTA is aborting or the limit expired (then it raises the abort flag
-// and records where it gave up).
-__device__ __noinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag, int* status, int where)
-{
-    if (mbar_try_wait(bar, parity)) return true;
-    const unsigned long long t0 = global_timer_ns();
-    for (uint32_t spin = 1;; ++spin) {
-        if (mbar_try_wait(bar, parity)) return true;
-        if ((spin & 63u) == 0u) {
-            if (*abort_flag) return false;
-            if (global_timer_ns() - t0 > kWaitLimitNs) {
-                *abort_flag = 1;
-                if (atomicCAS(status, 0, (int)BODA_ERR_DEVICE_TIMEOUT) == 0) {
-                    status[1] = KERNEL_ID_IGEMM;
-                    status[2] = (int)(blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z));
-                    status[3] = where;
-                }
-                return false;
-            }
-        }
-    }
-}
-
-__device__ __forceinline__ void tma_load_im2col_4d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int c, int w,
-                                                   int h, int n, uint16_t off_w, uint16_t off_h)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.4d.shared::cluster.global.im2col.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5, %6}], [%2], {%7, %8};"
-        :: "r"(dst), "l"((uint64_t)map), "r"(bar), "r"(c), "r"(w), "r"(h), "r"(n), "h"(off_w), "h"(off_h)
-        : "memory");
-}
-__device__ __forceinline__ void tma_load_3d(uint32_t dst, const CUtensorMap* map, uint32_t bar, int x, int y, int z)
-{
-    asm volatile(
-        "cp.async.bulk.tensor.3d.shared::cluster.global.mbarrier::complete_tx::bytes"
-        " [%0], [%1, {%3, %4, %5}], [%2];"
-        :: "r"(dst), "l"((uint64_t)map), "r"(bar), "r"(x), "r"(y), "r"(z) : "memory");
-}
-__device__ __forceinline__ void prefetch_tensormap(const CUtensorMap* map)
-{
-    asm volatile("prefetch.tensormap [%0];" ::"l"((uint64_t)map) : "memory");
-}
-
-__device__ __forceinline__ void tmem_alloc(uint32_t dst_smem, uint32_t ncols)
-{
-    asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], %1;" ::"r"(dst_smem), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tmem_relinquish()
-{
-    asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
-}
-__device__ __forceinline__ void tmem_dealloc(uint32_t taddr, uint32_t ncols)
-{
-    asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, %1;" ::"r"(taddr), "r"(ncols) : "memory");
-}
-__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
-__device__ __forceinline__ void tc_commit(uint32_t bar)
-{
-    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
-}
-// D[tmem] (+)= A[smem] * B[smem], TF32 operands, 128 x N x 8 per instruction
-__device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
-{
-    asm volatile(
-        "{\n\t.reg .pred p;\n\t"
-        "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
-        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&v)[32])
-{
-    asm volatile(
-        "tcgen05.ld.sync.aligned.32x32b.x32.b32 "
-        "{%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, "
-        "%16, %17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31}, [%32];"
-        : "=r"(v[0]), "=r"(v[1]), "=r"(v[2]), "=r"(v[3]), "=r"(v[4]), "=r"(v[5]), "=r"(v[6]), "=r"(v[7]),
-          "=r"(v[8]), "=r"(v[9]), "=r"(v[10]), "=r"(v[11]), "=r"(v[12]), "=r"(v[13]), "=r"(v[14]), "=r"(v[15]),
-          "=r"(v[16]), "=r"(v[17]), "=r"(v[18]), "=r"(v[19]), "=r"(v[20]), "=r"(v[21]), "=r"(v[22]), "=r"(v[23]),
-          "=r"(v[24]), "=r"(v[25]), "=r"(v[26]), "=r"(v[27]), "=r"(v[28]), "=r"(v[29]), "=r"(v[30]), "=r"(v[31])
-        : "r"(taddr) : "memory");
-}
-__device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
-
-// Shared-memory matrix descriptor of a K-major tile whose rows are 128 bytes, 128-byte swizzled, with
-// 8-row groups 1024 bytes apart (the layout both TMA loads above produce).
-__device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr)
-{
-    return (uint64_t)((addr & 0x3FFFFu) >> 4)      // start address, 16-byte units
-         | (1ull << 16)                            // leading byte offset (unused for swizzled K-major)
-         | ((uint64_t)(1024 >> 4) << 32)           // stride byte offset: next 8-row group
-         | (1ull << 46)                            // descriptor version of sm_100
-         | (2ull << 61);                           // 128-byte swizzle
-}
-
-template <int BN>
-__host__ __device__ constexpr uint32_t instr_desc_tf32()
-{
-    return (1u << 4)                   // accumulator format: fp32
-         | (2u << 7) | (2u << 10)      // A and B format: TF32
-         | (0u << 15) | (0u << 16)     // A and B are K-major
-         | ((uint32_t)(BN >> 3) << 17) // N
-         | ((uint32_t)(BM >> 4) << 24);// M
-}
+using namespace tc;
 
 template <int BN> struct TileCfg {
     static constexpr int B_STAGE_BYTES = BN * BKC * 4;
@@ -210,6 +80,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
     __shared__ int s_is_last;
+    __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -249,14 +120,17 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             int cc = it_begin - tap * p.cchunks;
             int r = tap / p.S;
             int s = tap - r * p.S;
+            // ring position, parity and addresses advance incrementally: this single thread's loop latency
+            // bounds the iteration rate, so it holds no division
+            uint32_t stage = 0, par = 1;
+            uint32_t fb = full_bar, eb = empty_bar, adst = smem_a, bdst = smem_b;
             for (int i = 0; i < my_iters; ++i) {
-                const int stage = i % STAGES;
-                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-                if (!mbar_wait(empty_bar + 8 * stage, ph ^ 1u, &s_abort, p.status, 1)) break;
-                const uint32_t fb = full_bar + 8 * stage;
+                if (!mbar_wait(eb, par, &s_abort, p.status, 1)) break;
                 mbar_expect_tx(fb, Cfg::STAGE_BYTES);
-                tma_load_im2col_4d(smem_a + stage * A_STAGE_BYTES, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
-                tma_load_3d(smem_b + stage * Cfg::B_STAGE_BYTES, &map_b, fb, cc * BKC, k0, tap);
+                tma_load_im2col_4d(adst, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                tma_load_3d(bdst, &map_b, fb, cc * BKC, k0, tap);
+                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; adst = smem_a; bdst = smem_b; }
+                else { fb += 8; eb += 8; adst += A_STAGE_BYTES; bdst += Cfg::B_STAGE_BYTES; }
                 if (++cc == p.cchunks) { cc = 0; ++tap; if (++s == p.S) { s = 0; ++r; } }
             }
         }
@@ -265,18 +139,22 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             // ---------------- MMA issuer
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
             bool ok = true;
-            for (int i = 0; i < my_iters && ok; ++i) {
-                const int stage = i % STAGES;
-                const uint32_t ph = (uint32_t)(i / STAGES) & 1u;
-                ok = mbar_wait(full_bar + 8 * stage, ph, &s_abort, p.status, 2);
+            uint32_t stage = 0, par = 0;
+            uint32_t fb = full_bar, eb = empty_bar;
+            const uint64_t da0 = smem_desc_k_sw128(smem_a), db0 = smem_desc_k_sw128(smem_b);
+            uint64_t da = da0, db = db0;
+            uint32_t accumulate = 0;
+            for (int i = 0; i < my_iters; ++i) {
+                ok = mbar_wait(fb, par, &s_abort, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t da = smem_desc_k_sw128(smem_a + stage * A_STAGE_BYTES);
-                const uint64_t db = smem_desc_k_sw128(smem_b + stage * Cfg::B_STAGE_BYTES);
 #pragma unroll
                 for (int k = 0; k < BKC / 8; ++k)       // 8 TF32 values = 32 bytes = 2 descriptor units per step
-                    umma_tf32(tmem_acc, da + 2 * k, db + 2 * k, idesc, (i > 0 || k > 0) ? 1u : 0u);
-                tc_commit(empty_bar + 8 * stage);       // frees the stage once these MMAs have read it
+                    umma_tf32(tmem_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
+                accumulate = 1u;
+                tc_commit(eb);                          // frees the stage once these MMAs have read it
+                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; da = da0; db = db0; }
+                else { fb += 8; eb += 8; da += (uint64_t)(A_STAGE_BYTES >> 4); db += (uint64_t)(Cfg::B_STAGE_BYTES >> 4); }
             }
             tc_commit(accum_bar);                       // accumulator complete (or: everything issued so far has drained)
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
@@ -286,7 +164,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         const int m = m0 + row;
-        (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 4);
+        // bias of this tile's channels into shared memory while the main loop runs (0 where there is none)
+        for (int j = threadIdx.x - 64; j < BN; j += 128)
+            s_bias[j] = (p.bias && k0 + j < p.K) ? __ldg(p.bias + k0 + j) : 0.f;
+        if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 4);   // one poller per warp
+        __syncwarp();
         // All 128 epilogue threads meet here whatever their wait returned, then take one common decision:
         // a failed wait has raised the abort flag before returning.
         asm volatile("bar.sync 1, 128;" ::: "memory");
@@ -304,15 +186,21 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 uint32_t v[32];
                 tmem_ld_32cols(trow + j0, v);
                 tmem_ld_wait();
-                if (m_ok) {
+                float y[32];
 #pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        const int k = k0 + j0 + j;
-                        if (k < p.K) {
-                            float y = __uint_as_float(v[j]) + (p.bias ? __ldg(p.bias + k) : 0.f);
-                            if (p.relu) y = fmaxf(y, 0.f);
-                            o[(size_t)k * p.PQ] = y;
-                        }
+                for (int j = 0; j < 32; ++j) {
+                    y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
+                    if (p.relu) y[j] = fmaxf(y[j], 0.f);
+                }
+                if (m_ok) {
+                    float* oj = o + (size_t)(k0 + j0) * p.PQ;
+                    if (k0 + j0 + 32 <= p.K) {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j) oj[(size_t)j * p.PQ] = y[j];
+                    } else {
+#pragma unroll
+                        for (int j = 0; j < 32; ++j)
+                            if (k0 + j0 + j < p.K) oj[(size_t)j * p.PQ] = y[j];
                     }
                 }
             }
@@ -339,14 +227,27 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 const float* base = p.partials + (size_t)tile_lin * p.splits * (BN * BM);
                 if (m_ok) {
                     float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
+                    // 16 channels at a time so that 16 independent loads are in flight per thread
 #pragma unroll 1
-                    for (int j = 0; j < BN; ++j) {
-                        const int k = k0 + j;
-                        if (k >= p.K) break;
-                        float acc = p.bias ? __ldg(p.bias + k) : 0.f;
-                        for (int z = 0; z < p.splits; ++z) acc += __ldcg(base + ((size_t)z * BN + j) * BM + row);
-                        if (p.relu) acc = fmaxf(acc, 0.f);
-                        o[(size_t)k * p.PQ] = acc;
+                    for (int j0 = 0; j0 < BN; j0 += 16) {
+                        if (k0 + j0 >= p.K) break;
+                        float acc[16];
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
+                        for (int z = 0; z < p.splits; ++z) {
+                            const float* src = base + ((size_t)z * BN + j0) * BM + row;
+#pragma unroll
+                            for (int j = 0; j < 16; ++j) acc[j] += __ldcg(src + (size_t)j * BM);
+                        }
+#pragma unroll
+                        for (int j = 0; j < 16; ++j) {
+                            const int k = k0 + j0 + j;
+                            if (k < p.K) {
+                                float y = acc[j] + s_bias[j0 + j];
+                                if (p.relu) y = fmaxf(y, 0.f);
+                                o[(size_t)k * p.PQ] = y;
+                            }
+                        }
                     }
                 }
                 if (threadIdx.x == 64) p.counters[tile_lin] = 0;
@@ -436,8 +337,12 @@ int load_driver_entry_points()
     return BODA_OK;
 }
 
-constexpr int kTileBN[] = {64, 96, 128, 192, 256};
+// Tile table.  Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
+// with NACC accumulators of 128 rows each.
+constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2};
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
+constexpr int kFirstHaloTile = 5;
 constexpr int kSplitCandidates[] = {1, 2, 3, 4, 6, 8};
 
 }  // namespace
@@ -459,7 +364,33 @@ struct IgemmPlan {
     CUtensorMap map_b;
     CUtensorMap map_a;
     const void* map_a_base = nullptr;
+    // halo kernel only
+    int nacc = 0;                    // 0: im2col kernel; 1 or 2: halo kernel with that many accumulators
+    int Hp = 0, Wp = 0, lead = 0, slab_rows = 0, nbox = 0, box_rows = 0, a_slot_bytes = 0, b_stages = 0;
 };
+
+// Geometry of the halo kernel for a shape and tile; false if the shape does not fit it.
+static bool halo_geometry(const ConvDims& d, int BN, int nacc, IgemmPlan* p)
+{
+    if (d.stride != 1 || d.R * d.S < 2) return false;
+    if (d.pad > d.R - 1 || d.pad > d.S - 1) return false;       // output extent must fit the padded row / image pitch
+    const int Hp = d.H + d.pad, Wp = d.W + d.pad;
+    const int slab_rows = 128 * nacc + (d.R - 1) * Wp + (d.S - 1);
+    const int nbox = (slab_rows + 255) / 256;
+    if (nbox > 2) return false;
+    const int box_rows = ((((slab_rows + nbox - 1) / nbox) + 7) / 8) * 8;
+    const int a_slot = nbox * box_rows * 128;
+    const int b_stage = BN * 128;
+    int b_stages = (halo::kSmemBudget - halo::kASlots * a_slot) / b_stage;
+    if (b_stages > halo::kMaxBStages) b_stages = halo::kMaxBStages;
+    if (b_stages < 2) return false;
+    if ((long long)d.N * Hp * Wp > 0x7fffffffLL / 2) return false;
+    if (p) {
+        p->Hp = Hp; p->Wp = Wp; p->lead = d.pad * Wp + d.pad; p->slab_rows = slab_rows; p->nbox = nbox;
+        p->box_rows = box_rows; p->a_slot_bytes = a_slot; p->b_stages = b_stages;
+    }
+    return true;
+}
 
 bool igemm_variant_legal(const ConvDims& d, int variant)
 {
@@ -493,10 +424,65 @@ double model_cost(const ConvDims& d, int Cp, int BN, int splits)
     const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
     const double waves = (double)(long long)((ctas + 147) / 148);
     const double mma_clk = BN * 2.0;                                     // 128 x BN x 32 MACs at 2048 MAC/clk
-    const double feed_clk = (A_STAGE_BYTES + BN * 128.0) / 48.0;         // about 48 B/clk/SM from L2
+    const double feed_clk = (A_STAGE_BYTES + BN * 128.0) / 40.0;         // about 40 B/clk/SM arrive from L2 (measured)
     const double per_iter = std::max(mma_clk, feed_clk);
-    const double epilogue = BN * 6.0 * (splits > 1 ? 2.0 + 0.6 * splits : 1.0) + 1500.0;
+    // epilogue: TMEM read + store; a split adds the parked partial tile and the last CTA's pass over all partials
+    const double epilogue = BN * 8.0 + (splits > 1 ? BN * 128.0 * 4.0 * (1.0 + splits) / 40.0 + 2000.0 : 0.0) + 3000.0;
     return waves * (ips * per_iter + epilogue);
+}
+
+double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
+{
+    const int taps = d.R * d.S;
+    const int iters = taps * (Cp / BKC);
+    const int ips = (iters + splits - 1) / splits;
+    const int Wp = d.W + d.pad, Hp = d.H + d.pad;
+    const long long mflat = (long long)d.N * Hp * Wp;
+    const long long tm = (mflat + 128 * nacc - 1) / (128 * nacc), tn = (d.K + BN - 1) / BN;
+    const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
+    const double waves = (double)(long long)((ctas + 147) / 148);
+    const double mma_clk = BN * 2.0 * nacc;
+    const double slab = (128.0 * nacc + (d.R - 1) * Wp + d.S - 1) * 128.0;
+    const double feed_clk = (BN * 128.0 + slab / taps) / 50.0;
+    const double per_iter = std::max(mma_clk, feed_clk);
+    const double cols = (double)BN * nacc;
+    const double epilogue = cols * 8.0 + (splits > 1 ? cols * 128.0 * 4.0 * (1.0 + splits) / 40.0 + 2000.0 : 0.0) + 3000.0;
+    return waves * (ips * per_iter + epilogue);
+}
+
+template <int BN, int NACC>
+int launch_halo(IgemmPlan* p, const halo::HaloParams& prm, cudaStream_t stream)
+{
+    const int smem = halo::kASlots * p->a_slot_bytes + p->b_stages * BN * 128 + 1024 + 256;
+    static int attr_smem = 0;
+    if (smem > attr_smem) {
+        BODA_CUDA_TRY(cudaFuncSetAttribute(halo::tconv_halo_kernel<BN, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
+        attr_smem = smem;
+    }
+    dim3 grid(p->tiles_m, p->tiles_n, p->splits);
+    halo::tconv_halo_kernel<BN, NACC><<<grid, halo::kThreads, smem, stream>>>(p->map_a, p->map_b, prm);
+    BODA_CUDA_TRY(cudaGetLastError());
+    count_launch();
+    return BODA_OK;
+}
+
+int encode_map_a_halo(IgemmPlan* p, const void* xs)
+{
+    const ConvDims& d = p->d;
+    const cuuint64_t dims[2] = {(cuuint64_t)p->Cp, (cuuint64_t)d.N * p->Hp * p->Wp};
+    const cuuint64_t strides[1] = {(cuuint64_t)p->Cp * 4};
+    const cuuint32_t box[2] = {BKC, (cuuint32_t)p->box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&p->map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, const_cast<void*>(xs), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (halo A) failed with CUresult %d", (int)r);
+        return record_cuda_error(cudaErrorInvalidValue, msg);
+    }
+    p->map_a_base = xs;
+    return BODA_OK;
 }
 
 template <int BN>
@@ -574,10 +560,12 @@ int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, 
     int best_t = 2, best_s = 1;
     for (int t = 0; t < kNumIgemmTiles; ++t) {
         if (tile_id >= 0 && t != tile_id) continue;
+        const int nacc = kTileNacc[t];
+        if (nacc > 0 && (variant != BODA_VARIANT_TCONV || !halo_geometry(d, kTileBN[t], nacc, nullptr))) continue;
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
             if (s > p->iters_total) continue;
-            const double c = model_cost(d, p->Cp, kTileBN[t], s);
+            const double c = nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp, kTileBN[t], s);
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
     }
@@ -585,12 +573,21 @@ int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, 
     if (tile_id >= 0) best_t = tile_id;
     p->tile_id = best_t;
     p->BN = kTileBN[best_t];
+    p->nacc = kTileNacc[best_t];
+    if (p->nacc > 0 && (variant != BODA_VARIANT_TCONV || !halo_geometry(d, p->BN, p->nacc, p))) { delete p; return BODA_ERR_UNSUPPORTED; }
     p->iters_per_split = (p->iters_total + best_s - 1) / best_s;
     p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;   // no empty split
-    p->tiles_m = (d.M + BM - 1) / BM;
     p->tiles_n = (d.K + p->BN - 1) / p->BN;
-    p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
-    p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * BM * 4 : 0;
+    if (p->nacc > 0) {
+        const long long mflat = (long long)d.N * p->Hp * p->Wp;
+        p->tiles_m = (int)((mflat + 128 * p->nacc - 1) / (128 * p->nacc));
+        p->xp_bytes = (((size_t)mflat * p->Cp * 4) + 1023) & ~(size_t)1023;
+        p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * p->nacc * 128 * 4 : 0;
+    } else {
+        p->tiles_m = (d.M + BM - 1) / BM;
+        p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
+        p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * BM * 4 : 0;
+    }
 
     cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cp * 4);
     if (e == cudaSuccess) e = cudaMalloc(&p->d_counters, (size_t)p->tiles_m * p->tiles_n * sizeof(int));
@@ -615,6 +612,11 @@ size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->
 
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
+    if (p->nacc > 0) {
+        std::snprintf(buf, n, "tile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d", 128 * p->nacc, p->BN,
+                      p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits);
+        return;
+    }
     std::snprintf(buf, n, "tile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", p->BN, p->tile_id,
                   p->BN == 64 ? TileCfg<64>::STAGES : p->BN == 96 ? TileCfg<96>::STAGES : p->BN == 128 ? TileCfg<128>::STAGES
                   : p->BN == 192 ? TileCfg<192>::STAGES : TileCfg<256>::STAGES,
@@ -653,6 +655,34 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
+    }
+    if (p->nacc > 0) {
+        dim3 grid((p->Hp * p->Wp + 31) / 32, p->Cp / 32, d.N);
+        halo::pack_input_halo_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, d.H, d.W, p->Hp, p->Wp);
+        BODA_CUDA_TRY(cudaGetLastError());
+        count_launch();
+        if (p->map_a_base != xp) {
+            int rc = encode_map_a_halo(p, xp);
+            if (rc != BODA_OK) return rc;
+        }
+        halo::HaloParams hp;
+        hp.Mflat = d.N * p->Hp * p->Wp; hp.HpWp = p->Hp * p->Wp; hp.Wp = p->Wp; hp.P = d.P; hp.Q = d.Q; hp.K = d.K;
+        hp.S = d.S; hp.taps = d.R * d.S; hp.cchunks = p->Cp / BKC; hp.lead = p->lead;
+        hp.nbox = p->nbox; hp.box_rows = p->box_rows; hp.a_slot_bytes = p->a_slot_bytes; hp.b_stages = p->b_stages;
+        hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
+        hp.relu = d.relu; hp.bias = bias; hp.out = out; hp.partials = partials; hp.counters = p->d_counters;
+        hp.status = p->d_status;
+        switch (p->BN * 10 + p->nacc) {
+            case 641: return launch_halo<64, 1>(p, hp, stream);
+            case 1281: return launch_halo<128, 1>(p, hp, stream);
+            case 1921: return launch_halo<192, 1>(p, hp, stream);
+            case 2561: return launch_halo<256, 1>(p, hp, stream);
+            case 962: return launch_halo<96, 2>(p, hp, stream);
+            case 1282: return launch_halo<128, 2>(p, hp, stream);
+            case 1922: return launch_halo<192, 2>(p, hp, stream);
+            case 2562: return launch_halo<256, 2>(p, hp, stream);
+            default: return BODA_ERR_UNSUPPORTED;
+        }
     }
     {
         const int HW = d.H * d.W;
@@ -725,7 +755,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     // tile and split by the cost model, among the choices whose partial sums still fit the region
     double best = 1e300;
     int best_t = -1, best_s = 1;
-    for (int t = 0; t < kNumIgemmTiles; ++t)
+    for (int t = 0; t < kFirstHaloTile; ++t)
         for (int s : kSplitCandidates) {
             if (s > p->iters_total) continue;
             const int ips = (p->iters_total + s - 1) / s;

@@ -1,0 +1,364 @@
+// TCONV for stride-1 layers with shared-memory reuse of the input across filter taps.
+//
+// The paper's tconv loads whole tiles of `in` once per workgroup and reuses them for every kernel offset,
+// which cuts input traffic by about (KSZ/stride)^2 (Section 5).  Here that reuse is arranged so that the
+// tensor core can read the shifted windows straight from one shared-memory slab:
+//
+//   The input is re-laid-out as rows of a flat matrix xs[(n*Hp + y)*Wp + x][Cp] (NHWC, channels padded to 32,
+//   TF32-rounded) with Hp = H + pad, Wp = W + pad, the extra rows and columns holding zeros.  Because the
+//   right-hand zero columns of one image row double as the left-hand padding of the next row (and the zero
+//   rows below an image as the padding above the next image), the input pixel of output position
+//   f = (n*Hp + p)*Wp + q under tap (r, s) is simply row  f - (pad*Wp + pad) + r*Wp + s  of xs.
+//   A CTA owns 128*NACC consecutive flat positions f.  For each 32-channel chunk it loads ONE slab of
+//   128*NACC + (R-1)*Wp + (S-1) rows (TMA tiled mode; rows before the start of xs are zero-filled) and then,
+//   for every tap, issues the MMAs with the A descriptor advanced by (r*Wp + s) rows of 128 bytes.
+//   Positions with p >= P or q >= Q are computed and dropped (for the AlexNet shapes: 7..16 % of the rows).
+//
+// NACC = 2 keeps two 128-row accumulators in tensor memory so that every filter tile fetched from L2 feeds
+// 256 output rows: operand traffic per MMA cycle halves again.
+// Roles, pipeline and bounded waits are those of the im2col kernel (igemm_tf32.cu).
+#pragma once
+
+#include "tc_ptx.cuh"
+
+namespace boda {
+namespace halo {
+
+using namespace tc;
+
+constexpr int kThreads = 192;
+constexpr int kMaxBStages = 8;
+constexpr int kASlots = 2;
+constexpr int kSmemBudget = 200 * 1024;
+
+struct HaloParams {
+    int Mflat;                   // N * Hp * Wp flat output positions
+    int HpWp, Wp, P, Q, K;
+    int S, taps, cchunks;
+    int lead;                    // pad*Wp + pad
+    int nbox, box_rows;          // slab = nbox TMA boxes of box_rows rows
+    int a_slot_bytes;            // nbox * box_rows * 128, multiple of 1024
+    int b_stages;
+    int iters_total, iters_per_split, splits;
+    int relu;
+    const float* bias;
+    float* out;
+    float* partials;             // [tile][split][NACC*BN][128]
+    int* counters;
+    int* status;
+};
+
+template <int BN, int NACC>
+struct HaloCfg {
+    static constexpr int B_STAGE_BYTES = BN * 128;
+    static constexpr int ACC_COLS = BN * NACC;
+    static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
+    static_assert(ACC_COLS <= 512, "accumulators exceed tensor memory");
+};
+
+template <int BN, int NACC>
+__global__ void __launch_bounds__(kThreads, 1)
+tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
+                  const HaloParams p)
+{
+    using Cfg = HaloCfg<BN, NACC>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    const uint32_t smem_a = smem_base;
+    const uint32_t smem_b = smem_base + kASlots * p.a_slot_bytes;
+    const uint32_t bars = smem_b + p.b_stages * Cfg::B_STAGE_BYTES;
+    const uint32_t a_full = bars, a_empty = bars + 8 * kASlots;
+    const uint32_t b_full = bars + 16 * kASlots, b_empty = b_full + 8 * kMaxBStages;
+    const uint32_t accum_bar = b_empty + 8 * kMaxBStages;
+    __shared__ uint32_t s_tmem_base;
+    __shared__ volatile int s_abort;
+    __shared__ int s_is_last;
+    __shared__ float s_bias[BN];
+
+    const int warp = threadIdx.x >> 5;
+    const int lane = threadIdx.x & 31;
+    const int f0 = blockIdx.x * (128 * NACC);
+    const int k0 = blockIdx.y * BN;
+    const int it_begin = blockIdx.z * p.iters_per_split;
+    const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
+    const int my_iters = it_end - it_begin;
+
+    if (threadIdx.x == 0) {
+        s_abort = 0;
+        for (int s = 0; s < kASlots; ++s) { mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); }
+        for (int s = 0; s < p.b_stages; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1); }
+        mbar_init(accum_bar, 1);
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        prefetch_tensormap(&map_a);
+        prefetch_tensormap(&map_b);
+    }
+    if (warp == 1) {
+        tmem_alloc(smem_u32(&s_tmem_base), Cfg::TMEM_COLS);
+        tmem_relinquish();
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_acc = s_tmem_base;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ---------------- TMA producer.  One thread; ring positions, phases and addresses are advanced
+            // incrementally (no division in the loop): the loop's own latency bounds the iteration rate.
+            const int row0 = f0 - p.lead;                 // may be negative: those rows read as zeros
+            const int chunk0 = it_begin / p.taps;
+            int tap = it_begin - chunk0 * p.taps;
+            int cx = chunk0 * 32;
+            uint32_t a_slot = 0, a_par = 1;               // parity the producer waits for on the empty barriers
+            uint32_t b_stage = 0, b_par = 1;
+            uint32_t bf = b_full, be = b_empty, bdst = smem_b;
+            bool need_slab = true;
+            for (int i = 0; i < my_iters; ++i) {
+                if (need_slab) {
+                    if (!mbar_wait(a_empty + 8 * a_slot, a_par, &s_abort, p.status, 11)) break;
+                    const uint32_t fb = a_full + 8 * a_slot;
+                    mbar_expect_tx(fb, (uint32_t)p.a_slot_bytes);
+                    const uint32_t dst = smem_a + a_slot * p.a_slot_bytes;
+                    tma_load_2d(dst, &map_a, fb, cx, row0);
+                    if (p.nbox > 1) tma_load_2d(dst + p.box_rows * 128, &map_a, fb, cx, row0 + p.box_rows);
+                    a_slot ^= 1u;
+                    if (a_slot == 0) a_par ^= 1u;
+                    need_slab = false;
+                }
+                if (!mbar_wait(be, b_par, &s_abort, p.status, 12)) break;
+                mbar_expect_tx(bf, Cfg::B_STAGE_BYTES);
+                tma_load_3d(bdst, &map_b, bf, cx, k0, tap);
+                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_par ^= 1u; bf = b_full; be = b_empty; bdst = smem_b; }
+                else { bf += 8; be += 8; bdst += Cfg::B_STAGE_BYTES; }
+                if (++tap == p.taps) { tap = 0; cx += 32; need_slab = true; }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ---------------- MMA issuer
+            constexpr uint32_t idesc = instr_desc_tf32<BN>();
+            const int chunk0 = it_begin / p.taps;
+            int tap = it_begin - chunk0 * p.taps;
+            int s = tap % p.S;
+            uint32_t a_row_off = (uint32_t)(tap / p.S) * (uint32_t)p.Wp * 128u;      // r * Wp rows
+            uint32_t a_off = a_row_off + (uint32_t)s * 128u;                          // (r*Wp + s) rows of 128 bytes
+            const uint32_t wp_bytes = (uint32_t)p.Wp * 128u;
+            uint32_t a_slot = 0, a_par = 0, b_stage = 0, b_par = 0;
+            uint32_t bf = b_full, be = b_empty;
+            const uint64_t db0 = smem_desc_k_sw128(smem_b);
+            uint64_t db = db0;
+            uint32_t slab_addr = 0, cur_slot = 0;
+            bool new_slab = true, ok = true;
+            uint32_t accumulate = 0;
+            for (int i = 0; i < my_iters; ++i) {
+                if (new_slab) {
+                    ok = mbar_wait(a_full + 8 * a_slot, a_par, &s_abort, p.status, 13);
+                    if (!ok) break;
+                    slab_addr = smem_a + a_slot * p.a_slot_bytes;
+                    cur_slot = a_slot;
+                    a_slot ^= 1u;
+                    if (a_slot == 0) a_par ^= 1u;
+                    new_slab = false;
+                }
+                ok = mbar_wait(bf, b_par, &s_abort, p.status, 14);
+                if (!ok) break;
+                tc_fence_after();
+                // The A tile of tap (r, s) starts (r*Wp + s) rows into the slab.  The start address may sit on any
+                // 128-byte row: the hardware derives every row's swizzle phase from its shared-memory address bits,
+                // exactly as the TMA write did (measured: the descriptor's base-offset field must stay zero).
+                const uint64_t da = smem_desc_k_sw128(slab_addr + a_off);
+#pragma unroll
+                for (int acc = 0; acc < NACC; ++acc) {
+#pragma unroll
+                    for (int k = 0; k < 4; ++k)
+                        umma_tf32(tmem_acc + acc * BN, da + (uint64_t)(acc * (128 * 128 / 16) + 2 * k), db + 2 * k, idesc,
+                                  (k == 0) ? accumulate : 1u);
+                }
+                accumulate = 1u;
+                tc_commit(be);
+                const bool chunk_done = (tap + 1 == p.taps);
+                if (chunk_done || i + 1 == my_iters) tc_commit(a_empty + 8 * cur_slot);
+                if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_par ^= 1u; bf = b_full; be = b_empty; db = db0; }
+                else { bf += 8; be += 8; db += (uint64_t)(Cfg::B_STAGE_BYTES >> 4); }
+                if (chunk_done) { tap = 0; s = 0; a_row_off = 0; a_off = 0; new_slab = true; }
+                else {
+                    ++tap;
+                    if (++s == p.S) { s = 0; a_row_off += wp_bytes; a_off = a_row_off; } else a_off += 128u;
+                }
+            }
+            tc_commit(accum_bar);
+            if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 15);
+        }
+    } else {
+        // ---------------- epilogue
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        for (int j = threadIdx.x - 64; j < BN; j += 128)
+            s_bias[j] = (p.bias && k0 + j < p.K) ? __ldg(p.bias + k0 + j) : 0.f;
+        if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 16);   // one poller per warp
+        __syncwarp();
+        asm volatile("bar.sync 1, 128;" ::: "memory");
+        const bool ok = (s_abort == 0);
+        tc_fence_after();
+        const int tile_lin = blockIdx.y * gridDim.x + blockIdx.x;
+        const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+        const int PQ = p.P * p.Q;
+        if (ok && p.splits == 1) {
+#pragma unroll 1
+            for (int acc = 0; acc < NACC; ++acc) {
+                const int f = f0 + acc * 128 + row;
+                bool valid = f < p.Mflat;
+                size_t obase = 0;
+                if (valid) {
+                    const int n = f / p.HpWp;
+                    const int rem = f - n * p.HpWp;
+                    const int pp = rem / p.Wp;
+                    const int qq = rem - pp * p.Wp;
+                    valid = pp < p.P && qq < p.Q;
+                    obase = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
+                }
+#pragma unroll 1
+                for (int j0 = 0; j0 < BN; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32cols(trow + acc * BN + j0, v);
+                    tmem_ld_wait();
+                    float y[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) {
+                        y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
+                        if (p.relu) y[j] = fmaxf(y[j], 0.f);
+                    }
+                    if (valid) {
+                        float* oj = p.out + obase + (size_t)(k0 + j0) * PQ;
+                        if (k0 + j0 + 32 <= p.K) {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j) oj[(size_t)j * PQ] = y[j];
+                        } else {
+#pragma unroll
+                            for (int j = 0; j < 32; ++j)
+                                if (k0 + j0 + j < p.K) oj[(size_t)j * PQ] = y[j];
+                        }
+                    }
+                }
+            }
+        } else if (ok) {
+            constexpr int COLS = NACC * BN;
+            float* part = p.partials + ((size_t)tile_lin * p.splits + blockIdx.z) * (size_t)(COLS * 128);
+#pragma unroll 1
+            for (int c0 = 0; c0 < COLS; c0 += 32) {
+                uint32_t v[32];
+                tmem_ld_32cols(trow + c0, v);
+                tmem_ld_wait();
+#pragma unroll
+                for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(c0 + j) * 128 + row, __uint_as_float(v[j]));
+            }
+            __threadfence();
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (threadIdx.x == 64) {
+                const int old = atomicAdd(p.counters + tile_lin, 1);
+                s_is_last = (old == p.splits - 1);
+            }
+            asm volatile("bar.sync 1, 128;" ::: "memory");
+            if (s_is_last) {
+                __threadfence();
+                // thread t sums rows 4*(t%32) .. +3 of the columns c with c % 4 == t/32, as float4 over rows
+                const int t = threadIdx.x - 64;
+                const int rbase = (t & 31) * 4;
+                const int csel = t >> 5;
+                const float* base = p.partials + (size_t)tile_lin * p.splits * (size_t)(COLS * 128);
+#pragma unroll 1
+                for (int acc = 0; acc < NACC; ++acc) {
+                    size_t obase[4];
+                    bool valid[4];
+#pragma unroll
+                    for (int e = 0; e < 4; ++e) {
+                        const int f = f0 + acc * 128 + rbase + e;
+                        valid[e] = f < p.Mflat;
+                        obase[e] = 0;
+                        if (valid[e]) {
+                            const int n = f / p.HpWp;
+                            const int rem = f - n * p.HpWp;
+                            const int pp = rem / p.Wp;
+                            const int qq = rem - pp * p.Wp;
+                            valid[e] = pp < p.P && qq < p.Q;
+                            obase[e] = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
+                        }
+                    }
+#pragma unroll 1
+                    for (int j0 = 0; j0 < BN; j0 += 16) {          // 4 columns per thread per pass
+                        float4 sum[4];
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+                        for (int z = 0; z < p.splits; ++z) {
+#pragma unroll
+                            for (int u = 0; u < 4; ++u) {
+                                const int col = acc * BN + j0 + 4 * u + csel;
+                                const float4 x = __ldcg(reinterpret_cast<const float4*>(
+                                    base + ((size_t)z * COLS + col) * 128 + rbase));
+                                sum[u].x += x.x; sum[u].y += x.y; sum[u].z += x.z; sum[u].w += x.w;
+                            }
+                        }
+#pragma unroll
+                        for (int u = 0; u < 4; ++u) {
+                            const int k = k0 + j0 + 4 * u + csel;
+                            if (k < p.K) {
+                                const float bv = s_bias[j0 + 4 * u + csel];
+                                float y[4] = {sum[u].x + bv, sum[u].y + bv, sum[u].z + bv, sum[u].w + bv};
+#pragma unroll
+                                for (int e = 0; e < 4; ++e) {
+                                    if (p.relu) y[e] = fmaxf(y[e], 0.f);
+                                    if (valid[e]) p.out[obase[e] + (size_t)k * PQ] = y[e];
+                                }
+                            }
+                        }
+                    }
+                }
+                if (threadIdx.x == 64) p.counters[tile_lin] = 0;
+            }
+        }
+        tc_fence_before();
+    }
+    __syncthreads();
+    if (warp == 1) {
+        __syncwarp();
+        tc_fence_after();
+        tmem_dealloc(tmem_acc, Cfg::TMEM_COLS);
+    }
+}
+
+// NCHW -> flat padded NHWC rows [(n*Hp + y)*Wp + x][Cp]; zeros in the padded rows, columns and channels;
+// values rounded to TF32 (nearest, ties away).
+__global__ void __launch_bounds__(256)
+pack_input_halo_kernel(const float* __restrict__ in, float* __restrict__ xs, int C, int Cp, int H, int W, int Hp, int Wp)
+{
+    __shared__ float tile[32][33];
+    const int n = blockIdx.z;
+    const int f0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const int HpWp = Hp * Wp;
+    const float* src = in + (size_t)n * C * H * W;
+    float* dst = xs + (size_t)n * HpWp * Cp;
+    {
+        const int f = f0 + tx;
+        const int y = f / Wp, x = f - y * Wp;
+        const bool inside = f < HpWp && y < H && x < W;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = c0 + ty + 8 * i;
+            tile[ty + 8 * i][tx] = (inside && c < C) ? __ldg(src + ((size_t)c * H + y) * W + x) : 0.f;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int f = f0 + ty + 8 * i, c = c0 + tx;
+        if (f < HpWp) {
+            uint32_t r;
+            asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(tile[tx][ty + 8 * i]));
+            dst[(size_t)f * Cp + c] = __uint_as_float(r);
+        }
+    }
+}
+
+}  // namespace halo
+}  // namespace boda

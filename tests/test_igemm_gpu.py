@@ -102,3 +102,41 @@ def test_same_result_twice_bitwise_and_tuned_plan():
     np.testing.assert_array_equal(a, c)          # split reduction is summed in split order: deterministic
     t, desc = run_planned(shape, x, w, b, tune=1)
     assert_parity(t, oracle_out(shape, x, w, b), TF32_TOL, desc)
+
+
+# ---------------------------------------------------------------- halo (input-reuse) tconv kernel, tile ids 5..12
+HALO_SHAPES = [
+    (1, 32, 6, 6, 16, 3, 3, 1, 1, 0),            # one tile
+    (3, 64, 13, 13, 80, 3, 3, 1, 1, 1),          # conv3-like, images share their zero rows
+    (2, 96, 27, 27, 72, 5, 5, 1, 2, 1),          # conv2-like: slab of 248 / 376 rows
+    (2, 40, 12, 10, 24, 3, 3, 1, 0, 0),          # no padding: outputs narrower than the row pitch
+    (2, 32, 9, 11, 40, 2, 4, 1, 1, 1),           # R != S, even sizes
+    (1, 48, 57, 57, 96, 3, 3, 1, 0, 1),          # space-to-depth view of an 11x11 stride-4 layer
+    (2, 33, 8, 8, 300, 3, 3, 1, 2, 1),           # pad = window - 1: output larger than the input
+]
+
+
+@pytest.mark.parametrize("tile", [5, 6, 7, 8, 9, 10, 11, 12])
+@pytest.mark.parametrize("shape", HALO_SHAPES)
+def test_halo_tiles_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 1100)
+    got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile)
+    assert "halo" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+@pytest.mark.parametrize("tile,split", [(6, 2), (7, 3), (10, 2), (11, 4), (12, 8), (9, 6)])
+def test_halo_split_exact(tile, split):
+    shape = (3, 96, 13, 13, 272, 3, 3, 1, 1, 1)
+    x, w, b = _int_tensors(shape, 1200)
+    got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile, split_k=split)
+    assert "halo" in desc and "split_k=1 " not in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_halo_refused_where_it_does_not_apply():
+    from paper_1606_00094_b200 import binding as B
+    for shape in [(2, 32, 15, 17, 24, 3, 3, 2, 1, 0), (1, 32, 5, 5, 16, 3, 3, 1, 3, 0), (1, 32, 8, 8, 16, 1, 1, 1, 0, 0)]:
+        with pytest.raises(B.BodaError) as e:
+            B.ConvPlan(shape, variant=TC if shape[5] > 1 else K1, tile_id=6)
+        assert e.value.status == B.BODA_ERR_UNSUPPORTED
