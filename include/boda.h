@@ -71,6 +71,10 @@ typedef struct boda_plan_opts {
     int tile_id;                 /* -1: automatic; otherwise index into the variant's tile table */
     int split_k;                 /* 0: automatic; otherwise the number of reduction splits of a tensor-core variant */
     int device;                  /* CUDA device ordinal; -1: the current device */
+    int s2d;                     /* strided TCONV layers: -1 automatic, 0 never, 1 always run the stride-1
+                                    "space-to-depth" view (stride t on C channels = stride 1 on C*t*t channels
+                                    with ceil(R/t) x ceil(S/t) taps); an input transformation in the sense of
+                                    Section 5 of the paper */
 } boda_plan_opts;
 
 typedef struct boda_conv_plan boda_conv_plan;   /* opaque; created and destroyed by the library */

@@ -37,7 +37,7 @@ class boda_conv_shape(ctypes.Structure):
 
 
 class boda_plan_opts(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("math", "tune", "variant", "tile_id", "split_k", "device")]
+    _fields_ = [(n, ctypes.c_int) for n in ("math", "tune", "variant", "tile_id", "split_k", "device", "s2d")]
 
 
 _vp = ctypes.c_void_p
@@ -212,11 +212,11 @@ def boda_clear_caches() -> None:
 class ConvPlan:
     """Owns a plan handle and its workspace; ``plan(x, w, b)`` runs the layer into a new tensor."""
 
-    def __init__(self, shape, math=BODA_MATH_AUTO, variant=BODA_VARIANT_AUTO, tile_id=-1, split_k=0, tune=0):
+    def __init__(self, shape, math=BODA_MATH_AUTO, variant=BODA_VARIANT_AUTO, tile_id=-1, split_k=0, tune=0, s2d=-1):
         import torch
         self.shape = tuple(int(v) for v in shape)
         o = boda_plan_opts_default()
-        o.math, o.variant, o.tile_id, o.split_k, o.tune = math, variant, tile_id, split_k, tune
+        o.math, o.variant, o.tile_id, o.split_k, o.tune, o.s2d = math, variant, tile_id, split_k, tune, s2d
         self.handle = boda_conv_plan_create(self.shape, o)
         nbytes = boda_conv_plan_workspace_bytes(self.handle)
         self.workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda") if nbytes else None

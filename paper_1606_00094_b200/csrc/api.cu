@@ -125,6 +125,7 @@ void boda_plan_opts_default(boda_plan_opts* o)
     o->tile_id = -1;
     o->split_k = 0;
     o->device = -1;
+    o->s2d = -1;
 }
 
 int boda_conv_plan_destroy(boda_conv_plan* plan)
@@ -167,12 +168,11 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
         p->ws_bytes = 0;
     } else {
         p->math = BODA_MATH_TF32;
-        rc = igemm_plan_create(p->d, variant, tile_id, split_k, ctx->d_status, &p->ig);
+        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig);
         if (rc == BODA_OK) { p->tile_id = igemm_plan_tile(p->ig); p->ws_bytes = igemm_plan_workspace_bytes(p->ig); }
     }
     if (rc != BODA_OK) { boda_conv_plan_destroy(p); return rc; }
     *out = p;
-    (void)o;
     return BODA_OK;
 }
 

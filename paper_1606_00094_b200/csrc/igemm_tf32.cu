@@ -46,8 +46,6 @@ struct IgemmParams {
     int relu;
     const float* bias;
     float* out;
-    float* partials;             // [tile][split][BN][128], splits > 1 only
-    int* counters;               // [tile], zero between launches
     int* status;
 };
 
@@ -79,7 +77,6 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t accum_bar = bars + 16 * STAGES;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ int s_is_last;
     __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
@@ -178,7 +175,6 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         int n = 0, pq = 0;
         if (m_ok) { n = m / p.PQ; pq = m - n * p.PQ; }
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-        const int tile_lin = blockIdx.y * gridDim.x + blockIdx.x;
         if (ok && p.splits == 1) {
             float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
 #pragma unroll 1
@@ -205,57 +201,36 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 }
             }
         } else if (ok) {
-            // split reduction: park the partial tile, the CTA that arrives last sums all partials in split order
-            float* part = p.partials + ((size_t)tile_lin * p.splits + blockIdx.z) * (BN * BM);
+            // split reduction, step 1: park this CTA's partial accumulator in its own shared memory (the stage
+            // buffers are idle now), column-major [channel][128 rows]; the cluster-wide sum follows below.
 #pragma unroll 1
             for (int j0 = 0; j0 < BN; j0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(trow + j0, v);
                 tmem_ld_wait();
 #pragma unroll
-                for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(j0 + j) * BM + row, __uint_as_float(v[j]));
-            }
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (threadIdx.x == 64) {
-                const int old = atomicAdd(p.counters + tile_lin, 1);
-                s_is_last = (old == p.splits - 1);
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (s_is_last) {
-                __threadfence();
-                const float* base = p.partials + (size_t)tile_lin * p.splits * (BN * BM);
-                if (m_ok) {
-                    float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
-                    // 16 channels at a time so that 16 independent loads are in flight per thread
-#pragma unroll 1
-                    for (int j0 = 0; j0 < BN; j0 += 16) {
-                        if (k0 + j0 >= p.K) break;
-                        float acc[16];
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) acc[j] = 0.f;
-                        for (int z = 0; z < p.splits; ++z) {
-                            const float* src = base + ((size_t)z * BN + j0) * BM + row;
-#pragma unroll
-                            for (int j = 0; j < 16; ++j) acc[j] += __ldcg(src + (size_t)j * BM);
-                        }
-#pragma unroll
-                        for (int j = 0; j < 16; ++j) {
-                            const int k = k0 + j0 + j;
-                            if (k < p.K) {
-                                float y = acc[j] + s_bias[j0 + j];
-                                if (p.relu) y = fmaxf(y, 0.f);
-                                o[(size_t)k * p.PQ] = y;
-                            }
-                        }
-                    }
-                }
-                if (threadIdx.x == 64) p.counters[tile_lin] = 0;
+                for (int j = 0; j < 32; ++j) st_shared_f32(smem_base + (uint32_t)((j0 + j) * 128 + row) * 4u, __uint_as_float(v[j]));
             }
         }
         tc_fence_before();
     }
     __syncthreads();
+    if (p.splits > 1) {
+        // split reduction, step 2: the CTAs of one output tile form a cluster (one per split); after the
+        // cluster barrier each of them sums its share of the channels over all peers' shared memory and stores it.
+        cluster_sync_all();
+        if (warp >= 2 && s_abort == 0) {
+            auto row_info = [&](int row, bool& valid, size_t& obase) {
+                const int m = m0 + row;
+                valid = m < p.M;
+                obase = 0;
+                if (valid) { const int n = m / p.PQ; obase = ((size_t)n * p.K) * p.PQ + (size_t)(m - n * p.PQ); }
+            };
+            cluster_reduce_store<BN>(smem_base, (int)threadIdx.x - 64, cluster_cta_rank(), p.splits, row_info, (size_t)p.PQ,
+                                     k0, p.K, p.relu, s_bias, p.out);
+        }
+        cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -311,6 +286,73 @@ pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int 
     }
 }
 
+// Space-to-depth staging for strided layers.  A convolution with stride t on C channels equals a stride-1
+// convolution with ceil(R/t) x ceil(S/t) taps on C*t*t channels, where "channel" (dy, dx, c) of block (yb, xb)
+// is pixel (yb*t + dy, xb*t + dx) of the zero-padded input and the filter taps past R or S are zeros.  It turns
+// a first layer such as 11x11 stride 4 on 3 channels into a 3x3 stride-1 layer on 48 channels, which the
+// tensor-core kernels can run; the paper's tconv likewise needs "an input transformation" (Section 5).
+// One CTA builds one block-row: it stages the t input rows of all channels in shared memory with coalesced
+// reads, then writes the [W'][Cp] row of blocks contiguously.
+__global__ void __launch_bounds__(256)
+pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int C, int H, int W, int t, int pad,
+                      int Hb, int Wb, int Cp)
+{
+    extern __shared__ float sm_rows[];            // [C][t][W]
+    const int yb = blockIdx.x, n = blockIdx.y;
+    const int tW = t * W;
+    for (int idx = threadIdx.x; idx < C * tW; idx += blockDim.x) {
+        const int c = idx / tW;
+        const int rem = idx - c * tW;
+        const int dy = rem / W;
+        const int x = rem - dy * W;
+        const int y = yb * t + dy - pad;
+        sm_rows[idx] = (y >= 0 && y < H) ? __ldg(in + (((size_t)n * C + c) * H + y) * W + x) : 0.f;
+    }
+    __syncthreads();
+    float* dst = xs + ((size_t)n * Hb + yb) * Wb * Cp;
+    const int Cs = C * t * t;
+    for (int o = threadIdx.x; o < Wb * Cp; o += blockDim.x) {
+        const int xb = o / Cp;
+        const int cp = o - xb * Cp;
+        float v = 0.f;
+        if (cp < Cs) {
+            const int g = cp / C;
+            const int c = cp - g * C;
+            const int dy = g / t;
+            const int dx = g - dy * t;
+            const int x = xb * t + dx - pad;
+            if (x >= 0 && x < W) v = sm_rows[(c * t + dy) * W + x];
+        }
+        dst[o] = round_tf32(v);
+    }
+}
+
+// filters KCRS -> [Rb*Sb][K][Cp] for the space-to-depth view (zeros where the tap or channel does not exist)
+__global__ void __launch_bounds__(256)
+pack_filters_s2d_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int R, int S, int t,
+                        int Rb, int Sb, int Cp)
+{
+    const long long total = (long long)Rb * Sb * K * Cp;
+    const int Cs = C * t * t;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int cp = (int)(idx % Cp);
+        const long long u = idx / Cp;
+        const int k = (int)(u % K);
+        const int tapb = (int)(u / K);
+        const int rb = tapb / Sb, sb = tapb - rb * Sb;
+        float v = 0.f;
+        if (cp < Cs) {
+            const int g = cp / C;
+            const int c = cp - g * C;
+            const int dy = g / t, dx = g - dy * t;
+            const int r = rb * t + dy, sx = sb * t + dx;
+            if (r < R && sx < S) v = __ldg(filt + (((size_t)k * C + c) * R + r) * S + sx);
+        }
+        wp[idx] = round_tf32(v);
+    }
+}
+
 // ------------------------------------------------------------------------------------------------
 // Host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
@@ -348,7 +390,9 @@ constexpr int kSplitCandidates[] = {1, 2, 3, 4, 6, 8};
 }  // namespace
 
 struct IgemmPlan {
-    ConvDims d;
+    ConvDims d;                      // the problem the kernels run (the space-to-depth view if s2d)
+    ConvDims orig;                   // the layer as given
+    bool s2d = false;
     int variant = 0;
     int tile_id = 0;
     int BN = 128;
@@ -358,7 +402,6 @@ struct IgemmPlan {
     int tiles_m = 0, tiles_n = 0;
     int* d_status = nullptr;
     float* d_wp = nullptr;           // packed filters [RS][K][Cp]
-    int* d_counters = nullptr;       // [tiles_m * tiles_n]
     const float* bound_filt = nullptr;
     size_t xp_bytes = 0, partial_bytes = 0;
     CUtensorMap map_b;
@@ -392,6 +435,37 @@ static bool halo_geometry(const ConvDims& d, int BN, int nacc, IgemmPlan* p)
     return true;
 }
 
+// Space-to-depth view of a strided layer (see pack_input_s2d_kernel); false if it does not apply.
+static bool s2d_view(const ConvDims& d, ConvDims* e)
+{
+    const int t = d.stride;
+    if (t < 2 || t > 4 || d.R * d.S < 2) return false;
+    if ((size_t)d.C * t * d.W * 4 > 40 * 1024) return false;       // shared-memory staging of the pack kernel
+    if ((long long)d.C * t * t > 1024) return false;
+    ConvDims v = d;
+    v.C = d.C * t * t;
+    v.R = (d.R + t - 1) / t;
+    v.S = (d.S + t - 1) / t;
+    v.H = d.P - 1 + v.R;
+    v.W = d.Q - 1 + v.S;
+    v.stride = 1;
+    v.pad = 0;
+    v.Kred = v.C * v.R * v.S;
+    if (e) *e = v;
+    return true;
+}
+
+bool igemm_s2d_applicable(const ConvDims& d) { return s2d_view(d, nullptr); }
+
+// Fraction of the multiply-accumulates of the space-to-depth view that are real work.
+static double s2d_efficiency(const ConvDims& d)
+{
+    ConvDims e;
+    if (!s2d_view(d, &e)) return 0.0;
+    const int Cp = ((e.C + BKC - 1) / BKC) * BKC;
+    return (double)d.C * d.R * d.S / ((double)Cp * e.R * e.S);
+}
+
 bool igemm_variant_legal(const ConvDims& d, int variant)
 {
     if (d.R > 11 || d.S > 11 || d.stride > 8 || d.pad > 100) return false;
@@ -405,7 +479,8 @@ bool igemm_variant_profitable(const ConvDims& d)
 {
     // Channels are padded to 32 per reduction chunk and pixels to 128 per tile: tiny C (first layers) and tiny
     // layers stay on the FP32 kernel.
-    return d.C >= 16 && d.K >= 16 && (long long)d.M * d.K >= 128 * 64;
+    if (d.K < 16 || (long long)d.M * d.K < 128 * 64) return false;
+    return d.C >= 16 || s2d_efficiency(d) >= 0.35;
 }
 
 int igemm_num_tiles() { return kNumIgemmTiles; }
@@ -414,40 +489,56 @@ int igemm_split_candidate(int i) { return kSplitCandidates[i]; }
 
 namespace {
 
-// Rough cost model (clocks) used when the plan is not tuned by timing: MMA issue versus operand bytes from L2.
+// Cost model (SM clocks) used when a plan is not tuned by timing.  Calibrated on B200: one thread issues the MMAs of
+// a stage, and a stage costs about 290 clocks of MMA issue per 128-row accumulator plus about 240 (im2col kernel) or
+// 390 (halo kernel) clocks of barrier hand-shakes, unless the MMAs themselves take longer (2*BN clocks per 32
+// channels and accumulator).  Prologue, pipeline fill and tail cost about 4500 clocks; the epilogue about 22 clocks
+// per channel, a cluster split reduction about 6 + 30/splits per channel plus 2500.
+double epilogue_cost(double cols, int splits)
+{
+    return splits > 1 ? cols * (6.0 + 30.0 / splits) + 2500.0 : cols * 22.0;
+}
+
 double model_cost(const ConvDims& d, int Cp, int BN, int splits)
 {
-    const int taps = d.R * d.S;
-    const int iters = taps * (Cp / BKC);
+    const int iters = d.R * d.S * (Cp / BKC);
     const int ips = (iters + splits - 1) / splits;
     const long long tm = (d.M + BM - 1) / BM, tn = (d.K + BN - 1) / BN;
     const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
     const double waves = (double)(long long)((ctas + 147) / 148);
-    const double mma_clk = BN * 2.0;                                     // 128 x BN x 32 MACs at 2048 MAC/clk
-    const double feed_clk = (A_STAGE_BYTES + BN * 128.0) / 40.0;         // about 40 B/clk/SM arrive from L2 (measured)
-    const double per_iter = std::max(mma_clk, feed_clk);
-    // epilogue: TMEM read + store; a split adds the parked partial tile and the last CTA's pass over all partials
-    const double epilogue = BN * 8.0 + (splits > 1 ? BN * 128.0 * 4.0 * (1.0 + splits) / 40.0 + 2000.0 : 0.0) + 3000.0;
-    return waves * (ips * per_iter + epilogue);
+    const double per_iter = std::max(2.0 * BN, 530.0);
+    return waves * (ips * per_iter + 4500.0 + epilogue_cost(BN, splits));
 }
 
 double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
 {
-    const int taps = d.R * d.S;
-    const int iters = taps * (Cp / BKC);
+    const int iters = d.R * d.S * (Cp / BKC);
     const int ips = (iters + splits - 1) / splits;
-    const int Wp = d.W + d.pad, Hp = d.H + d.pad;
-    const long long mflat = (long long)d.N * Hp * Wp;
+    const long long mflat = (long long)d.N * (d.H + d.pad) * (d.W + d.pad);
     const long long tm = (mflat + 128 * nacc - 1) / (128 * nacc), tn = (d.K + BN - 1) / BN;
     const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
     const double waves = (double)(long long)((ctas + 147) / 148);
-    const double mma_clk = BN * 2.0 * nacc;
-    const double slab = (128.0 * nacc + (d.R - 1) * Wp + d.S - 1) * 128.0;
-    const double feed_clk = (BN * 128.0 + slab / taps) / 50.0;
-    const double per_iter = std::max(mma_clk, feed_clk);
-    const double cols = (double)BN * nacc;
-    const double epilogue = cols * 8.0 + (splits > 1 ? cols * 128.0 * 4.0 * (1.0 + splits) / 40.0 + 2000.0 : 0.0) + 3000.0;
-    return waves * (ips * per_iter + epilogue);
+    const double per_iter = std::max(2.2 * BN * nacc, 290.0 * nacc + 390.0);
+    return waves * (ips * per_iter + 5000.0 + nacc * epilogue_cost(BN, splits));
+}
+
+// Launch with the CTAs of one output tile (grid.z = reduction splits) grouped into a thread-block cluster.
+template <typename Kernel, typename... Args>
+cudaError_t launch_clustered(Kernel kernel, dim3 grid, int threads, int smem, cudaStream_t stream, int cluster_z, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = dim3(threads);
+    cfg.dynamicSmemBytes = (size_t)smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = 1;
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = (unsigned)cluster_z;
+    cfg.attrs = attr;
+    cfg.numAttrs = cluster_z > 1 ? 1 : 0;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
 template <int BN, int NACC>
@@ -460,8 +551,8 @@ int launch_halo(IgemmPlan* p, const halo::HaloParams& prm, cudaStream_t stream)
         attr_smem = smem;
     }
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    halo::tconv_halo_kernel<BN, NACC><<<grid, halo::kThreads, smem, stream>>>(p->map_a, p->map_b, prm);
-    BODA_CUDA_TRY(cudaGetLastError());
+    BODA_CUDA_TRY(launch_clustered(halo::tconv_halo_kernel<BN, NACC>, grid, halo::kThreads, smem, stream, p->splits,
+                                   p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
 }
@@ -495,8 +586,8 @@ int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
         attr_set = true;
     }
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    igemm_tf32_kernel<BN><<<grid, kIgemmThreads, Cfg::SMEM_BYTES, stream>>>(p->map_a, p->map_b, prm);
-    BODA_CUDA_TRY(cudaGetLastError());
+    BODA_CUDA_TRY(launch_clustered(igemm_tf32_kernel<BN>, grid, kIgemmThreads, Cfg::SMEM_BYTES, stream, p->splits,
+                                   p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
 }
@@ -541,16 +632,29 @@ int encode_map_b(IgemmPlan* p)
 
 }  // namespace
 
-int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int* d_status, IgemmPlan** out)
+int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out)
 {
-    if (!igemm_variant_legal(d, variant)) return BODA_ERR_UNSUPPORTED;
+    if (!igemm_variant_legal(d_in, variant)) return BODA_ERR_UNSUPPORTED;
+    // strided tconv layers may run as their stride-1 space-to-depth view
+    ConvDims d = d_in;
+    bool use_s2d = false;
+    if (variant == BODA_VARIANT_TCONV && s2d != 0) {
+        ConvDims e;
+        const bool can = s2d_view(d_in, &e);
+        if (s2d > 0 && !can) return BODA_ERR_UNSUPPORTED;
+        if (can && (s2d > 0 || s2d_efficiency(d_in) >= 0.35)) { d = e; use_s2d = true; }
+    } else if (s2d > 0) {
+        return BODA_ERR_UNSUPPORTED;
+    }
     if (tile_id >= kNumIgemmTiles) return BODA_ERR_UNSUPPORTED;
-    if (split_k < 0 || split_k > 64) return BODA_ERR_INVALID_ARG;
+    if (split_k < 0 || split_k > 8) return BODA_ERR_INVALID_ARG;   // one cluster (at most 8 CTAs) per output tile
     int rc = load_driver_entry_points();
     if (rc != BODA_OK) return rc;
     IgemmPlan* p = new (std::nothrow) IgemmPlan();
     if (!p) return BODA_ERR_NOMEM;
     p->d = d;
+    p->orig = d_in;
+    p->s2d = use_s2d;
     p->variant = variant;
     p->d_status = d_status;
     p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
@@ -582,16 +686,14 @@ int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, 
         const long long mflat = (long long)d.N * p->Hp * p->Wp;
         p->tiles_m = (int)((mflat + 128 * p->nacc - 1) / (128 * p->nacc));
         p->xp_bytes = (((size_t)mflat * p->Cp * 4) + 1023) & ~(size_t)1023;
-        p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * p->nacc * 128 * 4 : 0;
+        p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     } else {
         p->tiles_m = (d.M + BM - 1) / BM;
         p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
-        p->partial_bytes = p->splits > 1 ? (size_t)p->tiles_m * p->tiles_n * p->splits * p->BN * BM * 4 : 0;
+        p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     }
 
     cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cp * 4);
-    if (e == cudaSuccess) e = cudaMalloc(&p->d_counters, (size_t)p->tiles_m * p->tiles_n * sizeof(int));
-    if (e == cudaSuccess) e = cudaMemset(p->d_counters, 0, (size_t)p->tiles_m * p->tiles_n * sizeof(int));
     if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
     rc = encode_map_b(p);
     if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -603,7 +705,6 @@ void igemm_plan_destroy(IgemmPlan* p)
 {
     if (!p) return;
     if (p->d_wp) cudaFree(p->d_wp);
-    if (p->d_counters) cudaFree(p->d_counters);
     delete p;
 }
 
@@ -612,12 +713,13 @@ size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->
 
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
+    const char* view = p->s2d ? "s2d " : "";
     if (p->nacc > 0) {
-        std::snprintf(buf, n, "tile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d", 128 * p->nacc, p->BN,
+        std::snprintf(buf, n, "%stile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d", view, 128 * p->nacc, p->BN,
                       p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits);
         return;
     }
-    std::snprintf(buf, n, "tile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", p->BN, p->tile_id,
+    std::snprintf(buf, n, "%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->BN, p->tile_id,
                   p->BN == 64 ? TileCfg<64>::STAGES : p->BN == 96 ? TileCfg<96>::STAGES : p->BN == 128 ? TileCfg<128>::STAGES
                   : p->BN == 192 ? TileCfg<192>::STAGES : TileCfg<256>::STAGES,
                   p->splits, p->tiles_m, p->tiles_n, p->splits);
@@ -628,6 +730,10 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const ConvDims& d = p->d;
     const long long total = (long long)d.R * d.S * d.K * p->Cp;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
+    if (p->s2d) {
+        const ConvDims& o = p->orig;
+        pack_filters_s2d_kernel<<<blocks, 256, 0, stream>>>(filt, p->d_wp, o.K, o.C, o.R, o.S, o.stride, d.R, d.S, p->Cp);
+    } else
     pack_filters_kernel<<<blocks, 256, 0, stream>>>(filt, p->d_wp, d.K, d.C, p->Cp, d.R * d.S);
     BODA_CUDA_TRY(cudaGetLastError());
     count_launch();
@@ -650,17 +756,27 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     if (!workspace) return BODA_ERR_NOMEM;
     if (((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
     float* xp = (float*)workspace;
-    float* partials = (float*)((char*)workspace + p->xp_bytes);
     if (filt != p->bound_filt || !filt) {
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
     }
-    if (p->nacc > 0) {
-        dim3 grid((p->Hp * p->Wp + 31) / 32, p->Cp / 32, d.N);
-        halo::pack_input_halo_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, d.H, d.W, p->Hp, p->Wp);
+    if (p->s2d) {
+        // both kernels read the same [N][H'][W'][Cp] layout here (the view has no padding)
+        const ConvDims& o = p->orig;
+        dim3 grid(d.H, d.N);
+        const size_t smem = (size_t)o.C * o.stride * o.W * 4;
+        pack_input_s2d_kernel<<<grid, 256, smem, stream>>>(in, xp, o.C, o.H, o.W, o.stride, o.pad, d.H, d.W, p->Cp);
         BODA_CUDA_TRY(cudaGetLastError());
         count_launch();
+    }
+    if (p->nacc > 0) {
+        if (!p->s2d) {
+            dim3 grid((p->Hp * p->Wp + 31) / 32, p->Cp / 32, d.N);
+            halo::pack_input_halo_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, d.H, d.W, p->Hp, p->Wp);
+            BODA_CUDA_TRY(cudaGetLastError());
+            count_launch();
+        }
         if (p->map_a_base != xp) {
             int rc = encode_map_a_halo(p, xp);
             if (rc != BODA_OK) return rc;
@@ -670,7 +786,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         hp.S = d.S; hp.taps = d.R * d.S; hp.cchunks = p->Cp / BKC; hp.lead = p->lead;
         hp.nbox = p->nbox; hp.box_rows = p->box_rows; hp.a_slot_bytes = p->a_slot_bytes; hp.b_stages = p->b_stages;
         hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
-        hp.relu = d.relu; hp.bias = bias; hp.out = out; hp.partials = partials; hp.counters = p->d_counters;
+        hp.relu = d.relu; hp.bias = bias; hp.out = out;
         hp.status = p->d_status;
         switch (p->BN * 10 + p->nacc) {
             case 641: return launch_halo<64, 1>(p, hp, stream);
@@ -684,7 +800,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
             default: return BODA_ERR_UNSUPPORTED;
         }
     }
-    {
+    if (!p->s2d) {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
         pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
@@ -704,8 +820,6 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     prm.relu = d.relu;
     prm.bias = bias;
     prm.out = out;
-    prm.partials = partials;
-    prm.counters = p->d_counters;
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: return launch_bn<64>(p, prm, stream);
@@ -743,6 +857,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     IgemmPlan plan;                       // lives on the host stack for the duration of this call only
     IgemmPlan* p = &plan;
     p->d = d;
+    p->orig = d;
     p->variant = variant;
     p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
     p->iters_total = d.R * d.S * (p->Cp / BKC);
@@ -760,9 +875,8 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
             if (s > p->iters_total) continue;
             const int ips = (p->iters_total + s - 1) / s;
             const int eff = (p->iters_total + ips - 1) / ips;
-            const size_t tn = (size_t)((d.K + kTileBN[t] - 1) / kTileBN[t]);
-            const size_t part = eff > 1 ? (size_t)p->tiles_m * tn * eff * kTileBN[t] * BM * 4 : 0;
-            if (fixed + part > region_bytes) continue;
+            (void)eff;
+            if (fixed > region_bytes) continue;
             const double c = model_cost(d, p->Cp, kTileBN[t], s);
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
@@ -775,23 +889,21 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
 
     char* base = (char*)region;
     p->d_status = (int*)base;
-    p->d_counters = (int*)(base + 256);
     char* cur = (char*)(((uintptr_t)(base + head_bytes) + 1023) & ~(uintptr_t)1023);
     p->d_wp = (float*)cur;
     float* xp = (float*)(cur + wp_bytes);
-    float* partials = (float*)(cur + wp_bytes + p->xp_bytes);
 
-    BODA_CUDA_TRY(cudaMemsetAsync(base, 0, head_bytes, stream));      // status word and split counters start at zero
+    BODA_CUDA_TRY(cudaMemsetAsync(base, 0, head_bytes, stream));      // the status word starts at zero
     rc = encode_map_b(p);
     if (rc == BODA_OK) rc = encode_map_a(p, xp);
     if (rc == BODA_OK) rc = pack_filters(p, filt, stream);
-    if (rc != BODA_OK) { p->d_wp = nullptr; p->d_counters = nullptr; return rc; }
+    if (rc != BODA_OK) { p->d_wp = nullptr; return rc; }
     {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
         pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
         cudaError_t e = cudaGetLastError();
-        if (e != cudaSuccess) { p->d_wp = nullptr; p->d_counters = nullptr; return record_cuda_error(e, "pack_input_nhwc_kernel"); }
+        if (e != cudaSuccess) { p->d_wp = nullptr; return record_cuda_error(e, "pack_input_nhwc_kernel"); }
         count_launch();
     }
     IgemmParams prm;
@@ -803,8 +915,6 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     prm.relu = d.relu;
     prm.bias = bias;
     prm.out = out;
-    prm.partials = partials;
-    prm.counters = p->d_counters;
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: rc = launch_bn<64>(p, prm, stream); break;
@@ -815,7 +925,6 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
         default: rc = BODA_ERR_UNSUPPORTED; break;
     }
     p->d_wp = nullptr;                    // the region is the caller's: nothing for a destructor to free
-    p->d_counters = nullptr;
     return rc;
 }
 

@@ -166,6 +166,102 @@ __device__ __forceinline__ uint64_t smem_desc_k_sw128(uint32_t addr)
          | (2ull << 61);                           // 128-byte swizzle
 }
 
+// ---- thread-block cluster helpers (split reductions through distributed shared memory)
+__device__ __forceinline__ void cluster_sync_all()
+{
+    asm volatile("barrier.cluster.arrive.release;\n\tbarrier.cluster.wait.acquire;" ::: "memory");
+}
+__device__ __forceinline__ uint32_t cluster_cta_rank()
+{
+    uint32_t r;
+    asm volatile("mov.u32 %0, %%cluster_ctarank;" : "=r"(r));
+    return r;
+}
+// shared-memory address of the same variable in the CTA of the given rank of this cluster
+__device__ __forceinline__ uint32_t map_to_cta(uint32_t local_smem_addr, uint32_t rank)
+{
+    uint32_t r;
+    asm volatile("mapa.shared::cluster.u32 %0, %1, %2;" : "=r"(r) : "r"(local_smem_addr), "r"(rank));
+    return r;
+}
+__device__ __forceinline__ float ld_cluster_f32(uint32_t addr)
+{
+    float v;
+    asm volatile("ld.shared::cluster.f32 %0, [%1];" : "=f"(v) : "r"(addr) : "memory");
+    return v;
+}
+__device__ __forceinline__ void st_shared_f32(uint32_t addr, float v)
+{
+    asm volatile("st.shared.f32 [%0], %1;" :: "r"(addr), "f"(v) : "memory");
+}
+
+__device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+
+// Split reduction of one 128-row accumulator over the CTAs of a cluster (one CTA per reduction split).
+// Every CTA has parked its partial accumulator in its own shared memory at `stash`, column-major
+// [col][128 rows]; the cluster has synchronised.  CTA `rank` owns the columns rank*per .. and sums them over
+// all CTAs in rank order (so the result does not depend on which CTA does the summing), adds the bias,
+// applies ReLU and stores: each split CTA writes its share of the output tile.
+// Work split inside the CTA (128 epilogue threads, t = 0..127): thread t sums rows 4*(t%32) .. +3 (one 16-byte
+// remote load per peer and column) of the columns c with (c - c_begin) % 4 == t/32, eight columns per pass so
+// that 8 x splits remote loads are in flight (remote shared memory has the latency of an L2 access).
+// `row_info(row, valid, obase)` locates a row in `out`: element (row, k) lives at out[obase + k * k_stride].
+template <int BN, typename RowInfo>
+__device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int t, uint32_t rank, int splits, RowInfo row_info,
+                                                     size_t k_stride, int k0, int K, int relu, const float* s_bias,
+                                                     float* out)
+{
+    const int per = (((BN + splits - 1) / splits) + 3) & ~3;
+    const int c_begin = (int)rank * per;
+    const int c_end = min(BN, c_begin + per);
+    const int rbase = (t & 31) * 4;
+    const int csel = t >> 5;
+    bool valid[4];
+    size_t obase[4];
+#pragma unroll
+    for (int e = 0; e < 4; ++e) row_info(rbase + e, valid[e], obase[e]);
+    uint32_t peer[8];
+#pragma unroll
+    for (int r = 0; r < 8; ++r) peer[r] = r < splits ? map_to_cta(stash + (uint32_t)rbase * 4u, (uint32_t)r) : 0u;
+#pragma unroll 1
+    for (int c0 = c_begin + csel; c0 < c_end; c0 += 32) {
+        float4 sum[8];
+#pragma unroll
+        for (int u = 0; u < 8; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int r = 0; r < 8; ++r) {
+            if (r < splits) {
+#pragma unroll
+                for (int u = 0; u < 8; ++u) {
+                    const int c = c0 + 4 * u;
+                    if (c < c_end) {
+                        const float4 x = ld_cluster_v4(peer[r] + (uint32_t)c * 512u);
+                        sum[u].x += x.x; sum[u].y += x.y; sum[u].z += x.z; sum[u].w += x.w;
+                    }
+                }
+            }
+        }
+#pragma unroll
+        for (int u = 0; u < 8; ++u) {
+            const int c = c0 + 4 * u, k = k0 + c;
+            if (c < c_end && k < K) {
+                const float bv = s_bias[c];
+                float y[4] = {sum[u].x + bv, sum[u].y + bv, sum[u].z + bv, sum[u].w + bv};
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    if (relu) y[e] = fmaxf(y[e], 0.f);
+                    if (valid[e]) out[obase[e] + (size_t)k * k_stride] = y[e];
+                }
+            }
+        }
+    }
+}
+
 template <int BN>
 __host__ __device__ constexpr uint32_t instr_desc_tf32()
 {

@@ -43,8 +43,6 @@ struct HaloParams {
     int relu;
     const float* bias;
     float* out;
-    float* partials;             // [tile][split][NACC*BN][128]
-    int* counters;
     int* status;
 };
 
@@ -72,7 +70,6 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t accum_bar = b_empty + 8 * kMaxBStages;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ int s_is_last;
     __shared__ float s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
@@ -200,7 +197,6 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const bool ok = (s_abort == 0);
         tc_fence_after();
-        const int tile_lin = blockIdx.y * gridDim.x + blockIdx.x;
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         const int PQ = p.P * p.Q;
         if (ok && p.splits == 1) {
@@ -241,84 +237,55 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     }
                 }
             }
-        } else if (ok) {
-            constexpr int COLS = NACC * BN;
-            float* part = p.partials + ((size_t)tile_lin * p.splits + blockIdx.z) * (size_t)(COLS * 128);
-#pragma unroll 1
-            for (int c0 = 0; c0 < COLS; c0 += 32) {
-                uint32_t v[32];
-                tmem_ld_32cols(trow + c0, v);
-                tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) __stcg(part + (size_t)(c0 + j) * 128 + row, __uint_as_float(v[j]));
-            }
-            __threadfence();
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (threadIdx.x == 64) {
-                const int old = atomicAdd(p.counters + tile_lin, 1);
-                s_is_last = (old == p.splits - 1);
-            }
-            asm volatile("bar.sync 1, 128;" ::: "memory");
-            if (s_is_last) {
-                __threadfence();
-                // thread t sums rows 4*(t%32) .. +3 of the columns c with c % 4 == t/32, as float4 over rows
-                const int t = threadIdx.x - 64;
-                const int rbase = (t & 31) * 4;
-                const int csel = t >> 5;
-                const float* base = p.partials + (size_t)tile_lin * p.splits * (size_t)(COLS * 128);
-#pragma unroll 1
-                for (int acc = 0; acc < NACC; ++acc) {
-                    size_t obase[4];
-                    bool valid[4];
-#pragma unroll
-                    for (int e = 0; e < 4; ++e) {
-                        const int f = f0 + acc * 128 + rbase + e;
-                        valid[e] = f < p.Mflat;
-                        obase[e] = 0;
-                        if (valid[e]) {
-                            const int n = f / p.HpWp;
-                            const int rem = f - n * p.HpWp;
-                            const int pp = rem / p.Wp;
-                            const int qq = rem - pp * p.Wp;
-                            valid[e] = pp < p.P && qq < p.Q;
-                            obase[e] = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
-                        }
-                    }
-#pragma unroll 1
-                    for (int j0 = 0; j0 < BN; j0 += 16) {          // 4 columns per thread per pass
-                        float4 sum[4];
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
-                        for (int z = 0; z < p.splits; ++z) {
-#pragma unroll
-                            for (int u = 0; u < 4; ++u) {
-                                const int col = acc * BN + j0 + 4 * u + csel;
-                                const float4 x = __ldcg(reinterpret_cast<const float4*>(
-                                    base + ((size_t)z * COLS + col) * 128 + rbase));
-                                sum[u].x += x.x; sum[u].y += x.y; sum[u].z += x.z; sum[u].w += x.w;
-                            }
-                        }
-#pragma unroll
-                        for (int u = 0; u < 4; ++u) {
-                            const int k = k0 + j0 + 4 * u + csel;
-                            if (k < p.K) {
-                                const float bv = s_bias[j0 + 4 * u + csel];
-                                float y[4] = {sum[u].x + bv, sum[u].y + bv, sum[u].z + bv, sum[u].w + bv};
-#pragma unroll
-                                for (int e = 0; e < 4; ++e) {
-                                    if (p.relu) y[e] = fmaxf(y[e], 0.f);
-                                    if (valid[e]) p.out[obase[e] + (size_t)k * PQ] = y[e];
-                                }
-                            }
-                        }
-                    }
-                }
-                if (threadIdx.x == 64) p.counters[tile_lin] = 0;
-            }
         }
         tc_fence_before();
     }
     __syncthreads();
+    if (p.splits > 1) {
+        // Split reduction through the cluster (one CTA per split), one 128-row accumulator at a time: park the
+        // partial accumulator in this CTA's own shared memory (the operand buffers are idle now), synchronise the
+        // cluster, sum this CTA's share of the channels over all peers and store it.
+        const bool ok = (s_abort == 0);
+        const int quarter = warp & 3;
+        const int row = quarter * 32 + lane;
+        const uint32_t rank = cluster_cta_rank();
+#pragma unroll 1
+        for (int acc = 0; acc < NACC; ++acc) {
+            if (warp >= 2 && ok) {
+                const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16) + acc * BN;
+                tc_fence_after();
+#pragma unroll 1
+                for (int j0 = 0; j0 < BN; j0 += 32) {
+                    uint32_t v[32];
+                    tmem_ld_32cols(trow + j0, v);
+                    tmem_ld_wait();
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) st_shared_f32(smem_base + (uint32_t)((j0 + j) * 128 + row) * 4u, __uint_as_float(v[j]));
+                }
+                tc_fence_before();
+            }
+            cluster_sync_all();
+            if (warp >= 2 && ok) {
+                const int PQ = p.P * p.Q;
+                auto row_info = [&](int r, bool& valid, size_t& obase) {
+                    const int f = f0 + acc * 128 + r;
+                    valid = f < p.Mflat;
+                    obase = 0;
+                    if (valid) {
+                        const int n = f / p.HpWp;
+                        const int rem = f - n * p.HpWp;
+                        const int pp = rem / p.Wp;
+                        const int qq = rem - pp * p.Wp;
+                        valid = pp < p.P && qq < p.Q;
+                        obase = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
+                    }
+                };
+                cluster_reduce_store<BN>(smem_base, (int)threadIdx.x - 64, rank, p.splits, row_info, (size_t)PQ, k0, p.K,
+                                         p.relu, s_bias, p.out);
+            }
+            cluster_sync_all();      // peers are done with this CTA's shared memory
+        }
+    }
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();

@@ -8,11 +8,11 @@ FP32_TOL = 1e-5   # relative L2 bar of the FP32 CUDA-core path
 TF32_TOL = 5e-3   # relative L2 bar of the TF32 tensor-core path
 
 
-def run_planned(shape, x, w, b, *, variant=-1, math=0, tile_id=-1, split_k=0, bind=False, tune=0):
+def run_planned(shape, x, w, b, *, variant=-1, math=0, tile_id=-1, split_k=0, bind=False, tune=0, s2d=-1):
     """shape = (N,C,H,W,K,R,S,stride,pad,relu); x,w,b numpy fp32.  Returns (out numpy, description)."""
     import torch
     from paper_1606_00094_b200 import binding as B
-    plan = B.ConvPlan(shape, math=math, variant=variant, tile_id=tile_id, split_k=split_k, tune=tune)
+    plan = B.ConvPlan(shape, math=math, variant=variant, tile_id=tile_id, split_k=split_k, tune=tune, s2d=s2d)
     try:
         dx = torch.from_numpy(x).cuda()
         dw = torch.from_numpy(w).cuda()

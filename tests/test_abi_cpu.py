@@ -55,4 +55,4 @@ def test_argument_validation_needs_no_device():
     assert B.boda_status_string(0) == "ok" and "timeout" not in B.boda_status_string(1)
     assert B.boda_version() >= 100
     o = B.boda_plan_opts_default()
-    assert (o.math, o.tune, o.variant, o.tile_id, o.split_k, o.device) == (0, 0, -1, -1, 0, -1)
+    assert (o.math, o.tune, o.variant, o.tile_id, o.split_k, o.device, o.s2d) == (0, 0, -1, -1, 0, -1, -1)

@@ -138,5 +138,48 @@ def test_halo_refused_where_it_does_not_apply():
     from paper_1606_00094_b200 import binding as B
     for shape in [(2, 32, 15, 17, 24, 3, 3, 2, 1, 0), (1, 32, 5, 5, 16, 3, 3, 1, 3, 0), (1, 32, 8, 8, 16, 1, 1, 1, 0, 0)]:
         with pytest.raises(B.BodaError) as e:
-            B.ConvPlan(shape, variant=TC if shape[5] > 1 else K1, tile_id=6)
+            B.ConvPlan(shape, variant=TC if shape[5] > 1 else K1, tile_id=6, s2d=0)
         assert e.value.status == B.BODA_ERR_UNSUPPORTED
+
+
+# ---------------------------------------------------------------- space-to-depth view of strided layers
+S2D_SHAPES = [
+    (1, 3, 43, 43, 24, 11, 11, 4, 0, 1),         # AlexNet conv1-like: 11x11 stride 4 on 3 channels -> 3x3 on 48
+    (2, 3, 227, 227, 96, 11, 11, 4, 0, 1),       # the real conv1 shape at batch 2
+    (2, 20, 15, 17, 24, 3, 5, 2, 1, 0),          # stride 2 with padding, R != S
+    (2, 8, 16, 16, 40, 2, 2, 2, 0, 1),           # window = stride: the view is a 1x1 convolution
+    (1, 5, 20, 23, 33, 7, 7, 3, 3, 0),           # stride 3, window not a multiple of the stride, padding
+    (3, 16, 9, 9, 16, 3, 3, 2, 1, 1),
+]
+
+
+@pytest.mark.parametrize("shape", S2D_SHAPES)
+@pytest.mark.parametrize("tile", [-1, 1, 6, 10])
+def test_space_to_depth_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 1300)
+    try:
+        got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile, s2d=1)
+    except Exception as e:                       # a halo tile is refused when the view has a single tap
+        from paper_1606_00094_b200 import binding as B
+        assert isinstance(e, B.BodaError) and e.status == B.BODA_ERR_UNSUPPORTED and tile in (6, 10) and shape[5] <= shape[7]
+        return
+    assert "s2d" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_space_to_depth_off_and_auto_agree_with_oracle():
+    shape = (2, 3, 99, 99, 96, 11, 11, 4, 0, 1)
+    x, w, b = _real_tensors(shape, 1400)
+    ref = oracle_out(shape, x, w, b)
+    a, da = run_planned(shape, x, w, b, variant=TC, s2d=0)
+    c, dc = run_planned(shape, x, w, b)                      # automatic: tconv through the space-to-depth view
+    assert "s2d" not in da and "s2d" in dc and "tconv" in dc
+    assert_parity(a, ref, TF32_TOL, da)
+    assert_parity(c, ref, TF32_TOL, dc)
+
+
+def test_space_to_depth_refused_for_stride_one():
+    from paper_1606_00094_b200 import binding as B
+    with pytest.raises(B.BodaError) as e:
+        B.ConvPlan((1, 32, 8, 8, 16, 3, 3, 1, 1, 0), variant=TC, s2d=1)
+    assert e.value.status == B.BODA_ERR_UNSUPPORTED
