@@ -110,6 +110,10 @@ int boda_conv_plan_describe(const boda_conv_plan* plan, char* buf, size_t buf_by
  * and split-reduction partial sums. */
 size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* plan);
 
+/* Kernels one boda_conv_fwd_planned call launches when the filters are bound (1 for DIRECT; 2 for the
+ * tensor-core variants: input staging and the main kernel). */
+int boda_conv_plan_kernels_per_call(const boda_conv_plan* plan);
+
 /*
  * Optional: pre-pack the filters (and remember the bias pointer's contents are NOT copied) for a
  * tensor-core plan, so that boda_conv_fwd_planned can skip the per-call filter re-layout.  Weights
@@ -191,6 +195,52 @@ int boda_conv_fwd_noalloc(const float* in, const float* filt, const float* bias,
  */
 int boda_maxpool_fwd(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,
                      void* stream);
+
+/*
+ * A chain of layers run as one unit: convolutions (each followed by its bias and ReLU) and max-pools, layer
+ * i+1 reading layer i's output - the shape of a CNN's convolutional trunk such as the AlexNet-shaped stack the
+ * benchmark uses.  (The paper's framework runs a whole compute graph, Section 4 and Figure "Boda flow"; this is
+ * the minimal form of it: a linear chain.)  The stack owns its plans, the activations between layers, one
+ * workspace and a CUDA graph of the chain, so that boda_stack_fwd is one graph launch.
+ */
+enum { BODA_STACK_CONV = 0, BODA_STACK_MAXPOOL = 1 };
+typedef struct boda_stack_op {
+    int kind;                    /* BODA_STACK_CONV or BODA_STACK_MAXPOOL */
+    boda_conv_shape conv;        /* CONV: the layer; its N, C, H, W must equal the previous op's output */
+    int ksz, stride;             /* MAXPOOL: window and stride (no padding, floor extent) */
+} boda_stack_op;
+typedef struct boda_stack boda_stack;
+
+/* Plans every convolution with `opts` (NULL = defaults) and allocates activations and workspace.  The first op
+ * must be a convolution (it fixes the input extent).  Errors as boda_conv_plan_create, INVALID_ARG if shapes do
+ * not chain. */
+int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts* opts, boda_stack** stack);
+int boda_stack_destroy(boda_stack* stack);
+int boda_stack_num_ops(const boda_stack* stack);
+/* Device pointers to the filters [K][C][R][S] and bias [K] (or NULL) of convolution op `op_index`; the stack keeps
+ * the pointers (the caller keeps the memory alive) and pre-packs the filters on `stream`. */
+int boda_stack_set_filters(boda_stack* stack, int op_index, const float* filt, const float* bias, void* stream);
+/* Output extent [N][C][H][W] of op `op_index`. */
+int boda_stack_out_dims(const boda_stack* stack, int op_index, int* N, int* C, int* H, int* W);
+/* Device pointer to the activation that op `op_index` writes (not for the last op, which writes the caller's buffer). */
+int boda_stack_layer_output(const boda_stack* stack, int op_index, const float** ptr);
+int boda_stack_describe(const boda_stack* stack, int op_index, char* buf, size_t buf_bytes);
+/* Kernels one forward pass launches. */
+int boda_stack_kernels_per_fwd(const boda_stack* stack);
+/*
+ * Forward pass, device pointers: in [N][C][H][W] of the first op, out = output of the last op.  The first call
+ * for a given (in, out) pair runs the chain once eagerly on `stream` and captures it into a CUDA graph (this
+ * allocates and must not itself be inside a stream capture); later calls with the same pointers are one
+ * cudaGraphLaunch on `stream`.  Asynchronous.
+ */
+int boda_stack_fwd(boda_stack* stack, const float* in, float* out, void* stream);
+/* Same without the graph: the kernels are launched one by one on `stream`.  `events`, if not NULL, points to
+ * 3 * n_ops cudaEvent_t handles; for op i the library records events[3i] before its first kernel, events[3i+1]
+ * between operand staging and the main kernel, and events[3i+2] after its last kernel (per-layer timing). */
+int boda_stack_fwd_eager(boda_stack* stack, const float* in, float* out, void* stream, void** events);
+/* Forward pass with HOST buffers: copies `in_host` to the device, runs boda_stack_fwd, copies the result into
+ * `out_host` and synchronises `stream`.  Pinned host memory makes the copies asynchronous. */
+int boda_stack_fwd_host(boda_stack* stack, const float* in_host, float* out_host, void* stream);
 
 /*
  * Reads the device-side status word of the current device: kernels never trap or spin for ever;

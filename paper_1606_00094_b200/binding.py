@@ -36,6 +36,13 @@ class boda_conv_shape(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("N", "C", "H", "W", "K", "R", "S", "stride", "pad", "relu")]
 
 
+class boda_stack_op(ctypes.Structure):
+    _fields_ = [("kind", ctypes.c_int), ("conv", boda_conv_shape), ("ksz", ctypes.c_int), ("stride", ctypes.c_int)]
+
+
+BODA_STACK_CONV, BODA_STACK_MAXPOOL = 0, 1
+
+
 class boda_plan_opts(ctypes.Structure):
     _fields_ = [(n, ctypes.c_int) for n in ("math", "tune", "variant", "tile_id", "split_k", "device", "s2d")]
 
@@ -66,6 +73,30 @@ _lib.boda_conv_fwd_noalloc.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd_noalloc.restype = _i
 _lib.boda_maxpool_fwd.argtypes = [_vp, _vp] + [_i] * 6 + [_vp]
 _lib.boda_maxpool_fwd.restype = _i
+_lib.boda_conv_plan_kernels_per_call.argtypes = [_vp]
+_lib.boda_conv_plan_kernels_per_call.restype = _i
+_lib.boda_stack_create.argtypes = [ctypes.POINTER(boda_stack_op), _i, ctypes.POINTER(boda_plan_opts), ctypes.POINTER(_vp)]
+_lib.boda_stack_create.restype = _i
+_lib.boda_stack_destroy.argtypes = [_vp]
+_lib.boda_stack_destroy.restype = _i
+_lib.boda_stack_num_ops.argtypes = [_vp]
+_lib.boda_stack_num_ops.restype = _i
+_lib.boda_stack_set_filters.argtypes = [_vp, _i, _vp, _vp, _vp]
+_lib.boda_stack_set_filters.restype = _i
+_lib.boda_stack_out_dims.argtypes = [_vp, _i] + [ctypes.POINTER(_i)] * 4
+_lib.boda_stack_out_dims.restype = _i
+_lib.boda_stack_layer_output.argtypes = [_vp, _i, ctypes.POINTER(_vp)]
+_lib.boda_stack_layer_output.restype = _i
+_lib.boda_stack_describe.argtypes = [_vp, _i, ctypes.c_char_p, ctypes.c_size_t]
+_lib.boda_stack_describe.restype = _i
+_lib.boda_stack_kernels_per_fwd.argtypes = [_vp]
+_lib.boda_stack_kernels_per_fwd.restype = _i
+_lib.boda_stack_fwd.argtypes = [_vp, _vp, _vp, _vp]
+_lib.boda_stack_fwd.restype = _i
+_lib.boda_stack_fwd_eager.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(_vp)]
+_lib.boda_stack_fwd_eager.restype = _i
+_lib.boda_stack_fwd_host.argtypes = [_vp, _vp, _vp, _vp]
+_lib.boda_stack_fwd_host.restype = _i
 _lib.boda_query_status.argtypes = [_vp, ctypes.POINTER(_i)]
 _lib.boda_query_status.restype = _i
 _lib.boda_clear_caches.argtypes = []
@@ -194,6 +225,73 @@ def boda_conv_fwd_noalloc(inp, filt, bias, out, N, C, H, W, K, R, S, stride, pad
 
 def boda_maxpool_fwd(inp, out, N, C, H, W, ksz=3, stride=2, stream=None) -> None:
     _check(_lib.boda_maxpool_fwd(_addr(inp), _addr(out), N, C, H, W, ksz, stride, _stream(stream)), "boda_maxpool_fwd")
+
+
+def boda_conv_plan_kernels_per_call(plan: int) -> int:
+    return int(_lib.boda_conv_plan_kernels_per_call(plan))
+
+
+def boda_stack_create(ops, opts: Optional[boda_plan_opts] = None) -> int:
+    """ops: list of boda_stack_op.  Returns the stack handle."""
+    arr = (boda_stack_op * len(ops))(*ops)
+    handle = _vp()
+    _check(_lib.boda_stack_create(arr, len(ops), ctypes.byref(opts) if opts is not None else None, ctypes.byref(handle)),
+           "boda_stack_create")
+    return handle.value
+
+
+def boda_stack_destroy(stack: int) -> None:
+    _check(_lib.boda_stack_destroy(stack), "boda_stack_destroy")
+
+
+def boda_stack_num_ops(stack: int) -> int:
+    return int(_lib.boda_stack_num_ops(stack))
+
+
+def boda_stack_set_filters(stack: int, op_index: int, filt, bias, stream=None) -> None:
+    _check(_lib.boda_stack_set_filters(stack, op_index, _addr(filt), _addr(bias), _stream(stream)), "boda_stack_set_filters")
+
+
+def boda_stack_out_dims(stack: int, op_index: int):
+    v = [_i(0) for _ in range(4)]
+    _check(_lib.boda_stack_out_dims(stack, op_index, *[ctypes.byref(x) for x in v]), "boda_stack_out_dims")
+    return tuple(x.value for x in v)
+
+
+def boda_stack_layer_output(stack: int, op_index: int) -> int:
+    ptr = _vp()
+    _check(_lib.boda_stack_layer_output(stack, op_index, ctypes.byref(ptr)), "boda_stack_layer_output")
+    return ptr.value
+
+
+def boda_stack_describe(stack: int, op_index: int) -> str:
+    buf = ctypes.create_string_buffer(512)
+    _check(_lib.boda_stack_describe(stack, op_index, buf, 512), "boda_stack_describe")
+    return buf.value.decode()
+
+
+def boda_stack_kernels_per_fwd(stack: int) -> int:
+    return int(_lib.boda_stack_kernels_per_fwd(stack))
+
+
+def boda_stack_fwd(stack: int, inp, out, stream=None) -> None:
+    _check(_lib.boda_stack_fwd(stack, _addr(inp), _addr(out), _stream(stream)), "boda_stack_fwd")
+
+
+def boda_stack_fwd_eager(stack: int, inp, out, stream=None, events=None) -> None:
+    """events: optional flat list of 3 * n_ops torch.cuda.Event objects (already created, timing enabled)."""
+    arr = None
+    if events is not None:
+        handles = []
+        for e in events:
+            e.record()            # torch creates the underlying cudaEvent lazily: record once to materialise it
+            handles.append(e.cuda_event)
+        arr = (_vp * len(handles))(*handles)
+    _check(_lib.boda_stack_fwd_eager(stack, _addr(inp), _addr(out), _stream(stream), arr), "boda_stack_fwd_eager")
+
+
+def boda_stack_fwd_host(stack: int, inp_host, out_host, stream=None) -> None:
+    _check(_lib.boda_stack_fwd_host(stack, _addr(inp_host), _addr(out_host), _stream(stream)), "boda_stack_fwd_host")
 
 
 def boda_query_status(stream=None) -> int:

@@ -106,6 +106,28 @@ struct boda_conv_plan {
     size_t ws_bytes = 0;
 };
 
+namespace boda {
+
+int conv_fwd_planned_ex(boda_conv_plan* p, const float* in, const float* filt, const float* bias, float* out,
+                        void* workspace, cudaStream_t stream, cudaEvent_t after_staging)
+{
+    if (!p || !in || !out) return BODA_ERR_INVALID_ARG;
+    if (p->variant == BODA_VARIANT_DIRECT) {
+        if (!filt) return BODA_ERR_INVALID_ARG;
+        if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
+        return direct_launch(p->d, p->tile_id, in, filt, bias, out, p->d_tab, stream);
+    }
+    if (p->ws_bytes && !workspace) return BODA_ERR_NOMEM;
+    return igemm_launch(p->ig, in, filt, bias, out, workspace, stream, after_staging);
+}
+
+void conv_plan_out_dims(const boda_conv_plan* p, int* N, int* K, int* P, int* Q)
+{
+    *N = p->d.N; *K = p->d.K; *P = p->d.P; *Q = p->d.Q;
+}
+
+}  // namespace boda
+
 extern "C" {
 
 int boda_conv_out_dim(int in_dim, int ksz, int stride, int pad)
@@ -261,6 +283,12 @@ int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
 
 size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* p) { return p ? p->ws_bytes : 0; }
 
+int boda_conv_plan_kernels_per_call(const boda_conv_plan* p)
+{
+    if (!p) return 0;
+    return p->variant == BODA_VARIANT_DIRECT ? 1 : 2;      // tensor-core variants: input staging + main kernel
+}
+
 int boda_conv_plan_bind_filters(boda_conv_plan* p, const float* filt, void* stream)
 {
     if (!p || !filt) return BODA_ERR_INVALID_ARG;
@@ -271,13 +299,7 @@ int boda_conv_plan_bind_filters(boda_conv_plan* p, const float* filt, void* stre
 int boda_conv_fwd_planned(boda_conv_plan* p, const float* in, const float* filt, const float* bias, float* out,
                           void* workspace, void* stream)
 {
-    if (!p || !in || !out) return BODA_ERR_INVALID_ARG;
-    if (p->variant == BODA_VARIANT_DIRECT) {
-        if (!filt) return BODA_ERR_INVALID_ARG;
-        return direct_launch(p->d, p->tile_id, in, filt, bias, out, p->d_tab, (cudaStream_t)stream);
-    }
-    if (p->ws_bytes && !workspace) return BODA_ERR_NOMEM;
-    return igemm_launch(p->ig, in, filt, bias, out, workspace, (cudaStream_t)stream);
+    return boda::conv_fwd_planned_ex(p, in, filt, bias, out, workspace, (cudaStream_t)stream, nullptr);
 }
 
 }  // extern "C"

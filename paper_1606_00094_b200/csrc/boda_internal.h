@@ -58,6 +58,11 @@ void direct_build_table(const ConvDims& d, DirectTapEntry* host_tab);
 int direct_launch(const ConvDims& d, int tile_id, const float* in, const float* filt, const float* bias,
                   float* out, const DirectTapEntry* dev_tab, cudaStream_t stream);
 
+// ---- the planned forward pass with an optional event between operand staging and the main kernel
+int conv_fwd_planned_ex(boda_conv_plan* plan, const float* in, const float* filt, const float* bias, float* out,
+                        void* workspace, cudaStream_t stream, cudaEvent_t after_staging);
+void conv_plan_out_dims(const boda_conv_plan* plan, int* N, int* K, int* P, int* Q);
+
 // ---- pooling -------------------------------------------------------------------------------------
 int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,
                    cudaStream_t stream);

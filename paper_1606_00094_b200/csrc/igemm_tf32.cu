@@ -750,7 +750,7 @@ int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
 void igemm_unbind_filters(IgemmPlan* p) { p->bound_filt = nullptr; }
 
 int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
-                 cudaStream_t stream)
+                 cudaStream_t stream, cudaEvent_t after_staging)
 {
     const ConvDims& d = p->d;
     if (!workspace) return BODA_ERR_NOMEM;
@@ -781,6 +781,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
             int rc = encode_map_a_halo(p, xp);
             if (rc != BODA_OK) return rc;
         }
+        if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
         halo::HaloParams hp;
         hp.Mflat = d.N * p->Hp * p->Wp; hp.HpWp = p->Hp * p->Wp; hp.Wp = p->Wp; hp.P = d.P; hp.Q = d.Q; hp.K = d.K;
         hp.S = d.S; hp.taps = d.R * d.S; hp.cchunks = p->Cp / BKC; hp.lead = p->lead;
@@ -811,6 +812,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         int rc = encode_map_a(p, xp);
         if (rc != BODA_OK) return rc;
     }
+    if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
     IgemmParams prm;
     prm.M = d.M; prm.K = d.K; prm.PQ = d.P * d.Q; prm.Q = d.Q; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
     prm.cchunks = p->Cp / BKC;

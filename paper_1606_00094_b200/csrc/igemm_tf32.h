@@ -23,8 +23,9 @@ size_t igemm_plan_workspace_bytes(const IgemmPlan* p);
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n);
 int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream);
 void igemm_unbind_filters(IgemmPlan* p);
+// after_staging (may be null): event recorded on the stream between the operand-staging kernels and the main kernel
 int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
-                 cudaStream_t stream);
+                 cudaStream_t stream, cudaEvent_t after_staging = nullptr);
 
 // Scratch-in-a-caller-region form (allocates nothing): bytes needed at least, and the run itself.
 size_t igemm_region_min_bytes(const ConvDims& d);

@@ -1,0 +1,253 @@
+// boda_stack: a chain of convolution and max-pool layers (layer i+1 reads layer i's output) run as one unit.
+// The stack owns the plans, the activations between layers, one workspace shared by all layers and a CUDA graph
+// of the whole chain, so that a forward pass is a single graph launch with no host work between kernels.
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "boda_internal.h"
+
+using namespace boda;
+
+struct boda_stack {
+    struct Op {
+        int kind = 0;                       // 0 conv, 1 max-pool
+        boda_conv_shape conv{};
+        int ksz = 0, stride = 0;
+        boda_conv_plan* plan = nullptr;
+        const float* filt = nullptr;
+        const float* bias = nullptr;
+        int N = 0, C = 0, H = 0, W = 0;     // input dims of this op
+        int oC = 0, oH = 0, oW = 0;         // output dims
+        float* out = nullptr;               // owned activation (nullptr for the last op: the caller's buffer)
+        size_t out_elems = 0;
+    };
+    std::vector<Op> ops;
+    int device = 0;
+    void* workspace = nullptr;
+    size_t ws_bytes = 0;
+    float* staging_in = nullptr;            // device copy of a host input
+    float* staging_out = nullptr;
+    size_t in_elems = 0, out_elems = 0;
+    cudaGraphExec_t graph_exec = nullptr;
+    const float* graph_in = nullptr;
+    float* graph_out = nullptr;
+    cudaStream_t capture_stream = nullptr;
+};
+
+namespace {
+
+int run_ops(boda_stack* s, const float* in, float* out, cudaStream_t stream, cudaEvent_t* events)
+{
+    const float* cur = in;
+    const int n = (int)s->ops.size();
+    for (int i = 0; i < n; ++i) {
+        boda_stack::Op& op = s->ops[i];
+        float* dst = (i == n - 1) ? out : op.out;
+        if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 0], stream));
+        int rc;
+        if (op.kind == 0) {
+            if (!op.filt) return BODA_ERR_INVALID_ARG;
+            rc = conv_fwd_planned_ex(op.plan, cur, op.filt, op.bias, dst, s->workspace, stream, events ? events[3 * i + 1] : nullptr);
+        } else {
+            if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 1], stream));
+            rc = maxpool_launch(cur, dst, op.N, op.C, op.H, op.W, op.ksz, op.stride, stream);
+        }
+        if (rc != BODA_OK) return rc;
+        if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 2], stream));
+        cur = dst;
+    }
+    return BODA_OK;
+}
+
+void drop_graph(boda_stack* s)
+{
+    if (s->graph_exec) { cudaGraphExecDestroy(s->graph_exec); s->graph_exec = nullptr; }
+    s->graph_in = nullptr;
+    s->graph_out = nullptr;
+}
+
+int build_graph(boda_stack* s, const float* in, float* out, cudaStream_t user_stream)
+{
+    drop_graph(s);
+    if (!s->capture_stream) BODA_CUDA_TRY(cudaStreamCreateWithFlags(&s->capture_stream, cudaStreamNonBlocking));
+    // one eager pass first, on the caller's stream: per-shape set-up (kernel attributes, tensor maps) must not
+    // happen inside a capture
+    int rc = run_ops(s, in, out, user_stream, nullptr);
+    if (rc != BODA_OK) return rc;
+    BODA_CUDA_TRY(cudaStreamBeginCapture(s->capture_stream, cudaStreamCaptureModeThreadLocal));
+    rc = run_ops(s, in, out, s->capture_stream, nullptr);
+    cudaGraph_t graph = nullptr;
+    cudaError_t e = cudaStreamEndCapture(s->capture_stream, &graph);
+    if (rc != BODA_OK) { if (graph) cudaGraphDestroy(graph); return rc; }
+    if (e != cudaSuccess) return record_cuda_error(e, "cudaStreamEndCapture");
+    e = cudaGraphInstantiate(&s->graph_exec, graph, 0);
+    cudaGraphDestroy(graph);
+    if (e != cudaSuccess) { s->graph_exec = nullptr; return record_cuda_error(e, "cudaGraphInstantiate"); }
+    s->graph_in = in;
+    s->graph_out = out;
+    return BODA_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int boda_stack_destroy(boda_stack* s)
+{
+    if (!s) return BODA_OK;
+    int prev = 0;
+    (void)cudaGetDevice(&prev);
+    (void)cudaSetDevice(s->device);
+    drop_graph(s);
+    if (s->capture_stream) cudaStreamDestroy(s->capture_stream);
+    for (auto& op : s->ops) {
+        if (op.plan) boda_conv_plan_destroy(op.plan);
+        if (op.out) cudaFree(op.out);
+    }
+    if (s->workspace) cudaFree(s->workspace);
+    if (s->staging_in) cudaFree(s->staging_in);
+    if (s->staging_out) cudaFree(s->staging_out);
+    (void)cudaSetDevice(prev);
+    delete s;
+    return BODA_OK;
+}
+
+int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts* opts, boda_stack** out)
+{
+    if (!ops || n_ops <= 0 || !out) return BODA_ERR_INVALID_ARG;
+    *out = nullptr;
+    if (ops[0].kind != BODA_STACK_CONV) return BODA_ERR_INVALID_ARG;     // the first op fixes the input dims
+    boda_stack* s = new (std::nothrow) boda_stack();
+    if (!s) return BODA_ERR_NOMEM;
+    int device = opts ? opts->device : -1;
+    if (device < 0) { cudaError_t e = cudaGetDevice(&device); if (e != cudaSuccess) { delete s; return record_cuda_error(e, "cudaGetDevice"); } }
+    s->device = device;
+    int N = ops[0].conv.N, C = ops[0].conv.C, H = ops[0].conv.H, W = ops[0].conv.W;
+    s->in_elems = (size_t)N * C * H * W;
+    int rc = BODA_OK;
+    for (int i = 0; i < n_ops && rc == BODA_OK; ++i) {
+        boda_stack::Op op;
+        op.kind = ops[i].kind;
+        op.N = N; op.C = C; op.H = H; op.W = W;
+        if (op.kind == BODA_STACK_CONV) {
+            op.conv = ops[i].conv;
+            if (op.conv.N != N || op.conv.C != C || op.conv.H != H || op.conv.W != W) { rc = BODA_ERR_INVALID_ARG; break; }
+            rc = boda_conv_plan_create(&op.conv, opts, &op.plan);
+            if (rc != BODA_OK) break;
+            int oN, oK, oP, oQ;
+            conv_plan_out_dims(op.plan, &oN, &oK, &oP, &oQ);
+            op.oC = oK; op.oH = oP; op.oW = oQ;
+            const size_t ws = boda_conv_plan_workspace_bytes(op.plan);
+            if (ws > s->ws_bytes) s->ws_bytes = ws;
+        } else if (op.kind == BODA_STACK_MAXPOOL) {
+            op.ksz = ops[i].ksz; op.stride = ops[i].stride;
+            op.oC = C;
+            op.oH = boda_conv_out_dim(H, op.ksz, op.stride, 0);
+            op.oW = boda_conv_out_dim(W, op.ksz, op.stride, 0);
+            if (op.oH <= 0 || op.oW <= 0) { rc = BODA_ERR_INVALID_ARG; break; }
+        } else { rc = BODA_ERR_INVALID_ARG; break; }
+        op.out_elems = (size_t)N * op.oC * op.oH * op.oW;
+        if (i < n_ops - 1) {
+            cudaError_t e = cudaMalloc(&op.out, op.out_elems * sizeof(float));
+            if (e != cudaSuccess) { if (op.plan) boda_conv_plan_destroy(op.plan); rc = record_cuda_error(e, "activation allocation"); break; }
+        }
+        s->ops.push_back(op);
+        C = op.oC; H = op.oH; W = op.oW;
+    }
+    if (rc == BODA_OK) {
+        s->out_elems = s->ops.back().out_elems;
+        if (s->ws_bytes) {
+            cudaError_t e = cudaMalloc(&s->workspace, s->ws_bytes);
+            if (e != cudaSuccess) rc = record_cuda_error(e, "workspace allocation");
+        }
+    }
+    if (rc != BODA_OK) { boda_stack_destroy(s); return rc; }
+    *out = s;
+    return BODA_OK;
+}
+
+int boda_stack_num_ops(const boda_stack* s) { return s ? (int)s->ops.size() : 0; }
+
+int boda_stack_set_filters(boda_stack* s, int op_index, const float* filt, const float* bias, void* stream)
+{
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size() || !filt) return BODA_ERR_INVALID_ARG;
+    boda_stack::Op& op = s->ops[op_index];
+    if (op.kind != BODA_STACK_CONV) return BODA_ERR_INVALID_ARG;
+    const int rc = boda_conv_plan_bind_filters(op.plan, filt, stream);
+    if (rc != BODA_OK) return rc;
+    op.filt = filt;
+    op.bias = bias;
+    drop_graph(s);                       // the graph holds the old pointers
+    return BODA_OK;
+}
+
+int boda_stack_out_dims(const boda_stack* s, int op_index, int* N, int* C, int* H, int* W)
+{
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size() || !N || !C || !H || !W) return BODA_ERR_INVALID_ARG;
+    const boda_stack::Op& op = s->ops[op_index];
+    *N = op.N; *C = op.oC; *H = op.oH; *W = op.oW;
+    return BODA_OK;
+}
+
+int boda_stack_layer_output(const boda_stack* s, int op_index, const float** ptr)
+{
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size() - 1 || !ptr) return BODA_ERR_INVALID_ARG;
+    *ptr = s->ops[op_index].out;
+    return BODA_OK;
+}
+
+int boda_stack_describe(const boda_stack* s, int op_index, char* buf, size_t n)
+{
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size() || !buf || n == 0) return BODA_ERR_INVALID_ARG;
+    const boda_stack::Op& op = s->ops[op_index];
+    if (op.kind == BODA_STACK_CONV) return boda_conv_plan_describe(op.plan, buf, n);
+    std::snprintf(buf, n, "maxpool %dx%d stride %d", op.ksz, op.ksz, op.stride);
+    return BODA_OK;
+}
+
+int boda_stack_kernels_per_fwd(const boda_stack* s);
+
+int boda_stack_fwd(boda_stack* s, const float* in, float* out, void* stream)
+{
+    if (!s || !in || !out) return BODA_ERR_INVALID_ARG;
+    if (!s->graph_exec || s->graph_in != in || s->graph_out != out) {
+        const int rc = build_graph(s, in, out, (cudaStream_t)stream);
+        if (rc != BODA_OK) return rc;
+    }
+    BODA_CUDA_TRY(cudaGraphLaunch(s->graph_exec, (cudaStream_t)stream));
+    count_launch(boda_stack_kernels_per_fwd(s));
+    return BODA_OK;
+}
+
+int boda_stack_fwd_eager(boda_stack* s, const float* in, float* out, void* stream, void** events)
+{
+    if (!s || !in || !out) return BODA_ERR_INVALID_ARG;
+    return run_ops(s, in, out, (cudaStream_t)stream, (cudaEvent_t*)events);
+}
+
+int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, void* stream)
+{
+    if (!s || !in_host || !out_host) return BODA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (!s->staging_in) BODA_CUDA_TRY(cudaMalloc(&s->staging_in, s->in_elems * sizeof(float)));
+    if (!s->staging_out) BODA_CUDA_TRY(cudaMalloc(&s->staging_out, s->out_elems * sizeof(float)));
+    BODA_CUDA_TRY(cudaMemcpyAsync(s->staging_in, in_host, s->in_elems * sizeof(float), cudaMemcpyHostToDevice, st));
+    const int rc = boda_stack_fwd(s, s->staging_in, s->staging_out, stream);
+    if (rc != BODA_OK) return rc;
+    BODA_CUDA_TRY(cudaMemcpyAsync(out_host, s->staging_out, s->out_elems * sizeof(float), cudaMemcpyDeviceToHost, st));
+    BODA_CUDA_TRY(cudaStreamSynchronize(st));
+    return BODA_OK;
+}
+
+int boda_stack_kernels_per_fwd(const boda_stack* s)
+{
+    if (!s) return 0;
+    int n = 0;
+    for (const auto& op : s->ops) n += op.kind == BODA_STACK_CONV ? boda_conv_plan_kernels_per_call(op.plan) : 1;
+    return n;
+}
+
+}  // extern "C"

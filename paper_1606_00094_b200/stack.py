@@ -1,7 +1,7 @@
-"""A chain of convolution and pooling layers driven through the C ABI (layer i+1 eats layer i's output).
+"""Python face of ``boda_stack``: a chain of convolution and pooling layers run as one CUDA graph.
 
-Host-side orchestration only: it creates one plan per convolution, keeps the activations in device
-tensors and issues the library calls in order on one stream.  No arithmetic happens here.
+Marshalling only: the chain, its plans, activations, workspace and graph live in the library
+(``csrc/stack.cu``); this class keeps the filter tensors alive and hands out torch views.
 """
 from __future__ import annotations
 
@@ -18,70 +18,97 @@ class ConvStack:
                  tune: int = 0, device: str = "cuda"):
         """ops: conv / pool descriptors; params: per conv layer (filters, bias) as numpy fp32 arrays."""
         self.ops = list(ops)
-        self.device = device
-        self.plans: List[Optional[B.ConvPlan]] = []
+        c_ops = []
+        for op in self.ops:
+            o = B.boda_stack_op()
+            if op.kind == "conv":
+                o.kind = B.BODA_STACK_CONV
+                o.conv = B.boda_conv_shape(*op.shape.as_tuple())
+            else:
+                o.kind = B.BODA_STACK_MAXPOOL
+                o.ksz, o.stride = op.ksz, op.stride
+            c_ops.append(o)
+        opts = B.boda_plan_opts_default()
+        opts.math, opts.tune = math, tune
+        self.handle = B.boda_stack_create(c_ops, opts)
         self.filters: List[Optional[torch.Tensor]] = []
         self.biases: List[Optional[torch.Tensor]] = []
-        self.outputs: List[torch.Tensor] = []
         it = iter(params)
-        shape_nchw = None
-        ws_bytes = 0
-        for op in self.ops:
+        for i, op in enumerate(self.ops):
             if op.kind == "conv":
-                s = op.shape
                 w, b = next(it)
-                plan = B.ConvPlan(s.as_tuple(), math=math, tune=tune)
                 fw = torch.from_numpy(w).to(device)
-                plan.bind_filters(fw)
-                self.plans.append(plan)
+                fb = torch.from_numpy(b).to(device) if b is not None else None
+                B.boda_stack_set_filters(self.handle, i, fw, fb)
                 self.filters.append(fw)
-                self.biases.append(torch.from_numpy(b).to(device) if b is not None else None)
-                shape_nchw = plan.out_shape
-                if shape_nchw is None:
-                    raise ValueError("bad conv shape")
+                self.biases.append(fb)
             else:
-                N, C, H, W = shape_nchw
-                shape_nchw = (N, C, B.boda_conv_out_dim(H, op.ksz, op.stride, 0), B.boda_conv_out_dim(W, op.ksz, op.stride, 0))
-                self.plans.append(None)
                 self.filters.append(None)
                 self.biases.append(None)
-            self.outputs.append(torch.empty(shape_nchw, dtype=torch.float32, device=device))
         first = self.ops[0].shape
         self.in_shape = (first.N, first.C, first.H, first.W)
-        self.out_shape = tuple(self.outputs[-1].shape)
-        self.staging_in = torch.empty(self.in_shape, dtype=torch.float32, device=device)
+        self.out_shape = B.boda_stack_out_dims(self.handle, len(self.ops) - 1)
+        self.out = torch.empty(self.out_shape, dtype=torch.float32, device=device)
         torch.cuda.synchronize()
 
     def describe(self) -> List[str]:
-        return [p.describe() if p is not None else "maxpool" for p in self.plans]
+        return [B.boda_stack_describe(self.handle, i) for i in range(len(self.ops))]
 
-    def forward(self, x: torch.Tensor, events=None) -> torch.Tensor:
-        """Runs every layer on the current stream.  events: optional list of (start, end) CUDA event pairs,
-        one per op, recorded around that op's launches."""
-        cur = x
-        for i, op in enumerate(self.ops):
-            if events is not None:
-                events[i][0].record()
-            out = self.outputs[i]
-            if op.kind == "conv":
-                B.boda_conv_fwd_planned(self.plans[i].handle, cur, self.filters[i], self.biases[i], out,
-                                        self.plans[i].workspace)
-            else:
-                N, C, H, W = cur.shape
-                B.boda_maxpool_fwd(cur, out, N, C, H, W, op.ksz, op.stride)
-            if events is not None:
-                events[i][1].record()
-            cur = out
-        return cur
+    def kernels_per_forward(self) -> int:
+        return B.boda_stack_kernels_per_fwd(self.handle)
+
+    def forward(self, x: torch.Tensor, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """One graph launch on the current stream (the graph is captured on the first call)."""
+        out = self.out if out is None else out
+        B.boda_stack_fwd(self.handle, x, out)
+        return out
+
+    def forward_eager(self, x: torch.Tensor, events=None, out: Optional[torch.Tensor] = None) -> torch.Tensor:
+        """Kernel-by-kernel launches; events = flat list of 3 * n_ops CUDA events for per-layer timing."""
+        out = self.out if out is None else out
+        B.boda_stack_fwd_eager(self.handle, x, out, None, events)
+        return out
 
     def forward_host(self, x_host: torch.Tensor, out_host: torch.Tensor) -> None:
         """Host buffers in and out (pinned for asynchronous copies); returns after the result has landed."""
-        self.staging_in.copy_(x_host, non_blocking=True)
-        y = self.forward(self.staging_in)
-        out_host.copy_(y, non_blocking=True)
-        torch.cuda.current_stream().synchronize()
+        B.boda_stack_fwd_host(self.handle, x_host, out_host)
+
+    def layer_output(self, i: int) -> torch.Tensor:
+        """Copy of the activation op i wrote during the last forward pass."""
+        if i == len(self.ops) - 1:
+            return self.out.clone()
+        shape = B.boda_stack_out_dims(self.handle, i)
+        n = shape[0] * shape[1] * shape[2] * shape[3]
+        ptr = B.boda_stack_layer_output(self.handle, i)
+        dst = torch.empty(shape, dtype=torch.float32, device=self.out.device)
+        # device-to-device copy of the library-owned buffer into a torch tensor
+        _copy_d2d(dst.data_ptr(), ptr, n * 4)
+        return dst
 
     def close(self) -> None:
-        for p in self.plans:
-            if p is not None:
-                p.close()
+        if self.handle:
+            B.boda_stack_destroy(self.handle)
+            self.handle = None
+
+    def __del__(self):
+        try:
+            self.close()
+        except Exception:
+            pass
+
+
+def _copy_d2d(dst_ptr: int, src_ptr: int, nbytes: int) -> None:
+    """Device-to-device copy through torch's view of raw memory (plumbing only)."""
+    torch.cuda.synchronize()
+    src = _as_tensor(src_ptr, nbytes)
+    dst = _as_tensor(dst_ptr, nbytes)
+    dst.copy_(src)
+    torch.cuda.synchronize()
+
+
+def _as_tensor(ptr: int, nbytes: int) -> torch.Tensor:
+    class _Holder:
+        pass
+    h = _Holder()
+    h.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (ptr, False), "version": 2}
+    return torch.as_tensor(h, device="cuda")

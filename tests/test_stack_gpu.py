@@ -1,0 +1,77 @@
+"""The AlexNet-shaped conv stack end to end on the GPU against the fp64 oracle chain."""
+import numpy as np
+import pytest
+
+from oracle import conv_oracle as orc
+from paper_1606_00094_b200 import workloads as wl
+from helpers import FP32_TOL, TF32_TOL
+
+pytestmark = pytest.mark.gpu
+
+
+def _oracle_chain(x, params, ops):
+    """fp64 end to end: layer i feeds layer i+1 without ever being rounded to fp32."""
+    outs = []
+    a = x.astype(np.float64)
+    it = iter(params)
+    for op in ops:
+        if op.kind == "conv":
+            w, b = next(it)
+            s = op.shape
+            a = orc.conv_fwd(a, w, b, stride=s.stride, pad=s.pad, relu=True)
+        else:
+            a = orc.maxpool_fwd(a, op.ksz, op.stride)
+        outs.append(a)
+    return outs
+
+
+@pytest.mark.parametrize("batch,math,tol", [(2, 0, TF32_TOL), (1, 1, FP32_TOL), (20, 0, TF32_TOL)])
+def test_stack_every_layer_matches_fp64_chain(batch, math, tol):
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    from paper_1606_00094_b200.stack import ConvStack
+    ops = wl.alexnet_stack(batch)
+    x, params = wl.stack_tensors(batch)
+    ref = _oracle_chain(x, params, ops)
+    stack = ConvStack(ops, params, math=math)
+    try:
+        dx = torch.from_numpy(x).cuda()
+        out_graph = stack.forward(dx).clone()            # first call: eager pass + graph capture + launch
+        out_graph2 = stack.forward(dx).clone()           # pure graph replay
+        torch.cuda.synchronize()
+        assert B.boda_query_status() == 0
+        assert torch.equal(out_graph, out_graph2)
+        descs = stack.describe()
+        for i, r in enumerate(ref):
+            got = stack.layer_output(i).cpu().numpy()
+            assert got.shape == r.shape
+            err = orc.rel_l2(got, r)
+            assert err <= tol, f"op {i} ({descs[i]}): rel-L2 {err:.3e} > {tol:.0e}"
+        # host-buffer entry point and the eager path give the same numbers
+        hx = torch.from_numpy(x).pin_memory()
+        ho = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+        stack.forward_host(hx, ho)
+        assert torch.equal(ho, out_graph.cpu())
+        eager = stack.forward_eager(dx).clone()
+        torch.cuda.synchronize()
+        assert torch.equal(eager, out_graph)
+        if math == 0:
+            assert any("tconv" in d for d in descs)
+        else:
+            assert all("direct" in d or "maxpool" in d for d in descs)
+        assert stack.kernels_per_forward() >= len(ops)
+    finally:
+        stack.close()
+
+
+def test_stack_rejects_shapes_that_do_not_chain():
+    from paper_1606_00094_b200 import binding as B
+    a = B.boda_stack_op()
+    a.kind = B.BODA_STACK_CONV
+    a.conv = B.boda_conv_shape(1, 3, 16, 16, 8, 3, 3, 1, 1, 1)
+    b = B.boda_stack_op()
+    b.kind = B.BODA_STACK_CONV
+    b.conv = B.boda_conv_shape(1, 4, 16, 16, 8, 3, 3, 1, 1, 1)      # expects 4 channels, gets 8
+    with pytest.raises(B.BodaError) as e:
+        B.boda_stack_create([a, b])
+    assert e.value.status == B.BODA_ERR_INVALID_ARG
