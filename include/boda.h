@@ -92,7 +92,8 @@ void boda_plan_opts_default(boda_plan_opts* opts);
  * "operation -> variant -> blocking constants" (Section 4, Figure "codegen", and the variant rules
  * of Section 5: k1conv for kernel size 1, tconv for kernel sizes 2..11, conv otherwise).  With
  * opts->tune != 0 the legal candidates are timed on scratch buffers and the fastest is kept (the
- * automated tuning the paper names as future work); this synchronises the device.
+ * automated tuning the paper names as future work); this synchronises the device.  If the environment variable
+ * BODA_TUNE_CACHE names a file, tuned choices are read from and appended to it (one text line per shape).
  * `opts` may be NULL (defaults).  On success *plan owns device memory (index tables, packed filter
  * storage, workspace); destroy it with boda_conv_plan_destroy.
  * Errors: INVALID_ARG (bad shape), UNSUPPORTED (forced variant illegal, device not sm_100), CUDA, NOMEM.

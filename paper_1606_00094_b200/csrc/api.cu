@@ -1,6 +1,7 @@
 // C ABI: plans (variant selection + blocking), the forward entry points, caches and status.
 #include <atomic>
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <map>
 #include <mutex>
@@ -15,6 +16,12 @@ namespace boda {
 
 static thread_local std::string t_last_error;
 static std::atomic<unsigned long long> g_launches{0};
+
+bool pdl_enabled()
+{
+    static const bool on = []() { const char* e = std::getenv("BODA_NO_PDL"); return !(e && *e && *e != '0'); }();
+    return on;
+}
 
 void count_launch(int n) { g_launches.fetch_add((unsigned long long)n, std::memory_order_relaxed); }
 unsigned long long launch_count() { return g_launches.load(std::memory_order_relaxed); }
@@ -71,6 +78,32 @@ int get_ctx(int device, DeviceCtx** out)
     }
     *out = &it->second;
     return BODA_OK;
+}
+
+// ---- autotune cache: a text file "key tile split" per line, named by the environment variable BODA_TUNE_CACHE
+bool tune_cache_lookup(const char* key, int* tile, int* split)
+{
+    const char* path = std::getenv("BODA_TUNE_CACHE");
+    if (!path || !*path) return false;
+    FILE* f = std::fopen(path, "r");
+    if (!f) return false;
+    char k[200];
+    int t = 0, sp = 0;
+    bool hit = false;
+    while (std::fscanf(f, "%199s %d %d", k, &t, &sp) == 3)
+        if (std::strcmp(k, key) == 0) { *tile = t; *split = sp; hit = true; }
+    std::fclose(f);
+    return hit;
+}
+
+void tune_cache_store(const char* key, int tile, int split)
+{
+    const char* path = std::getenv("BODA_TUNE_CACHE");
+    if (!path || !*path) return;
+    FILE* f = std::fopen(path, "a");
+    if (!f) return;
+    std::fprintf(f, "%s %d %d\n", key, tile, split);
+    std::fclose(f);
 }
 
 bool shape_ok(const boda_conv_shape& s)
@@ -238,7 +271,16 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
     if (!o.tune || o.tile_id >= 0) {
         rc = plan_build(*shape, o, ctx, variant, o.tile_id, o.split_k, plan);
     } else {
-        // Automated tuning: time every tile (and split) of the chosen variant, keep the fastest.
+        // Automated tuning: time every tile (and split) of the chosen variant, keep the fastest.  Winners are
+        // remembered in the file named by BODA_TUNE_CACHE (if set), one line per (shape, variant).
+        char key[160];
+        std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,m%d", shape->N, shape->C, shape->H, shape->W,
+                      shape->K, shape->R, shape->S, shape->stride, shape->pad, variant, o.s2d, o.split_k);
+        int c_tile = -1, c_split = 0;
+        if (tune_cache_lookup(key, &c_tile, &c_split)) {
+            rc = plan_build(*shape, o, ctx, variant, c_tile, c_split, plan);
+            if (rc == BODA_OK) { (void)cudaSetDevice(prev); return rc; }
+        }
         boda_conv_plan* best = nullptr;
         float best_ms = 1e30f;
         const int ntiles = variant == BODA_VARIANT_DIRECT ? direct_num_tiles() : igemm_num_tiles();
@@ -259,7 +301,11 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
                 }
             }
         }
-        if (best) { *plan = best; rc = BODA_OK; }
+        if (best) {
+            *plan = best;
+            rc = BODA_OK;
+            tune_cache_store(key, best->tile_id, best->ig ? igemm_plan_splits(best->ig) : 0);
+        }
         else rc = plan_build(*shape, o, ctx, variant, -1, o.split_k, plan);
     }
     (void)cudaSetDevice(prev);

@@ -43,6 +43,45 @@ int record_cuda_error(cudaError_t e, const char* what);
         if (_e != cudaSuccess) return ::boda::record_cuda_error(_e, #expr);  \
     } while (0)
 
+// ---- kernel launch helper
+// Every kernel of the library is launched with programmatic dependent launch: it calls pdl_launch_dependents()
+// at once and pdl_wait() before it first touches global memory that an earlier kernel on the stream may have
+// written (or may still read), so its prologue overlaps the previous kernel's tail.  cluster_z > 1 groups the
+// CTAs along grid.z into a thread-block cluster.  BODA_NO_PDL=1 in the environment turns the overlap off.
+bool pdl_enabled();
+
+template <typename Kernel, typename... Args>
+cudaError_t launch_kernel(Kernel kernel, dim3 grid, dim3 block, size_t smem, cudaStream_t stream, int cluster_z, Args... args)
+{
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = stream;
+    cudaLaunchAttribute attr[2];
+    unsigned n = 0;
+    if (cluster_z > 1) {
+        attr[n].id = cudaLaunchAttributeClusterDimension;
+        attr[n].val.clusterDim.x = 1;
+        attr[n].val.clusterDim.y = 1;
+        attr[n].val.clusterDim.z = (unsigned)cluster_z;
+        ++n;
+    }
+    if (pdl_enabled()) {
+        attr[n].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+        attr[n].val.programmaticStreamSerializationAllowed = 1;
+        ++n;
+    }
+    cfg.attrs = attr;
+    cfg.numAttrs = n;
+    return cudaLaunchKernelEx(&cfg, kernel, args...);
+}
+
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+#endif
+
 // ---- DIRECT (FP32 CUDA-core) variant -----------------------------------------------------------
 // Reduction-index table entry: for flattened reduction index j = (c*R + r)*S + s the element offset
 // c*H*W + r*W + s inside one image and the tap (r, s); entries past C*R*S have r = 0x4000 so that

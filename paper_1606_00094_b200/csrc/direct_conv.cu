@@ -32,6 +32,8 @@ direct_conv_kernel(const ConvDims d, const float* __restrict__ in, const float* 
     __shared__ __align__(16) float As[2][BK][BM];
     __shared__ __align__(16) float Bs[2][BK][BNP];
 
+    pdl_launch_dependents();
+    pdl_wait();
     const int tid = threadIdx.x;
     const int tx = tid & 15;                          // pixel group
     const int ty = tid >> 4;                          // channel group
@@ -192,9 +194,8 @@ int launch_tile(const ConvDims& d, const float* in, const float* filt, const flo
 {
     constexpr int BM = 16 * TM, BN = 16 * TN;
     dim3 grid((d.M + BM - 1) / BM, (d.K + BN - 1) / BN);
-    direct_conv_kernel<TM, TN><<<grid, kThreads, 0, stream>>>(d, in, filt, bias, out, tab);
+    BODA_CUDA_TRY(launch_kernel(direct_conv_kernel<TM, TN>, grid, dim3(kThreads), 0, stream, 1, d, in, filt, bias, out, tab));
     count_launch();
-    BODA_CUDA_TRY(cudaGetLastError());
     return BODA_OK;
 }
 

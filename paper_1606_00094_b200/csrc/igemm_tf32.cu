@@ -87,6 +87,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
     const int my_iters = it_end - it_begin;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -103,6 +104,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_acc = s_tmem_base;
+    pdl_wait();          // everything above overlapped the previous kernel; its results are needed from here on
 
     if (warp == 0) {
         if (lane == 0) {
@@ -253,6 +255,8 @@ __global__ void __launch_bounds__(256)
 pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int C, int Cp, int HW)
 {
     __shared__ float tile[32][33];
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = blockIdx.z;
     const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8
@@ -275,6 +279,8 @@ pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int
 __global__ void __launch_bounds__(256)
 pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int Cp, int RS)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long total = (long long)RS * K * Cp;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
@@ -297,33 +303,48 @@ __global__ void __launch_bounds__(256)
 pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int C, int H, int W, int t, int pad,
                       int Hb, int Wb, int Cp)
 {
-    extern __shared__ float sm_rows[];            // [C][t][W]
+    extern __shared__ float sm_rows[];            // [C*t rows][W], then two int tables [Cp]
+    int* sm_src = reinterpret_cast<int*>(sm_rows + C * t * W);
+    int* sm_dx = sm_src + Cp;
+    pdl_launch_dependents();
     const int yb = blockIdx.x, n = blockIdx.y;
-    const int tW = t * W;
-    for (int idx = threadIdx.x; idx < C * tW; idx += blockDim.x) {
-        const int c = idx / tW;
-        const int rem = idx - c * tW;
-        const int dy = rem / W;
-        const int x = rem - dy * W;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    // tables: packed channel cp = (dy*t + dx)*C + c  ->  start of staged row (c, dy) in sm_rows, and dx - pad
+    const int Cs = C * t * t;
+    for (int cp = threadIdx.x; cp < Cp; cp += blockDim.x) {
+        int v = -1, dxp = 0;
+        if (cp < Cs) {
+            const int g = cp / C, c = cp - g * C;
+            const int dy = g / t, dx = g - dy * t;
+            v = (c * t + dy) * W;
+            dxp = dx - pad;
+        }
+        sm_src[cp] = v;
+        sm_dx[cp] = dxp;
+    }
+    pdl_wait();
+    // stage the t input rows of every channel: one warp per (c, dy) row, lanes along x (coalesced)
+    for (int row = warp; row < C * t; row += nwarps) {
+        const int c = row / t, dy = row - c * t;
         const int y = yb * t + dy - pad;
-        sm_rows[idx] = (y >= 0 && y < H) ? __ldg(in + (((size_t)n * C + c) * H + y) * W + x) : 0.f;
+        const bool inside = y >= 0 && y < H;
+        const float* src = in + (((size_t)n * C + c) * H + (inside ? y : 0)) * W;
+        for (int x = lane; x < W; x += 32) sm_rows[row * W + x] = inside ? __ldg(src + x) : 0.f;
     }
     __syncthreads();
+    // write the row of blocks: one warp per block xb, lanes along the packed channels (contiguous 128-byte stores)
     float* dst = xs + ((size_t)n * Hb + yb) * Wb * Cp;
-    const int Cs = C * t * t;
-    for (int o = threadIdx.x; o < Wb * Cp; o += blockDim.x) {
-        const int xb = o / Cp;
-        const int cp = o - xb * Cp;
-        float v = 0.f;
-        if (cp < Cs) {
-            const int g = cp / C;
-            const int c = cp - g * C;
-            const int dy = g / t;
-            const int dx = g - dy * t;
-            const int x = xb * t + dx - pad;
-            if (x >= 0 && x < W) v = sm_rows[(c * t + dy) * W + x];
+    for (int xb = warp; xb < Wb; xb += nwarps) {
+        const int xoff = xb * t;
+        for (int cp = lane; cp < Cp; cp += 32) {
+            const int rowbase = sm_src[cp];
+            float v = 0.f;
+            if (rowbase >= 0) {
+                const int x = xoff + sm_dx[cp];                  // column in the input image
+                if (x >= 0 && x < W) v = sm_rows[rowbase + x];
+            }
+            dst[(size_t)xb * Cp + cp] = round_tf32(v);
         }
-        dst[o] = round_tf32(v);
     }
 }
 
@@ -332,6 +353,8 @@ __global__ void __launch_bounds__(256)
 pack_filters_s2d_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int R, int S, int t,
                         int Rb, int Sb, int Cp)
 {
+    pdl_launch_dependents();
+    pdl_wait();
     const long long total = (long long)Rb * Sb * K * Cp;
     const int Cs = C * t * t;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
@@ -522,25 +545,6 @@ double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
     return waves * (ips * per_iter + 5000.0 + nacc * epilogue_cost(BN, splits));
 }
 
-// Launch with the CTAs of one output tile (grid.z = reduction splits) grouped into a thread-block cluster.
-template <typename Kernel, typename... Args>
-cudaError_t launch_clustered(Kernel kernel, dim3 grid, int threads, int smem, cudaStream_t stream, int cluster_z, Args... args)
-{
-    cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = grid;
-    cfg.blockDim = dim3(threads);
-    cfg.dynamicSmemBytes = (size_t)smem;
-    cfg.stream = stream;
-    cudaLaunchAttribute attr[1];
-    attr[0].id = cudaLaunchAttributeClusterDimension;
-    attr[0].val.clusterDim.x = 1;
-    attr[0].val.clusterDim.y = 1;
-    attr[0].val.clusterDim.z = (unsigned)cluster_z;
-    cfg.attrs = attr;
-    cfg.numAttrs = cluster_z > 1 ? 1 : 0;
-    return cudaLaunchKernelEx(&cfg, kernel, args...);
-}
-
 template <int BN, int NACC>
 int launch_halo(IgemmPlan* p, const halo::HaloParams& prm, cudaStream_t stream)
 {
@@ -551,8 +555,8 @@ int launch_halo(IgemmPlan* p, const halo::HaloParams& prm, cudaStream_t stream)
         attr_smem = smem;
     }
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    BODA_CUDA_TRY(launch_clustered(halo::tconv_halo_kernel<BN, NACC>, grid, halo::kThreads, smem, stream, p->splits,
-                                   p->map_a, p->map_b, prm));
+    BODA_CUDA_TRY(launch_kernel(halo::tconv_halo_kernel<BN, NACC>, grid, dim3(halo::kThreads), (size_t)smem, stream, p->splits,
+                                p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
 }
@@ -586,8 +590,8 @@ int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
         attr_set = true;
     }
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    BODA_CUDA_TRY(launch_clustered(igemm_tf32_kernel<BN>, grid, kIgemmThreads, Cfg::SMEM_BYTES, stream, p->splits,
-                                   p->map_a, p->map_b, prm));
+    BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
+                                p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
 }
@@ -709,6 +713,7 @@ void igemm_plan_destroy(IgemmPlan* p)
 }
 
 int igemm_plan_tile(const IgemmPlan* p) { return p->tile_id; }
+int igemm_plan_splits(const IgemmPlan* p) { return p->splits; }
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->partial_bytes; }
 
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
@@ -732,10 +737,12 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
     if (p->s2d) {
         const ConvDims& o = p->orig;
-        pack_filters_s2d_kernel<<<blocks, 256, 0, stream>>>(filt, p->d_wp, o.K, o.C, o.R, o.S, o.stride, d.R, d.S, p->Cp);
-    } else
-    pack_filters_kernel<<<blocks, 256, 0, stream>>>(filt, p->d_wp, d.K, d.C, p->Cp, d.R * d.S);
-    BODA_CUDA_TRY(cudaGetLastError());
+        BODA_CUDA_TRY(launch_kernel(pack_filters_s2d_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, o.K, o.C, o.R,
+                                    o.S, o.stride, d.R, d.S, p->Cp));
+    } else {
+        BODA_CUDA_TRY(launch_kernel(pack_filters_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.C, p->Cp,
+                                    d.R * d.S));
+    }
     count_launch();
     return BODA_OK;
 }
@@ -765,16 +772,16 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         // both kernels read the same [N][H'][W'][Cp] layout here (the view has no padding)
         const ConvDims& o = p->orig;
         dim3 grid(d.H, d.N);
-        const size_t smem = (size_t)o.C * o.stride * o.W * 4;
-        pack_input_s2d_kernel<<<grid, 256, smem, stream>>>(in, xp, o.C, o.H, o.W, o.stride, o.pad, d.H, d.W, p->Cp);
-        BODA_CUDA_TRY(cudaGetLastError());
+        const size_t smem = (size_t)o.C * o.stride * o.W * 4 + (size_t)p->Cp * 8;
+        BODA_CUDA_TRY(launch_kernel(pack_input_s2d_kernel, grid, dim3(256), smem, stream, 1, in, xp, o.C, o.H, o.W, o.stride,
+                                    o.pad, d.H, d.W, p->Cp));
         count_launch();
     }
     if (p->nacc > 0) {
         if (!p->s2d) {
             dim3 grid((p->Hp * p->Wp + 31) / 32, p->Cp / 32, d.N);
-            halo::pack_input_halo_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, d.H, d.W, p->Hp, p->Wp);
-            BODA_CUDA_TRY(cudaGetLastError());
+            BODA_CUDA_TRY(launch_kernel(halo::pack_input_halo_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, d.H, d.W,
+                                        p->Hp, p->Wp));
             count_launch();
         }
         if (p->map_a_base != xp) {
@@ -804,8 +811,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     if (!p->s2d) {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
-        pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
-        BODA_CUDA_TRY(cudaGetLastError());
+        BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW));
         count_launch();
     }
     if (p->map_a_base != xp) {
@@ -903,8 +909,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
-        pack_input_nhwc_kernel<<<grid, 256, 0, stream>>>(in, xp, d.C, p->Cp, HW);
-        cudaError_t e = cudaGetLastError();
+        cudaError_t e = launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW);
         if (e != cudaSuccess) { p->d_wp = nullptr; return record_cuda_error(e, "pack_input_nhwc_kernel"); }
         count_launch();
     }

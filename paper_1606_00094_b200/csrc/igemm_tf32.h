@@ -19,6 +19,7 @@ int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, 
 bool igemm_s2d_applicable(const ConvDims& d);
 void igemm_plan_destroy(IgemmPlan* p);
 int igemm_plan_tile(const IgemmPlan* p);
+int igemm_plan_splits(const IgemmPlan* p);
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p);
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n);
 int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream);

@@ -80,6 +80,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
     const int my_iters = it_end - it_begin;
 
+    pdl_launch_dependents();
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < kASlots; ++s) { mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); }
@@ -97,6 +98,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_acc = s_tmem_base;
+    pdl_wait();          // everything above overlapped the previous kernel; its results are needed from here on
 
     if (warp == 0) {
         if (lane == 0) {
@@ -299,6 +301,8 @@ __global__ void __launch_bounds__(256)
 pack_input_halo_kernel(const float* __restrict__ in, float* __restrict__ xs, int C, int Cp, int H, int W, int Hp, int Wp)
 {
     __shared__ float tile[32][33];
+    pdl_launch_dependents();
+    pdl_wait();
     const int n = blockIdx.z;
     const int f0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
