@@ -223,8 +223,12 @@ int boda_stack_num_ops(const boda_stack* stack);
 int boda_stack_set_filters(boda_stack* stack, int op_index, const float* filt, const float* bias, void* stream);
 /* Output extent [N][C][H][W] of op `op_index`. */
 int boda_stack_out_dims(const boda_stack* stack, int op_index, int* N, int* C, int* H, int* W);
-/* Device pointer to the activation that op `op_index` writes (not for the last op, which writes the caller's buffer). */
-int boda_stack_layer_output(const boda_stack* stack, int op_index, const float** ptr);
+/* Copies the activation that op `op_index` wrote in the last forward pass into dst [N][C][H][W] (device memory, the
+ * extent boda_stack_out_dims reports), on `stream`.  Not for the last op, which writes the caller's buffer.
+ * Between tensor-core layers the stack keeps activations in the consumer's staged layout (channels innermost,
+ * zero padded, rounded to TF32 - the paper's "input transformation", written directly by the producing kernel);
+ * this call converts back. */
+int boda_stack_copy_layer_output(const boda_stack* stack, int op_index, float* dst, void* stream);
 int boda_stack_describe(const boda_stack* stack, int op_index, char* buf, size_t buf_bytes);
 /* Kernels one forward pass launches. */
 int boda_stack_kernels_per_fwd(const boda_stack* stack);

@@ -85,8 +85,8 @@ _lib.boda_stack_set_filters.argtypes = [_vp, _i, _vp, _vp, _vp]
 _lib.boda_stack_set_filters.restype = _i
 _lib.boda_stack_out_dims.argtypes = [_vp, _i] + [ctypes.POINTER(_i)] * 4
 _lib.boda_stack_out_dims.restype = _i
-_lib.boda_stack_layer_output.argtypes = [_vp, _i, ctypes.POINTER(_vp)]
-_lib.boda_stack_layer_output.restype = _i
+_lib.boda_stack_copy_layer_output.argtypes = [_vp, _i, _vp, _vp]
+_lib.boda_stack_copy_layer_output.restype = _i
 _lib.boda_stack_describe.argtypes = [_vp, _i, ctypes.c_char_p, ctypes.c_size_t]
 _lib.boda_stack_describe.restype = _i
 _lib.boda_stack_kernels_per_fwd.argtypes = [_vp]
@@ -258,10 +258,8 @@ def boda_stack_out_dims(stack: int, op_index: int):
     return tuple(x.value for x in v)
 
 
-def boda_stack_layer_output(stack: int, op_index: int) -> int:
-    ptr = _vp()
-    _check(_lib.boda_stack_layer_output(stack, op_index, ctypes.byref(ptr)), "boda_stack_layer_output")
-    return ptr.value
+def boda_stack_copy_layer_output(stack: int, op_index: int, dst, stream=None) -> None:
+    _check(_lib.boda_stack_copy_layer_output(stack, op_index, _addr(dst), _stream(stream)), "boda_stack_copy_layer_output")
 
 
 def boda_stack_describe(stack: int, op_index: int) -> str:

@@ -137,6 +137,7 @@ struct boda_conv_plan {
     DirectTapEntry* d_tab = nullptr;     // DIRECT
     IgemmPlan* ig = nullptr;             // K1CONV / TCONV
     size_t ws_bytes = 0;
+    bool in_packed = false;              // chained layers: the input arrives in the staged layout
 };
 
 namespace boda {
@@ -150,13 +151,28 @@ int conv_fwd_planned_ex(boda_conv_plan* p, const float* in, const float* filt, c
         if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
         return direct_launch(p->d, p->tile_id, in, filt, bias, out, p->d_tab, stream);
     }
-    if (p->ws_bytes && !workspace) return BODA_ERR_NOMEM;
+    if (p->ws_bytes && !workspace && !p->in_packed) return BODA_ERR_NOMEM;
     return igemm_launch(p->ig, in, filt, bias, out, workspace, stream, after_staging);
 }
 
 void conv_plan_out_dims(const boda_conv_plan* p, int* N, int* K, int* P, int* Q)
 {
     *N = p->d.N; *K = p->d.K; *P = p->d.P; *Q = p->d.Q;
+}
+
+bool conv_plan_input_geometry(const boda_conv_plan* p, int* Hp, int* Wp, int* Cp)
+{
+    return p->ig ? igemm_plan_input_geometry(p->ig, Hp, Wp, Cp) : false;
+}
+
+bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr; }
+
+int conv_plan_set_io(boda_conv_plan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
+{
+    if (!p->ig) return (in_packed || out_packed) ? BODA_ERR_UNSUPPORTED : BODA_OK;
+    const int rc = igemm_plan_set_io(p->ig, in_packed, out_packed, oHp, oWp, oCp);
+    if (rc == BODA_OK) p->in_packed = in_packed != 0;
+    return rc;
 }
 
 }  // namespace boda
@@ -332,7 +348,8 @@ size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* p) { return p ? p->w
 int boda_conv_plan_kernels_per_call(const boda_conv_plan* p)
 {
     if (!p) return 0;
-    return p->variant == BODA_VARIANT_DIRECT ? 1 : 2;      // tensor-core variants: input staging + main kernel
+    if (p->variant == BODA_VARIANT_DIRECT) return 1;
+    return p->in_packed ? 1 : 2;                           // tensor-core variants: input staging + main kernel
 }
 
 int boda_conv_plan_bind_filters(boda_conv_plan* p, const float* filt, void* stream)

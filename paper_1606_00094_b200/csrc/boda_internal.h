@@ -101,9 +101,18 @@ int direct_launch(const ConvDims& d, int tile_id, const float* in, const float* 
 int conv_fwd_planned_ex(boda_conv_plan* plan, const float* in, const float* filt, const float* bias, float* out,
                         void* workspace, cudaStream_t stream, cudaEvent_t after_staging);
 void conv_plan_out_dims(const boda_conv_plan* plan, int* N, int* K, int* P, int* Q);
+// chained layers: the staged input layout a tensor-core plan reads (false: the plan reads NCHW only), and the
+// switch that makes it read that layout directly / write its output in a consumer's staged layout
+bool conv_plan_input_geometry(const boda_conv_plan* plan, int* Hp, int* Wp, int* Cp);
+bool conv_plan_can_write_packed(const boda_conv_plan* plan);
+int conv_plan_set_io(boda_conv_plan* plan, int in_packed, int out_packed, int oHp, int oWp, int oCp);
 
 // ---- pooling -------------------------------------------------------------------------------------
 int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,
                    cudaStream_t stream);
+// the same on the staged layout rows [(n*Hp + y)*Wp + x][Cp]; output staged (out_packed) or NCHW
+int maxpool_packed_launch(const float* in, float* out, int N, int C, int H, int W, int iHp, int iWp, int iCp, int ksz, int stride,
+                          int out_packed, int oHp, int oWp, int oCp, cudaStream_t stream);
+int unpack_to_nchw_launch(const float* in, float* out, int N, int C, int H, int W, int Hp, int Wp, int Cp, cudaStream_t stream);
 
 }  // namespace boda

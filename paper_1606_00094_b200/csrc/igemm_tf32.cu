@@ -37,19 +37,19 @@ constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of f
 constexpr int A_STAGE_BYTES = BM * BKC * 4;
 constexpr int kIgemmThreads = 192;
 
+using namespace tc;
+
 struct IgemmParams {
-    int M, K, PQ, Q, stride, pad, S;
+    int M, stride, pad, S;
     int cchunks;                 // Cp / 32
     int iters_total;             // taps * cchunks
     int iters_per_split;
     int splits;
-    int relu;
     const float* bias;
-    float* out;
+    OutSpec o;                   // output tensor, layout and activation
     int* status;
 };
 
-using namespace tc;
 
 template <int BN> struct TileCfg {
     static constexpr int B_STAGE_BYTES = BN * BKC * 4;
@@ -58,6 +58,20 @@ template <int BN> struct TileCfg {
     static constexpr int TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
+
+// output location of GEMM row m = (n, p, q)
+__device__ __forceinline__ RowDst igemm_row_dst(const IgemmParams& p, int m)
+{
+    const bool valid = m < p.M;
+    int n = 0, pp = 0, qq = 0;
+    if (valid) {
+        n = m / p.o.PQ;
+        const int pq = m - n * p.o.PQ;
+        pp = pq / p.o.Q;
+        qq = pq - pp * p.o.Q;
+    }
+    return row_dst(p.o, valid, n, pp, qq);
+}
 
 // ------------------------------------------------------------------------------------------------
 template <int BN>
@@ -109,10 +123,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (warp == 0) {
         if (lane == 0) {
             // ---------------- TMA producer
-            const int n0 = m0 / p.PQ;
-            const int rem = m0 - n0 * p.PQ;
-            const int p0 = rem / p.Q;
-            const int q0 = rem - p0 * p.Q;
+            const int n0 = m0 / p.o.PQ;
+            const int rem = m0 - n0 * p.o.PQ;
+            const int p0 = rem / p.o.Q;
+            const int q0 = rem - p0 * p.o.Q;
             const int w0 = q0 * p.stride - p.pad;
             const int h0 = p0 * p.stride - p.pad;
             int tap = it_begin / p.cchunks;
@@ -165,7 +179,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int m = m0 + row;
         // bias of this tile's channels into shared memory while the main loop runs (0 where there is none)
         for (int j = threadIdx.x - 64; j < BN; j += 128)
-            s_bias[j] = (p.bias && k0 + j < p.K) ? __ldg(p.bias + k0 + j) : 0.f;
+            s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
         if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 4);   // one poller per warp
         __syncwarp();
         // All 128 epilogue threads meet here whatever their wait returned, then take one common decision:
@@ -173,12 +187,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const bool ok = (s_abort == 0);
         tc_fence_after();
-        const bool m_ok = m < p.M;
-        int n = 0, pq = 0;
-        if (m_ok) { n = m / p.PQ; pq = m - n * p.PQ; }
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         if (ok && p.splits == 1) {
-            float* o = p.out + ((size_t)n * p.K) * p.PQ + pq;
+            const RowDst d = igemm_row_dst(p, m);
 #pragma unroll 1
             for (int j0 = 0; j0 < BN; j0 += 32) {
                 uint32_t v[32];
@@ -188,30 +199,19 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
                     y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
-                    if (p.relu) y[j] = fmaxf(y[j], 0.f);
+                    if (p.o.relu) y[j] = fmaxf(y[j], 0.f);
                 }
-                if (m_ok) {
-                    float* oj = o + (size_t)(k0 + j0) * p.PQ;
-                    if (k0 + j0 + 32 <= p.K) {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j) oj[(size_t)j * p.PQ] = y[j];
-                    } else {
-#pragma unroll
-                        for (int j = 0; j < 32; ++j)
-                            if (k0 + j0 + j < p.K) oj[(size_t)j * p.PQ] = y[j];
-                    }
-                }
+                store_row32(p.o, d, k0 + j0, y, smem_base + (uint32_t)(warp & 3) * 4224u);
             }
         } else if (ok) {
             // split reduction, step 1: park this CTA's partial accumulator in its own shared memory (the stage
-            // buffers are idle now), column-major [channel][128 rows]; the cluster-wide sum follows below.
+            // buffers are idle now); the cluster-wide sum follows below.
 #pragma unroll 1
             for (int j0 = 0; j0 < BN; j0 += 32) {
                 uint32_t v[32];
                 tmem_ld_32cols(trow + j0, v);
                 tmem_ld_wait();
-#pragma unroll
-                for (int j = 0; j < 32; ++j) st_shared_f32(smem_base + (uint32_t)((j0 + j) * 128 + row) * 4u, __uint_as_float(v[j]));
+                stash_row32<BN>(smem_base, row, j0, v);
             }
         }
         tc_fence_before();
@@ -222,14 +222,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // cluster barrier each of them sums its share of the channels over all peers' shared memory and stores it.
         cluster_sync_all();
         if (warp >= 2 && s_abort == 0) {
-            auto row_info = [&](int row, bool& valid, size_t& obase) {
-                const int m = m0 + row;
-                valid = m < p.M;
-                obase = 0;
-                if (valid) { const int n = m / p.PQ; obase = ((size_t)n * p.K) * p.PQ + (size_t)(m - n * p.PQ); }
-            };
-            cluster_reduce_store<BN>(smem_base, (int)threadIdx.x - 64, cluster_cta_rank(), p.splits, row_info, (size_t)p.PQ,
-                                     k0, p.K, p.relu, s_bias, p.out);
+            const int row = (warp & 3) * 32 + lane;
+            cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
         }
         cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
     }
@@ -430,6 +424,9 @@ struct IgemmPlan {
     CUtensorMap map_b;
     CUtensorMap map_a;
     const void* map_a_base = nullptr;
+    // activation layouts on either side (set by igemm_plan_set_io; NCHW by default)
+    bool in_packed = false;          // the input already is this plan's staged layout: skip the staging kernel
+    int out_packed = 0, oHp = 0, oWp = 0, oCp = 0;
     // halo kernel only
     int nacc = 0;                    // 0: im2col kernel; 1 or 2: halo kernel with that many accumulators
     int Hp = 0, Wp = 0, lead = 0, slab_rows = 0, nbox = 0, box_rows = 0, a_slot_bytes = 0, b_stages = 0;
@@ -756,19 +753,49 @@ int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
 
 void igemm_unbind_filters(IgemmPlan* p) { p->bound_filt = nullptr; }
 
+static OutSpec make_out_spec(const IgemmPlan* p, float* out)
+{
+    const ConvDims& d = p->d;
+    OutSpec o;
+    o.out = out;
+    o.packed = p->out_packed;
+    o.K = d.K; o.P = d.P; o.Q = d.Q; o.PQ = d.P * d.Q;
+    o.Hp = p->oHp; o.Wp = p->oWp; o.Cp = p->oCp;
+    o.relu = d.relu;
+    return o;
+}
+
+bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
+{
+    if (p->s2d) return false;                       // the space-to-depth staging reads NCHW only
+    if (p->nacc > 0) { *Hp = p->Hp; *Wp = p->Wp; } else { *Hp = p->d.H; *Wp = p->d.W; }
+    *Cp = p->Cp;
+    return true;
+}
+
+int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
+{
+    if (in_packed && p->s2d) return BODA_ERR_UNSUPPORTED;
+    if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < p->d.P || oWp < p->d.Q)) return BODA_ERR_INVALID_ARG;
+    p->in_packed = in_packed != 0;
+    p->out_packed = out_packed ? 1 : 0;
+    p->oHp = oHp; p->oWp = oWp; p->oCp = oCp;
+    return BODA_OK;
+}
+
 int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
                  cudaStream_t stream, cudaEvent_t after_staging)
 {
     const ConvDims& d = p->d;
-    if (!workspace) return BODA_ERR_NOMEM;
-    if (((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
-    float* xp = (float*)workspace;
+    if (!p->in_packed && !workspace) return BODA_ERR_NOMEM;
+    if (!p->in_packed && ((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
+    float* xp = p->in_packed ? const_cast<float*>(in) : (float*)workspace;
     if (filt != p->bound_filt || !filt) {
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
     }
-    if (p->s2d) {
+    if (p->s2d && !p->in_packed) {
         // both kernels read the same [N][H'][W'][Cp] layout here (the view has no padding)
         const ConvDims& o = p->orig;
         dim3 grid(d.H, d.N);
@@ -778,7 +805,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         count_launch();
     }
     if (p->nacc > 0) {
-        if (!p->s2d) {
+        if (!p->s2d && !p->in_packed) {
             dim3 grid((p->Hp * p->Wp + 31) / 32, p->Cp / 32, d.N);
             BODA_CUDA_TRY(launch_kernel(halo::pack_input_halo_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, d.H, d.W,
                                         p->Hp, p->Wp));
@@ -790,11 +817,11 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         }
         if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
         halo::HaloParams hp;
-        hp.Mflat = d.N * p->Hp * p->Wp; hp.HpWp = p->Hp * p->Wp; hp.Wp = p->Wp; hp.P = d.P; hp.Q = d.Q; hp.K = d.K;
+        hp.Mflat = d.N * p->Hp * p->Wp; hp.HpWp = p->Hp * p->Wp; hp.Wp = p->Wp;
         hp.S = d.S; hp.taps = d.R * d.S; hp.cchunks = p->Cp / BKC; hp.lead = p->lead;
         hp.nbox = p->nbox; hp.box_rows = p->box_rows; hp.a_slot_bytes = p->a_slot_bytes; hp.b_stages = p->b_stages;
         hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
-        hp.relu = d.relu; hp.bias = bias; hp.out = out;
+        hp.bias = bias; hp.o = make_out_spec(p, out);
         hp.status = p->d_status;
         switch (p->BN * 10 + p->nacc) {
             case 641: return launch_halo<64, 1>(p, hp, stream);
@@ -808,7 +835,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
             default: return BODA_ERR_UNSUPPORTED;
         }
     }
-    if (!p->s2d) {
+    if (!p->s2d && !p->in_packed) {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
         BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW));
@@ -820,14 +847,13 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     }
     if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
     IgemmParams prm;
-    prm.M = d.M; prm.K = d.K; prm.PQ = d.P * d.Q; prm.Q = d.Q; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
+    prm.M = d.M; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
     prm.cchunks = p->Cp / BKC;
     prm.iters_total = p->iters_total;
     prm.iters_per_split = p->iters_per_split;
     prm.splits = p->splits;
-    prm.relu = d.relu;
     prm.bias = bias;
-    prm.out = out;
+    prm.o = make_out_spec(p, out);
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: return launch_bn<64>(p, prm, stream);
@@ -914,14 +940,13 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
         count_launch();
     }
     IgemmParams prm;
-    prm.M = d.M; prm.K = d.K; prm.PQ = d.P * d.Q; prm.Q = d.Q; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
+    prm.M = d.M; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
     prm.cchunks = p->Cp / BKC;
     prm.iters_total = p->iters_total;
     prm.iters_per_split = p->iters_per_split;
     prm.splits = p->splits;
-    prm.relu = d.relu;
     prm.bias = bias;
-    prm.out = out;
+    prm.o = make_out_spec(p, out);
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: rc = launch_bn<64>(p, prm, stream); break;

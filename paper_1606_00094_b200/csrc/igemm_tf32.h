@@ -28,6 +28,13 @@ void igemm_unbind_filters(IgemmPlan* p);
 int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* bias, float* out, void* workspace,
                  cudaStream_t stream, cudaEvent_t after_staging = nullptr);
 
+// Activation layouts for chained layers.  igemm_plan_input_geometry: the staged input layout this plan reads,
+// rows [(n*Hp + y)*Wp + x][Cp] (false if the plan cannot take a staged input).  igemm_plan_set_io: in_packed =
+// the `in` pointer of igemm_launch already is that layout (no staging kernel, no workspace); out_packed = write
+// the output as rows [(n*oHp + p)*oWp + q][oCp] rounded to TF32 instead of NCHW.
+bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp);
+int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp);
+
 // Scratch-in-a-caller-region form (allocates nothing): bytes needed at least, and the run itself.
 size_t igemm_region_min_bytes(const ConvDims& d);
 int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const float* filt, const float* bias,

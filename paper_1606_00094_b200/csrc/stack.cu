@@ -2,6 +2,7 @@
 // The stack owns the plans, the activations between layers, one workspace shared by all layers and a CUDA graph
 // of the whole chain, so that a forward pass is a single graph launch with no host work between kernels.
 #include <cstdio>
+#include <cstdlib>
 #include <cstring>
 #include <new>
 #include <string>
@@ -22,7 +23,12 @@ struct boda_stack {
         int N = 0, C = 0, H = 0, W = 0;     // input dims of this op
         int oC = 0, oH = 0, oW = 0;         // output dims
         float* out = nullptr;               // owned activation (nullptr for the last op: the caller's buffer)
-        size_t out_elems = 0;
+        size_t out_elems = 0;               // elements of the NCHW view of the output
+        // layout of the output activation: NCHW, or the consumer's staged layout rows [(n*Hp + y)*Wp + x][Cp]
+        bool out_packed = false;
+        int oHp = 0, oWp = 0, oCp = 0;
+        bool in_packed = false;             // = out_packed of the previous op
+        int iHp = 0, iWp = 0, iCp = 0;
     };
     std::vector<Op> ops;
     int device = 0;
@@ -53,7 +59,11 @@ int run_ops(boda_stack* s, const float* in, float* out, cudaStream_t stream, cud
             rc = conv_fwd_planned_ex(op.plan, cur, op.filt, op.bias, dst, s->workspace, stream, events ? events[3 * i + 1] : nullptr);
         } else {
             if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 1], stream));
-            rc = maxpool_launch(cur, dst, op.N, op.C, op.H, op.W, op.ksz, op.stride, stream);
+            if (op.in_packed)
+                rc = maxpool_packed_launch(cur, dst, op.N, op.C, op.H, op.W, op.iHp, op.iWp, op.iCp, op.ksz, op.stride,
+                                           op.out_packed ? 1 : 0, op.oHp, op.oWp, op.oCp, stream);
+            else
+                rc = maxpool_launch(cur, dst, op.N, op.C, op.H, op.W, op.ksz, op.stride, stream);
         }
         if (rc != BODA_OK) return rc;
         if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 2], stream));
@@ -150,12 +160,37 @@ int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts*
             if (op.oH <= 0 || op.oW <= 0) { rc = BODA_ERR_INVALID_ARG; break; }
         } else { rc = BODA_ERR_INVALID_ARG; break; }
         op.out_elems = (size_t)N * op.oC * op.oH * op.oW;
-        if (i < n_ops - 1) {
-            cudaError_t e = cudaMalloc(&op.out, op.out_elems * sizeof(float));
-            if (e != cudaSuccess) { if (op.plan) boda_conv_plan_destroy(op.plan); rc = record_cuda_error(e, "activation allocation"); break; }
-        }
         s->ops.push_back(op);
         C = op.oC; H = op.oH; W = op.oW;
+    }
+    // Layout of every activation between two ops: the consumer's staged layout whenever the producer can write it
+    // (a tensor-core convolution, or a pool whose own input is staged) and the consumer can read it (a tensor-core
+    // convolution that is not a space-to-depth view, or a pool); NCHW otherwise.  The chain's input and output are NCHW.
+    const bool chain_layouts = !std::getenv("BODA_STACK_NCHW");
+    for (int i = 0; rc == BODA_OK && i + 1 < (int)s->ops.size(); ++i) {
+        boda_stack::Op& prod = s->ops[i];
+        boda_stack::Op& cons = s->ops[i + 1];
+        const bool can_write = prod.kind == BODA_STACK_CONV ? conv_plan_can_write_packed(prod.plan) : prod.in_packed;
+        int Hp = cons.H, Wp = cons.W, Cp = ((cons.C + 31) / 32) * 32;
+        bool can_read = true;
+        if (cons.kind == BODA_STACK_CONV) can_read = conv_plan_input_geometry(cons.plan, &Hp, &Wp, &Cp);
+        if (chain_layouts && can_write && can_read) {
+            prod.out_packed = true; prod.oHp = Hp; prod.oWp = Wp; prod.oCp = Cp;
+            cons.in_packed = true; cons.iHp = Hp; cons.iWp = Wp; cons.iCp = Cp;
+        }
+    }
+    for (int i = 0; rc == BODA_OK && i < (int)s->ops.size(); ++i) {
+        boda_stack::Op& op = s->ops[i];
+        if (op.kind == BODA_STACK_CONV) {
+            rc = conv_plan_set_io(op.plan, op.in_packed ? 1 : 0, op.out_packed ? 1 : 0, op.oHp, op.oWp, op.oCp);
+            if (rc != BODA_OK) break;
+        }
+        if (i + 1 < (int)s->ops.size()) {
+            const size_t elems = op.out_packed ? (size_t)op.N * op.oHp * op.oWp * op.oCp : op.out_elems;
+            cudaError_t e = cudaMalloc(&op.out, elems * sizeof(float));
+            if (e == cudaSuccess) e = cudaMemset(op.out, 0, elems * sizeof(float));   // staged layouts: the padding stays zero
+            if (e != cudaSuccess) { rc = record_cuda_error(e, "activation allocation"); break; }
+        }
     }
     if (rc == BODA_OK) {
         s->out_elems = s->ops.back().out_elems;
@@ -192,10 +227,13 @@ int boda_stack_out_dims(const boda_stack* s, int op_index, int* N, int* C, int* 
     return BODA_OK;
 }
 
-int boda_stack_layer_output(const boda_stack* s, int op_index, const float** ptr)
+int boda_stack_copy_layer_output(const boda_stack* s, int op_index, float* dst_nchw, void* stream)
 {
-    if (!s || op_index < 0 || op_index >= (int)s->ops.size() - 1 || !ptr) return BODA_ERR_INVALID_ARG;
-    *ptr = s->ops[op_index].out;
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size() - 1 || !dst_nchw) return BODA_ERR_INVALID_ARG;
+    const boda_stack::Op& op = s->ops[op_index];
+    if (op.out_packed)
+        return unpack_to_nchw_launch(op.out, dst_nchw, op.N, op.oC, op.oH, op.oW, op.oHp, op.oWp, op.oCp, (cudaStream_t)stream);
+    BODA_CUDA_TRY(cudaMemcpyAsync(dst_nchw, op.out, op.out_elems * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
     return BODA_OK;
 }
 
@@ -203,8 +241,14 @@ int boda_stack_describe(const boda_stack* s, int op_index, char* buf, size_t n)
 {
     if (!s || op_index < 0 || op_index >= (int)s->ops.size() || !buf || n == 0) return BODA_ERR_INVALID_ARG;
     const boda_stack::Op& op = s->ops[op_index];
-    if (op.kind == BODA_STACK_CONV) return boda_conv_plan_describe(op.plan, buf, n);
-    std::snprintf(buf, n, "maxpool %dx%d stride %d", op.ksz, op.ksz, op.stride);
+    char tmp[400];
+    if (op.kind == BODA_STACK_CONV) {
+        const int rc = boda_conv_plan_describe(op.plan, tmp, sizeof(tmp));
+        if (rc != BODA_OK) return rc;
+    } else {
+        std::snprintf(tmp, sizeof(tmp), "maxpool %dx%d stride %d", op.ksz, op.ksz, op.stride);
+    }
+    std::snprintf(buf, n, "%s in=%s out=%s", tmp, op.in_packed ? "staged" : "nchw", op.out_packed ? "staged" : "nchw");
     return BODA_OK;
 }
 

@@ -201,64 +201,114 @@ __device__ __forceinline__ float4 ld_cluster_v4(uint32_t addr)
     asm volatile("ld.shared::cluster.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
     return v;
 }
-
-// Split reduction of one 128-row accumulator over the CTAs of a cluster (one CTA per reduction split).
-// Every CTA has parked its partial accumulator in its own shared memory at `stash`, column-major
-// [col][128 rows]; the cluster has synchronised.  CTA `rank` owns the columns rank*per .. and sums them over
-// all CTAs in rank order (so the result does not depend on which CTA does the summing), adds the bias,
-// applies ReLU and stores: each split CTA writes its share of the output tile.
-// Work split inside the CTA (128 epilogue threads, t = 0..127): thread t sums rows 4*(t%32) .. +3 (one 16-byte
-// remote load per peer and column) of the columns c with (c - c_begin) % 4 == t/32, eight columns per pass so
-// that 8 x splits remote loads are in flight (remote shared memory has the latency of an L2 access).
-// `row_info(row, valid, obase)` locates a row in `out`: element (row, k) lives at out[obase + k * k_stride].
-template <int BN, typename RowInfo>
-__device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int t, uint32_t rank, int splits, RowInfo row_info,
-                                                     size_t k_stride, int k0, int K, int relu, const float* s_bias,
-                                                     float* out)
+__device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, float c, float d)
 {
-    const int per = (((BN + splits - 1) / splits) + 3) & ~3;
+    asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" :: "r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
+}
+__device__ __forceinline__ float round_to_tf32(float x)
+{
+    uint32_t r;
+    asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
+    return __uint_as_float(r);
+}
+
+// ---- where a tensor-core kernel writes its output tile (fused bias + ReLU epilogue, Section 2 of the paper)
+struct OutSpec {
+    float* out;
+    int packed;          // 0: NCHW [N][K][P][Q] fp32.  1: the next layer's staged input, rows [(n*Hp + p)*Wp + q][Cp]
+                         //    of fp32 values rounded to TF32 (padding rows, columns and channels are never written)
+    int K, P, Q, PQ;
+    int Hp, Wp, Cp;      // packed geometry
+    int relu;
+};
+struct RowDst { bool valid; size_t base; };
+
+__device__ __forceinline__ RowDst row_dst(const OutSpec& o, bool valid, int n, int pp, int qq)
+{
+    RowDst d;
+    d.valid = valid;
+    d.base = !valid ? 0 : o.packed ? ((size_t)(n * o.Hp + pp) * o.Wp + qq) * (size_t)o.Cp
+                                   : (size_t)n * o.K * o.PQ + (size_t)pp * o.Q + qq;
+    return d;
+}
+
+// 32 consecutive output channels kc .. kc+31 of one output row (one row per lane; bias and ReLU already applied).
+// NCHW: lane = pixel, so each of the 32 stores of a lane joins its neighbours' into one 128-byte line.
+// Staged layout: see below.  (`tile` is a per-warp shared-memory scratch address, currently unused.)
+__device__ __forceinline__ void store_row32(const OutSpec& o, const RowDst& d, int kc, const float (&y)[32], uint32_t tile)
+{
+    if (o.packed) {
+        // channels are innermost: the lane's 32 values are 128 contiguous bytes; four 32-byte stores, each a whole sector
+        if (d.valid && kc < o.Cp) {    // Cp is a multiple of 32; channels K..Cp-1 hold exact zeros here (zero filters, zero bias)
+            float* dst = o.out + d.base + kc;
+#pragma unroll
+            for (int g = 0; g < 4; ++g)
+                asm volatile("st.global.v8.f32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8};"
+                             :: "l"(dst + 8 * g), "f"(round_to_tf32(y[8 * g])), "f"(round_to_tf32(y[8 * g + 1])),
+                                "f"(round_to_tf32(y[8 * g + 2])), "f"(round_to_tf32(y[8 * g + 3])), "f"(round_to_tf32(y[8 * g + 4])),
+                                "f"(round_to_tf32(y[8 * g + 5])), "f"(round_to_tf32(y[8 * g + 6])), "f"(round_to_tf32(y[8 * g + 7]))
+                             : "memory");
+        }
+        (void)tile;
+    } else if (d.valid) {
+        float* oj = o.out + d.base + (size_t)kc * o.PQ;
+        if (kc + 32 <= o.K) {
+#pragma unroll
+            for (int j = 0; j < 32; ++j) oj[(size_t)j * o.PQ] = y[j];
+        } else {
+#pragma unroll
+            for (int j = 0; j < 32; ++j)
+                if (kc + j < o.K) oj[(size_t)j * o.PQ] = y[j];
+        }
+    }
+}
+
+// ---- split reduction of one 128-row accumulator over the CTAs of a cluster (one CTA per reduction split).
+// Step 1: every CTA parks its partial accumulator in its own shared memory, column-major [channel][128 rows]:
+// a warp (32 consecutive rows) then touches 128 contiguous bytes per channel, both when it writes here and when a
+// peer reads it through distributed shared memory (remote reads want to be coalesced like global ones).
+template <int BN>
+__device__ __forceinline__ void stash_row32(uint32_t stash, int row, int j0, const uint32_t (&v)[32])
+{
+    const uint32_t a = stash + (uint32_t)(j0 * 128 + row) * 4u;
+#pragma unroll
+    for (int j = 0; j < 32; ++j) st_shared_f32(a + 512u * j, __uint_as_float(v[j]));
+}
+// Step 2 (after a cluster barrier): CTA `rank` owns a slice of the channels (a multiple of 32 wide); thread `row`
+// sums its row of that slice over all CTAs in rank order - so the result does not depend on which CTA sums -
+// adds the bias, applies ReLU and stores.  Remote shared memory has the latency of an L2 access, so each pass
+// keeps 32 loads per peer in flight.
+template <int BN>
+__device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int row, uint32_t rank, int splits, const RowDst& d,
+                                                     const OutSpec& o, int k0, const float* s_bias, uint32_t tile)
+{
+    const int per = ((((BN + splits - 1) / splits) + 31) / 32) * 32;
     const int c_begin = (int)rank * per;
     const int c_end = min(BN, c_begin + per);
-    const int rbase = (t & 31) * 4;
-    const int csel = t >> 5;
-    bool valid[4];
-    size_t obase[4];
-#pragma unroll
-    for (int e = 0; e < 4; ++e) row_info(rbase + e, valid[e], obase[e]);
     uint32_t peer[8];
 #pragma unroll
-    for (int r = 0; r < 8; ++r) peer[r] = r < splits ? map_to_cta(stash + (uint32_t)rbase * 4u, (uint32_t)r) : 0u;
+    for (int r = 0; r < 8; ++r) peer[r] = r < splits ? map_to_cta(stash + (uint32_t)row * 4u, (uint32_t)r) : 0u;
 #pragma unroll 1
-    for (int c0 = c_begin + csel; c0 < c_end; c0 += 32) {
-        float4 sum[8];
+    for (int c0 = c_begin; c0 < c_end; c0 += 32) {
+        float y[32];
 #pragma unroll
-        for (int u = 0; u < 8; ++u) sum[u] = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int j = 0; j < 32; ++j) y[j] = 0.f;
 #pragma unroll
         for (int r = 0; r < 8; ++r) {
             if (r < splits) {
+                float x[32];
 #pragma unroll
-                for (int u = 0; u < 8; ++u) {
-                    const int c = c0 + 4 * u;
-                    if (c < c_end) {
-                        const float4 x = ld_cluster_v4(peer[r] + (uint32_t)c * 512u);
-                        sum[u].x += x.x; sum[u].y += x.y; sum[u].z += x.z; sum[u].w += x.w;
-                    }
-                }
+                for (int j = 0; j < 32; ++j) x[j] = ld_cluster_f32(peer[r] + (uint32_t)(c0 + j) * 512u);
+#pragma unroll
+                for (int j = 0; j < 32; ++j) y[j] += x[j];
             }
         }
 #pragma unroll
-        for (int u = 0; u < 8; ++u) {
-            const int c = c0 + 4 * u, k = k0 + c;
-            if (c < c_end && k < K) {
-                const float bv = s_bias[c];
-                float y[4] = {sum[u].x + bv, sum[u].y + bv, sum[u].z + bv, sum[u].w + bv};
-#pragma unroll
-                for (int e = 0; e < 4; ++e) {
-                    if (relu) y[e] = fmaxf(y[e], 0.f);
-                    if (valid[e]) out[obase[e] + (size_t)k * k_stride] = y[e];
-                }
-            }
+        for (int j = 0; j < 32; ++j) {
+            y[j] += s_bias[c0 + j];
+            if (o.relu) y[j] = fmaxf(y[j], 0.f);
         }
+        store_row32(o, d, k0 + c0, y, tile);
     }
 }
 

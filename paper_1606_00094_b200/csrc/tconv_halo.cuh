@@ -33,18 +33,32 @@ constexpr int kSmemBudget = 200 * 1024;
 
 struct HaloParams {
     int Mflat;                   // N * Hp * Wp flat output positions
-    int HpWp, Wp, P, Q, K;
+    int HpWp, Wp;
     int S, taps, cchunks;
     int lead;                    // pad*Wp + pad
     int nbox, box_rows;          // slab = nbox TMA boxes of box_rows rows
     int a_slot_bytes;            // nbox * box_rows * 128, multiple of 1024
     int b_stages;
     int iters_total, iters_per_split, splits;
-    int relu;
     const float* bias;
-    float* out;
+    OutSpec o;                   // output tensor, layout and activation
     int* status;
 };
+
+// output location of flat position f = (n*Hp + p)*Wp + q; positions with p >= P or q >= Q are dropped
+__device__ __forceinline__ RowDst halo_row_dst(const HaloParams& p, int f)
+{
+    bool valid = f < p.Mflat;
+    int n = 0, pp = 0, qq = 0;
+    if (valid) {
+        n = f / p.HpWp;
+        const int rem = f - n * p.HpWp;
+        pp = rem / p.Wp;
+        qq = rem - pp * p.Wp;
+        valid = pp < p.o.P && qq < p.o.Q;
+    }
+    return row_dst(p.o, valid, n, pp, qq);
+}
 
 template <int BN, int NACC>
 struct HaloCfg {
@@ -193,28 +207,17 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const int quarter = warp & 3;
         const int row = quarter * 32 + lane;
         for (int j = threadIdx.x - 64; j < BN; j += 128)
-            s_bias[j] = (p.bias && k0 + j < p.K) ? __ldg(p.bias + k0 + j) : 0.f;
+            s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
         if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 16);   // one poller per warp
         __syncwarp();
         asm volatile("bar.sync 1, 128;" ::: "memory");
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-        const int PQ = p.P * p.Q;
         if (ok && p.splits == 1) {
 #pragma unroll 1
             for (int acc = 0; acc < NACC; ++acc) {
-                const int f = f0 + acc * 128 + row;
-                bool valid = f < p.Mflat;
-                size_t obase = 0;
-                if (valid) {
-                    const int n = f / p.HpWp;
-                    const int rem = f - n * p.HpWp;
-                    const int pp = rem / p.Wp;
-                    const int qq = rem - pp * p.Wp;
-                    valid = pp < p.P && qq < p.Q;
-                    obase = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
-                }
+                const RowDst d = halo_row_dst(p, f0 + acc * 128 + row);
 #pragma unroll 1
                 for (int j0 = 0; j0 < BN; j0 += 32) {
                     uint32_t v[32];
@@ -224,19 +227,9 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) {
                         y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
-                        if (p.relu) y[j] = fmaxf(y[j], 0.f);
+                        if (p.o.relu) y[j] = fmaxf(y[j], 0.f);
                     }
-                    if (valid) {
-                        float* oj = p.out + obase + (size_t)(k0 + j0) * PQ;
-                        if (k0 + j0 + 32 <= p.K) {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j) oj[(size_t)j * PQ] = y[j];
-                        } else {
-#pragma unroll
-                            for (int j = 0; j < 32; ++j)
-                                if (k0 + j0 + j < p.K) oj[(size_t)j * PQ] = y[j];
-                        }
-                    }
+                    store_row32(p.o, d, k0 + j0, y, smem_base + (uint32_t)(warp & 3) * 4224u);
                 }
             }
         }
@@ -261,30 +254,13 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     uint32_t v[32];
                     tmem_ld_32cols(trow + j0, v);
                     tmem_ld_wait();
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) st_shared_f32(smem_base + (uint32_t)((j0 + j) * 128 + row) * 4u, __uint_as_float(v[j]));
+                    stash_row32<BN>(smem_base, row, j0, v);
                 }
                 tc_fence_before();
             }
             cluster_sync_all();
-            if (warp >= 2 && ok) {
-                const int PQ = p.P * p.Q;
-                auto row_info = [&](int r, bool& valid, size_t& obase) {
-                    const int f = f0 + acc * 128 + r;
-                    valid = f < p.Mflat;
-                    obase = 0;
-                    if (valid) {
-                        const int n = f / p.HpWp;
-                        const int rem = f - n * p.HpWp;
-                        const int pp = rem / p.Wp;
-                        const int qq = rem - pp * p.Wp;
-                        valid = pp < p.P && qq < p.Q;
-                        obase = ((size_t)n * p.K) * PQ + (size_t)pp * p.Q + qq;
-                    }
-                };
-                cluster_reduce_store<BN>(smem_base, (int)threadIdx.x - 64, rank, p.splits, row_info, (size_t)PQ, k0, p.K,
-                                         p.relu, s_bias, p.out);
-            }
+            if (warp >= 2 && ok)
+                cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
             cluster_sync_all();      // peers are done with this CTA's shared memory
         }
     }

@@ -74,15 +74,13 @@ class ConvStack:
         B.boda_stack_fwd_host(self.handle, x_host, out_host)
 
     def layer_output(self, i: int) -> torch.Tensor:
-        """Copy of the activation op i wrote during the last forward pass."""
+        """NCHW copy of the activation op i wrote during the last forward pass."""
         if i == len(self.ops) - 1:
             return self.out.clone()
         shape = B.boda_stack_out_dims(self.handle, i)
-        n = shape[0] * shape[1] * shape[2] * shape[3]
-        ptr = B.boda_stack_layer_output(self.handle, i)
         dst = torch.empty(shape, dtype=torch.float32, device=self.out.device)
-        # device-to-device copy of the library-owned buffer into a torch tensor
-        _copy_d2d(dst.data_ptr(), ptr, n * 4)
+        B.boda_stack_copy_layer_output(self.handle, i, dst)
+        torch.cuda.synchronize()
         return dst
 
     def close(self) -> None:
@@ -95,20 +93,3 @@ class ConvStack:
             self.close()
         except Exception:
             pass
-
-
-def _copy_d2d(dst_ptr: int, src_ptr: int, nbytes: int) -> None:
-    """Device-to-device copy through torch's view of raw memory (plumbing only)."""
-    torch.cuda.synchronize()
-    src = _as_tensor(src_ptr, nbytes)
-    dst = _as_tensor(dst_ptr, nbytes)
-    dst.copy_(src)
-    torch.cuda.synchronize()
-
-
-def _as_tensor(ptr: int, nbytes: int) -> torch.Tensor:
-    class _Holder:
-        pass
-    h = _Holder()
-    h.__cuda_array_interface__ = {"shape": (nbytes,), "typestr": "|u1", "data": (ptr, False), "version": 2}
-    return torch.as_tensor(h, device="cuda")
