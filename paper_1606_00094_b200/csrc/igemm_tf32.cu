@@ -397,9 +397,9 @@ int load_driver_entry_points()
 }
 
 // Tile table.  Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
-// with NACC accumulators of 128 rows each.
-constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256};
-constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2};
+// with NACC accumulators of 128 rows each (ids 5..8: 1, 9..12: 2, 13..15: 4).
+constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4};
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
 constexpr int kFirstHaloTile = 5;
 constexpr int kSplitCandidates[] = {1, 2, 3, 4, 6, 8};
@@ -440,7 +440,7 @@ static bool halo_geometry(const ConvDims& d, int BN, int nacc, IgemmPlan* p)
     const int Hp = d.H + d.pad, Wp = d.W + d.pad;
     const int slab_rows = 128 * nacc + (d.R - 1) * Wp + (d.S - 1);
     const int nbox = (slab_rows + 255) / 256;
-    if (nbox > 2) return false;
+    if (nbox > 3) return false;
     const int box_rows = ((((slab_rows + nbox - 1) / nbox) + 7) / 8) * 8;
     const int a_slot = nbox * box_rows * 128;
     const int b_stage = BN * 128;
@@ -832,6 +832,9 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
             case 1282: return launch_halo<128, 2>(p, hp, stream);
             case 1922: return launch_halo<192, 2>(p, hp, stream);
             case 2562: return launch_halo<256, 2>(p, hp, stream);
+            case 644: return launch_halo<64, 4>(p, hp, stream);
+            case 964: return launch_halo<96, 4>(p, hp, stream);
+            case 1284: return launch_halo<128, 4>(p, hp, stream);
             default: return BODA_ERR_UNSUPPORTED;
         }
     }

@@ -26,7 +26,7 @@ namespace halo {
 
 using namespace tc;
 
-constexpr int kThreads = 192;
+constexpr int kThreads = 224;      // warp 0 producer, 1 and 6 MMA issuers, 2..5 epilogue
 constexpr int kMaxBStages = 8;
 constexpr int kASlots = 2;
 constexpr int kSmemBudget = 200 * 1024;
@@ -66,6 +66,9 @@ struct HaloCfg {
     static constexpr int ACC_COLS = BN * NACC;
     static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
     static_assert(ACC_COLS <= 512, "accumulators exceed tensor memory");
+    // One thread can issue an MMA about every 70 clocks; two threads in different warps, each feeding its own
+    // accumulators, reach about 50 (measured).  With two or more accumulators the work is split between two issuers.
+    static constexpr int ISSUERS = NACC >= 2 ? 2 : 1;
 };
 
 template <int BN, int NACC>
@@ -97,9 +100,9 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         s_abort = 0;
-        for (int s = 0; s < kASlots; ++s) { mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, 1); }
-        for (int s = 0; s < p.b_stages; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, 1); }
-        mbar_init(accum_bar, 1);
+        for (int s = 0; s < kASlots; ++s) { mbar_init(a_full + 8 * s, 1); mbar_init(a_empty + 8 * s, Cfg::ISSUERS); }
+        for (int s = 0; s < p.b_stages; ++s) { mbar_init(b_full + 8 * s, 1); mbar_init(b_empty + 8 * s, Cfg::ISSUERS); }
+        mbar_init(accum_bar, Cfg::ISSUERS);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
@@ -134,6 +137,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     const uint32_t dst = smem_a + a_slot * p.a_slot_bytes;
                     tma_load_2d(dst, &map_a, fb, cx, row0);
                     if (p.nbox > 1) tma_load_2d(dst + p.box_rows * 128, &map_a, fb, cx, row0 + p.box_rows);
+                    if (p.nbox > 2) tma_load_2d(dst + 2 * p.box_rows * 128, &map_a, fb, cx, row0 + 2 * p.box_rows);
                     a_slot ^= 1u;
                     if (a_slot == 0) a_par ^= 1u;
                     need_slab = false;
@@ -146,9 +150,11 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (++tap == p.taps) { tap = 0; cx += 32; need_slab = true; }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
+    } else if (warp == 1 || warp == 6) {
+        if (lane == 0 && (warp == 1 || Cfg::ISSUERS == 2)) {
+            // ---------------- MMA issuer(s): warp 1 feeds the first half of the accumulators, warp 6 the second half
+            constexpr int ACC_PER = NACC / Cfg::ISSUERS;
+            const int acc0 = warp == 1 ? 0 : ACC_PER;
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
             const int chunk0 = it_begin / p.taps;
             int tap = it_begin - chunk0 * p.taps;
@@ -181,7 +187,8 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 // exactly as the TMA write did (measured: the descriptor's base-offset field must stay zero).
                 const uint64_t da = smem_desc_k_sw128(slab_addr + a_off);
 #pragma unroll
-                for (int acc = 0; acc < NACC; ++acc) {
+                for (int a = 0; a < ACC_PER; ++a) {
+                    const int acc = acc0 + a;
 #pragma unroll
                     for (int k = 0; k < 4; ++k)
                         umma_tf32(tmem_acc + acc * BN, da + (uint64_t)(acc * (128 * 128 / 16) + 2 * k), db + 2 * k, idesc,
@@ -246,7 +253,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const uint32_t rank = cluster_cta_rank();
 #pragma unroll 1
         for (int acc = 0; acc < NACC; ++acc) {
-            if (warp >= 2 && ok) {
+            if (warp >= 2 && warp <= 5 && ok) {
                 const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16) + acc * BN;
                 tc_fence_after();
 #pragma unroll 1
@@ -259,7 +266,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 tc_fence_before();
             }
             cluster_sync_all();
-            if (warp >= 2 && ok)
+            if (warp >= 2 && warp <= 5 && ok)
                 cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
             cluster_sync_all();      // peers are done with this CTA's shared memory
         }

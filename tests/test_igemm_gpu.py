@@ -116,7 +116,7 @@ HALO_SHAPES = [
 ]
 
 
-@pytest.mark.parametrize("tile", [5, 6, 7, 8, 9, 10, 11, 12])
+@pytest.mark.parametrize("tile", [5, 6, 7, 8, 9, 10, 11, 12, 13, 14, 15])
 @pytest.mark.parametrize("shape", HALO_SHAPES)
 def test_halo_tiles_exact(shape, tile):
     x, w, b = _int_tensors(shape, 1100)
