@@ -107,8 +107,7 @@ int boda_conv_plan_destroy(boda_conv_plan* plan);
 int boda_conv_plan_describe(const boda_conv_plan* plan, char* buf, size_t buf_bytes);
 
 /* Bytes of caller-provided scratch that boda_conv_fwd_planned needs (0 if none).  The scratch holds
- * the re-laid-out input (the "input transformation" that the paper's k1conv and tconv apply, Section 5)
- * and split-reduction partial sums. */
+ * the re-laid-out input (the "input transformation" that the paper's k1conv and tconv apply, Section 5). */
 size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* plan);
 
 /* Kernels one boda_conv_fwd_planned call launches when the filters are bound (1 for DIRECT; 2 for the
@@ -163,8 +162,8 @@ int boda_conv_fwd_host(const float* in_host, const float* filt_host, const float
  * allocates a plan and a workspace the first time it sees a shape; this entry point never does.
  *
  * What it does: the same operation as boda_conv_fwd, always on the tensor-core path (K1CONV for R = S = 1,
- * TCONV otherwise; TF32 operands, fp32 accumulation), with the kernel's scratch - re-laid-out input and
- * filters, split partial sums, split counters - in a device array of BODA_NOALLOC_SCRATCH_BYTES that is
+ * TCONV otherwise; TF32 operands, fp32 accumulation), with the kernel's scratch - the re-laid-out input and
+ * filters and a status word - in a device array of BODA_NOALLOC_SCRATCH_BYTES that is
  * part of the library image.  Every GPU that loads the library holds that array until the process exits.
  * It calls no cudaMalloc / cudaFree and no allocating library routine.  in / filt / bias / out are device
  * pointers owned by the caller, as for boda_conv_fwd.

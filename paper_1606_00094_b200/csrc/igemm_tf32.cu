@@ -869,7 +869,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
 }
 
 // ------------------------------------------------------------------------------------------------
-// The same convolution with every piece of scratch (status word, split counters, re-laid-out filters and
+// The same convolution with every piece of scratch (status word, re-laid-out filters and
 // input, split partial sums) carved out of ONE device region handed in by the caller.  Nothing is
 // allocated here; the region keeps its previous contents, so what must start at zero is cleared first.
 size_t igemm_region_min_bytes(const ConvDims& d)

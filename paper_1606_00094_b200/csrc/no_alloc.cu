@@ -1,6 +1,6 @@
 // boda_conv_fwd_noalloc: the tensor-core convolution for callers that cannot allocate device memory.
 //
-// All scratch of the kernel (re-laid-out input and filters, split partial sums, split counters, status word)
+// All scratch of the kernel (re-laid-out input and filters, status word)
 // lives in one file-scope device array of fixed size.  Every GPU that loads this library holds the array
 // until the process exits.  Host code cannot use the array's name as a device address, so the address is
 // fetched once per device with cudaGetSymbolAddress and handed to the launch code.
