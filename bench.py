@@ -127,6 +127,22 @@ def time_oracle(batch: int, reps: int):
     return wl.stack_flops(batch) / best / 1e9, best, orc.num_threads()
 
 
+def max_over_ranks(values, world: int, device: str):
+    """Each rank passes its own device-measured times; every rank gets the maximum over all ranks."""
+    import torch
+    import torch.distributed as dist
+    t = torch.tensor(list(values), dtype=torch.float64, device=device)
+    if world > 1:
+        dist.all_reduce(t, op=dist.ReduceOp.MAX)
+    return [float(v) for v in t]
+
+
+def whole_job_gflops(flops_per_replica_step: int, world: int, ms_per_step: float) -> float:
+    """Weak scaling over replicas: every rank runs one full step on its own batch, so the job does
+    world x FLOPs in the time of the slowest rank."""
+    return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e9
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -241,13 +257,10 @@ def run_ours(args):
     status = B.boda_query_status()
     assert status == 0, f"device status word {status}"
 
-    t = torch.tensor([total_ms, e2e_total_ms], dtype=torch.float64, device="cuda")
-    if world > 1:
-        dist.all_reduce(t, op=dist.ReduceOp.MAX)
-    total_ms, e2e_total_ms = float(t[0]), float(t[1])
+    total_ms, e2e_total_ms = max_over_ranks([total_ms, e2e_total_ms], world, "cuda")
     ms_per_step = total_ms / args.steps
-    value = world * flops_step / (ms_per_step * 1e-3) / 1e9
-    e2e_value = world * flops_step / (e2e_total_ms / args.steps * 1e-3) / 1e9
+    value = whole_job_gflops(flops_step, world, ms_per_step)
+    e2e_value = whole_job_gflops(flops_step, world, e2e_total_ms / args.steps)
 
     if rank == 0:
         descs = stack.describe()
