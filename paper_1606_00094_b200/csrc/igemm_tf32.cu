@@ -48,6 +48,7 @@ struct IgemmParams {
     const float* bias;
     OutSpec o;                   // output tensor, layout and activation
     int* status;
+    int tx_extra;                // test hook: bytes added to the first stage's expected transfer size of CTA (0,0,0)
 };
 
 
@@ -139,7 +140,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             uint32_t fb = full_bar, eb = empty_bar, adst = smem_a, bdst = smem_b;
             for (int i = 0; i < my_iters; ++i) {
                 if (!mbar_wait(eb, par, &s_abort, p.status, 1)) break;
-                mbar_expect_tx(fb, Cfg::STAGE_BYTES);
+                mbar_expect_tx(fb, Cfg::STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
                 tma_load_im2col_4d(adst, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
                 tma_load_3d(bdst, &map_b, fb, cc * BKC, k0, tap);
                 if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; adst = smem_a; bdst = smem_b; }
@@ -425,6 +426,7 @@ struct IgemmPlan {
     CUtensorMap map_a;
     const void* map_a_base = nullptr;
     // activation layouts on either side (set by igemm_plan_set_io; NCHW by default)
+    int tx_extra = 0;                // test hook (BODA_TEST_TX_MISMATCH): makes one bounded wait of one CTA expire
     bool in_packed = false;          // the input already is this plan's staged layout: skip the staging kernel
     int out_packed = 0, oHp = 0, oWp = 0, oCp = 0;
     // halo kernel only
@@ -656,6 +658,17 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->d = d;
     p->orig = d_in;
     p->s2d = use_s2d;
+    {
+        // Test hooks, off unless the environment asks: a transfer-size mismatch that lets one bounded wait run out,
+        // and a shorter limit for that wait (failure detection is tested without faulting or hanging the GPU).
+        const char* mm = std::getenv("BODA_TEST_TX_MISMATCH");
+        p->tx_extra = (mm && *mm == '1') ? 16 : 0;
+        const char* lim = std::getenv("BODA_WAIT_LIMIT_CYCLES");
+        long long cycles = lim ? std::atoll(lim) : kWaitLimitCycles;
+        if (cycles < 1000000) cycles = 1000000;
+        cudaError_t ce = cudaMemcpyToSymbol(c_wait_limit_cycles, &cycles, sizeof(cycles));
+        if (ce != cudaSuccess) { delete p; return record_cuda_error(ce, "wait limit upload"); }
+    }
     p->variant = variant;
     p->d_status = d_status;
     p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
@@ -821,7 +834,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         hp.S = d.S; hp.taps = d.R * d.S; hp.cchunks = p->Cp / BKC; hp.lead = p->lead;
         hp.nbox = p->nbox; hp.box_rows = p->box_rows; hp.a_slot_bytes = p->a_slot_bytes; hp.b_stages = p->b_stages;
         hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
-        hp.bias = bias; hp.o = make_out_spec(p, out);
+        hp.bias = bias; hp.o = make_out_spec(p, out); hp.tx_extra = p->tx_extra;
         hp.status = p->d_status;
         switch (p->BN * 10 + p->nacc) {
             case 641: return launch_halo<64, 1>(p, hp, stream);
@@ -857,6 +870,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     prm.splits = p->splits;
     prm.bias = bias;
     prm.o = make_out_spec(p, out);
+    prm.tx_extra = p->tx_extra;
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: return launch_bn<64>(p, prm, stream);
@@ -950,6 +964,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     prm.splits = p->splits;
     prm.bias = bias;
     prm.o = make_out_spec(p, out);
+    prm.tx_extra = p->tx_extra;
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: rc = launch_bn<64>(p, prm, stream); break;

@@ -12,6 +12,8 @@ namespace boda {
 namespace tc {
 
 constexpr long long kWaitLimitCycles = 4000000000ll;
+// The limit actually used (SM cycles).  Tests shorten it through the environment variable BODA_WAIT_LIMIT_CYCLES.
+__constant__ long long c_wait_limit_cycles = kWaitLimitCycles;
 
 __device__ __forceinline__ uint32_t smem_u32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
 
@@ -46,7 +48,7 @@ __device__ __noinline__ bool mbar_wait_slow(uint32_t bar, uint32_t parity, volat
             if (*abort_flag) return false;
             if (spin == 256u) {
                 t0 = clock64();
-            } else if (clock64() - t0 > kWaitLimitCycles) {
+            } else if (clock64() - t0 > c_wait_limit_cycles) {
                 *abort_flag = 1;
                 if (atomicCAS(status, 0, (int)BODA_ERR_DEVICE_TIMEOUT) == 0) {
                     status[1] = KERNEL_ID_IGEMM;
@@ -73,7 +75,7 @@ __device__ __noinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, vo
     for (;;) {
         if (mbar_try_wait(bar, parity)) return true;
         if (*abort_flag) return false;
-        if (clock64() - t0 > kWaitLimitCycles) {
+        if (clock64() - t0 > c_wait_limit_cycles) {
             *abort_flag = 1;
             if (atomicCAS(status, 0, (int)BODA_ERR_DEVICE_TIMEOUT) == 0) {
                 status[1] = KERNEL_ID_IGEMM;

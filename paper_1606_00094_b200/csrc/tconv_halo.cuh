@@ -43,6 +43,7 @@ struct HaloParams {
     const float* bias;
     OutSpec o;                   // output tensor, layout and activation
     int* status;
+    int tx_extra;                // test hook: bytes added to the first stage's expected transfer size of CTA (0,0,0)
 };
 
 // output location of flat position f = (n*Hp + p)*Wp + q; positions with p >= P or q >= Q are dropped
@@ -143,7 +144,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     need_slab = false;
                 }
                 if (!mbar_wait(be, b_par, &s_abort, p.status, 12)) break;
-                mbar_expect_tx(bf, Cfg::B_STAGE_BYTES);
+                mbar_expect_tx(bf, Cfg::B_STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
                 tma_load_3d(bdst, &map_b, bf, cx, k0, tap);
                 if (++b_stage == (uint32_t)p.b_stages) { b_stage = 0; b_par ^= 1u; bf = b_full; be = b_empty; bdst = smem_b; }
                 else { bf += 8; be += 8; bdst += Cfg::B_STAGE_BYTES; }
