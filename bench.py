@@ -60,7 +60,7 @@ class ClockSampler:
         try:
             self.proc = subprocess.Popen(
                 ["nvidia-smi", f"--id={self.gpu_index}", f"--query-gpu={self.FIELDS}", "--format=csv,noheader,nounits",
-                 "-lms", "100"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+                 "-lms", "20"], stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
         except OSError:
             self.proc = None
             return
@@ -143,6 +143,38 @@ def whole_job_gflops(flops_per_replica_step: int, world: int, ms_per_step: float
     return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e9
 
 
+def single_layer_configs(B, wl, torch, peaks):
+    """The four single-layer configurations (parity-test cases; reported for context): NCHW in and out through
+    boda_conv_fwd_planned, input staging included, 20 back-to-back launches per event pair (L2-warm)."""
+    out = []
+    for cid in (1, 2, 3, 4):
+        cfg = wl.CONFIGS[cid]
+        s = cfg.shape
+        x, w, b = (torch.from_numpy(t).cuda() for t in cfg.tensors())
+        plan = B.ConvPlan(s.as_tuple(), tune=1)
+        y = torch.empty(plan.out_shape, dtype=torch.float32, device="cuda")
+        plan.bind_filters(w)
+        for _ in range(5):
+            plan(x, w, b, out=y)
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        reps = 20
+        e0.record()
+        for _ in range(reps):
+            plan(x, w, b, out=y)
+        e1.record()
+        torch.cuda.synchronize()
+        us = e0.elapsed_time(e1) / reps * 1e3
+        desc = plan.describe()
+        plan.close()
+        tf = s.flops / us / 1e6
+        out.append({"config": cid, "name": cfg.name, "us_per_call": round(us, 2), "gflops": round(tf * 1e3, 1),
+                    "algorithmic_gbs": round(s.min_bytes / us / 1e3, 1),
+                    "frac_of_hbm_peak": round(s.min_bytes / us / 1e3 / peaks["hbm_gbs"], 4),
+                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4), "plan": desc})
+    return out
+
+
 def run_reference(args):
     rank = int(os.environ.get("RANK", "0"))
     if rank != 0:
@@ -204,6 +236,10 @@ def run_ours(args):
     flops_step = wl.stack_flops(BATCH)
     n_ops = len(ops)
 
+    # clocks and throttle reasons are sampled from the warm-up to the end of the last timed region
+    sampler = ClockSampler(local_rank)
+    sampler.start()
+    time.sleep(0.3)                                     # let nvidia-smi come up before the GPU work starts
     for _ in range(max(args.warmup, 3)):
         flush.zero_()
         stack.forward(x_dev)
@@ -211,8 +247,6 @@ def run_ours(args):
     assert B.boda_query_status() == 0, "device status word set during warm-up"
 
     # ---------------- timed region 1: inputs resident in HBM; one CUDA-graph launch per step
-    sampler = ClockSampler(local_rank)
-    sampler.start()
     launches0 = B.boda_kernel_launch_count()
     barrier()
     step_ev = []
@@ -238,6 +272,23 @@ def run_ours(args):
     barrier()
     layer_ms = [sum(ev[3 * i].elapsed_time(ev[3 * i + 2]) for ev in layer_ev) / args.steps for i in range(n_ops)]
     main_ms = [sum(ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for ev in layer_ev) / args.steps for i in range(n_ops)]
+
+    # ---------------- the dominant kernel on its own: the conv layer whose main kernel is slowest, re-launched in
+    # place on the activations of the last step, 20 launches back to back between two events (so that host launch
+    # gaps do not count), repeated `steps` times
+    conv_ops = [i for i, op in enumerate(ops) if op.kind == "conv"]
+    dom = max(conv_ops, key=lambda i: main_ms[i])
+    dom_reps = 20
+    dom_ev = []
+    for _ in range(args.steps):
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record()
+        for _ in range(dom_reps):
+            stack.run_op(dom, x_dev)
+        e1.record()
+        dom_ev.append((e0, e1))
+    barrier()
+    dom_ms = sum(a.elapsed_time(b) for a, b in dom_ev) / (args.steps * dom_reps)
 
     # ---------------- timed region 2: end to end from pinned host buffers
     for _ in range(2):
@@ -273,10 +324,8 @@ def run_ours(args):
                                "gflops": round(gf, 1), "plan": descs[i]})
             else:
                 layers.append({"op": "pool", "ms": round(layer_ms[i], 5)})
-        # dominant kernel: the main kernel of the conv layer that takes the most time in the step
-        conv_idx = [i for i, op in enumerate(ops) if op.kind == "conv"]
-        dom = max(conv_idx, key=lambda i: main_ms[i])
-        dom_tf = ops[dom].shape.flops / (main_ms[dom] * 1e-3) / 1e12
+        # dominant kernel: the main kernel of the conv layer that takes the most time in the step (timed above)
+        dom_tf = ops[dom].shape.flops / (dom_ms * 1e-3) / 1e12
         tensor_path = "variant=direct" not in descs[dom]
         if tensor_path:
             peak = 0.5 * peaks["bf16_tflops"]      # dense TF32 = half the bf16 rate; measured bf16 burst
@@ -290,7 +339,9 @@ def run_ours(args):
             traffic = json.load(open(tpath)).get("dram_bytes_per_launch")
         roofline = {"bound": bound, "achieved": round(dom_tf, 3), "peak": round(peak, 2), "unit": "TFLOP/s",
                     "frac": round(dom_tf / peak, 4), "traffic": traffic, "kernel": layers[dom]["op"] + ": " + descs[dom],
-                    "peak_source": peak_note, "launch_ms": round(main_ms[dom], 5)}
+                    "peak_source": peak_note, "launch_ms": round(dom_ms, 5),
+                    "timing": f"{dom_reps} back-to-back launches of that layer in place per event pair, L2-warm as inside the step"}
+        per_config = single_layer_configs(B, wl, torch, peaks)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -307,6 +358,7 @@ def run_ours(args):
             "cpu_baseline": {"value": round(cpu_v, 2) if cpu_v else None, "unit": UNIT, "cores": cpu_threads,
                              "kind": "oracle", "sample": f"the whole batch-{BATCH} stack, best of 2 ({cpu_t:.2f} s)" if cpu_t else "skipped"},
             "layers": layers,
+            "single_layer_configs": per_config,
             "frac_of_tf32_peak_whole_step": round(value / 1e3 / (0.5 * peaks["bf16_tflops"]) / world, 4),
         }
         print(json.dumps(line))

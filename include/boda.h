@@ -242,6 +242,9 @@ int boda_stack_fwd(boda_stack* stack, const float* in, float* out, void* stream)
  * 3 * n_ops cudaEvent_t handles; for op i the library records events[3i] before its first kernel, events[3i+1]
  * between operand staging and the main kernel, and events[3i+2] after its last kernel (per-layer timing). */
 int boda_stack_fwd_eager(boda_stack* stack, const float* in, float* out, void* stream, void** events);
+/* Runs op `op_index` alone on the activations that the last forward pass left in the stack (for timing one layer
+ * in place).  `in` is read only by op 0 and `out` written only by the last op; pass NULL otherwise. */
+int boda_stack_run_op(boda_stack* stack, int op_index, const float* in, float* out, void* stream);
 /* Forward pass with HOST buffers: copies `in_host` to the device, runs boda_stack_fwd, copies the result into
  * `out_host` and synchronises `stream`.  Pinned host memory makes the copies asynchronous. */
 int boda_stack_fwd_host(boda_stack* stack, const float* in_host, float* out_host, void* stream);

@@ -95,6 +95,8 @@ _lib.boda_stack_fwd.argtypes = [_vp, _vp, _vp, _vp]
 _lib.boda_stack_fwd.restype = _i
 _lib.boda_stack_fwd_eager.argtypes = [_vp, _vp, _vp, _vp, ctypes.POINTER(_vp)]
 _lib.boda_stack_fwd_eager.restype = _i
+_lib.boda_stack_run_op.argtypes = [_vp, _i, _vp, _vp, _vp]
+_lib.boda_stack_run_op.restype = _i
 _lib.boda_stack_fwd_host.argtypes = [_vp, _vp, _vp, _vp]
 _lib.boda_stack_fwd_host.restype = _i
 _lib.boda_query_status.argtypes = [_vp, ctypes.POINTER(_i)]
@@ -286,6 +288,10 @@ def boda_stack_fwd_eager(stack: int, inp, out, stream=None, events=None) -> None
             handles.append(e.cuda_event)
         arr = (_vp * len(handles))(*handles)
     _check(_lib.boda_stack_fwd_eager(stack, _addr(inp), _addr(out), _stream(stream), arr), "boda_stack_fwd_eager")
+
+
+def boda_stack_run_op(stack: int, op_index: int, inp=None, out=None, stream=None) -> None:
+    _check(_lib.boda_stack_run_op(stack, op_index, _addr(inp), _addr(out), _stream(stream)), "boda_stack_run_op")
 
 
 def boda_stack_fwd_host(stack: int, inp_host, out_host, stream=None) -> None:

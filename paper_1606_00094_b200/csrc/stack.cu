@@ -272,6 +272,25 @@ int boda_stack_fwd_eager(boda_stack* s, const float* in, float* out, void* strea
     return run_ops(s, in, out, (cudaStream_t)stream, (cudaEvent_t*)events);
 }
 
+int boda_stack_run_op(boda_stack* s, int op_index, const float* in, float* out, void* stream)
+{
+    if (!s || op_index < 0 || op_index >= (int)s->ops.size()) return BODA_ERR_INVALID_ARG;
+    const int n = (int)s->ops.size();
+    boda_stack::Op& op = s->ops[op_index];
+    const float* src = op_index == 0 ? in : s->ops[op_index - 1].out;
+    float* dst = op_index == n - 1 ? out : op.out;
+    if (!src || !dst) return BODA_ERR_INVALID_ARG;
+    cudaStream_t st = (cudaStream_t)stream;
+    if (op.kind == BODA_STACK_CONV) {
+        if (!op.filt) return BODA_ERR_INVALID_ARG;
+        return conv_fwd_planned_ex(op.plan, src, op.filt, op.bias, dst, s->workspace, st, nullptr);
+    }
+    if (op.in_packed)
+        return maxpool_packed_launch(src, dst, op.N, op.C, op.H, op.W, op.iHp, op.iWp, op.iCp, op.ksz, op.stride,
+                                     op.out_packed ? 1 : 0, op.oHp, op.oWp, op.oCp, st);
+    return maxpool_launch(src, dst, op.N, op.C, op.H, op.W, op.ksz, op.stride, st);
+}
+
 int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, void* stream)
 {
     if (!s || !in_host || !out_host) return BODA_ERR_INVALID_ARG;

@@ -69,6 +69,10 @@ class ConvStack:
         B.boda_stack_fwd_eager(self.handle, x, out, None, events)
         return out
 
+    def run_op(self, i: int, x: Optional[torch.Tensor] = None) -> None:
+        """Re-runs op i alone on the activations of the last forward pass (timing aid)."""
+        B.boda_stack_run_op(self.handle, i, x, self.out)
+
     def forward_host(self, x_host: torch.Tensor, out_host: torch.Tensor) -> None:
         """Host buffers in and out (pinned for asynchronous copies); returns after the result has landed."""
         B.boda_stack_fwd_host(self.handle, x_host, out_host)
