@@ -35,7 +35,7 @@ namespace {
 constexpr int BM = 128;          // pixels per CTA tile (UMMA M)
 constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of fp32)
 constexpr int A_STAGE_BYTES = BM * BKC * 4;
-constexpr int kIgemmThreads = 192;
+constexpr int kIgemmThreads = 224;   // warp 0 producer, 1 and 6 MMA issuers, 2..5 epilogue
 
 using namespace tc;
 
@@ -55,8 +55,19 @@ struct IgemmParams {
 template <int BN> struct TileCfg {
     static constexpr int B_STAGE_BYTES = BN * BKC * 4;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
+#ifndef BODA_IGEMM_DUAL_ISSUE_MAX_BN
+#define BODA_IGEMM_DUAL_ISSUE_MAX_BN 192
+#endif
+    // MMA issuers: two for the narrower tiles, where one thread's issue cost (about 530 clocks per stage) exceeds
+    // the MMA work of a stage (2*BN clocks); one for BN = 256, which is bound by the tensor pipe either way.
+    // Each issuer OWNS a contiguous set of ring stages ([0, SPLIT) and [SPLIT, STAGES)) and walks it in order, so
+    // every barrier has one waiter and a wait can never alias a phase that its issuer has not seen yet.
+    static constexpr int ISSUERS = BN <= BODA_IGEMM_DUAL_ISSUE_MAX_BN ? 2 : 1;
     static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
-    static constexpr int TMEM_COLS = BN <= 32 ? 32 : BN <= 64 ? 64 : BN <= 128 ? 128 : 256;
+    static constexpr int SPLIT = ISSUERS == 2 ? (STAGES + 1) / 2 : STAGES;   // first stage of the second issuer
+    static_assert(STAGES >= 2, "both issuers need a stage");
+    static constexpr int ACC_COLS = ISSUERS * BN;                                         // one accumulator per issuer
+    static constexpr int TMEM_COLS = ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -106,7 +117,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
-        mbar_init(accum_bar, 1);
+        mbar_init(accum_bar, Cfg::ISSUERS);           // one arrival per MMA issuer
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
@@ -148,29 +159,37 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (++cc == p.cchunks) { cc = 0; ++tap; if (++s == p.S) { s = 0; ++r; } }
             }
         }
-    } else if (warp == 1) {
-        if (lane == 0) {
-            // ---------------- MMA issuer
+    } else if (warp == 1 || warp == 6) {
+        if (lane == 0 && (warp == 1 || Cfg::ISSUERS == 2)) {
+            const int me = warp == 1 ? 0 : 1;
+            // ---------------- MMA issuers: warp 1 owns ring stages [0, SPLIT), warp 6 the rest.  One thread needs
+            // about 530 clocks per stage (barrier hand-shake plus four MMA issues); two threads share that, so the
+            // tensor pipe itself becomes the limit for BN >= 128.  Each issuer accumulates into its own TMEM
+            // accumulator (columns [0, BN) and [BN, 2*BN)); the epilogue adds the two, so the summation order - and
+            // with it every output bit - is the same in every run.
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
+            const int lo = me == 0 ? 0 : Cfg::SPLIT, hi = me == 0 ? Cfg::SPLIT : STAGES;
             bool ok = true;
-            uint32_t stage = 0, par = 0;
-            uint32_t fb = full_bar, eb = empty_bar;
+            uint32_t par = 0;
+            int stage = lo;
             const uint64_t da0 = smem_desc_k_sw128(smem_a), db0 = smem_desc_k_sw128(smem_b);
-            uint64_t da = da0, db = db0;
+            const uint32_t my_acc = tmem_acc + (uint32_t)(me * BN);
             uint32_t accumulate = 0;
-            for (int i = 0; i < my_iters; ++i) {
-                ok = mbar_wait(fb, par, &s_abort, p.status, 2);
+            for (int i = lo; i < my_iters;) {
+                ok = mbar_wait(full_bar + 8 * stage, par, &s_abort, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
+                const uint64_t da = da0 + (uint64_t)stage * (A_STAGE_BYTES >> 4);
+                const uint64_t db = db0 + (uint64_t)stage * (Cfg::B_STAGE_BYTES >> 4);
 #pragma unroll
                 for (int k = 0; k < BKC / 8; ++k)       // 8 TF32 values = 32 bytes = 2 descriptor units per step
-                    umma_tf32(tmem_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
+                    umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
                 accumulate = 1u;
-                tc_commit(eb);                          // frees the stage once these MMAs have read it
-                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; da = da0; db = db0; }
-                else { fb += 8; eb += 8; da += (uint64_t)(A_STAGE_BYTES >> 4); db += (uint64_t)(Cfg::B_STAGE_BYTES >> 4); }
+                tc_commit(empty_bar + 8 * stage);       // frees the stage once these MMAs have read it
+                ++stage; ++i;
+                if (stage == hi) { stage = lo; i += STAGES - (hi - lo); par ^= 1u; }
             }
-            tc_commit(accum_bar);                       // accumulator complete (or: everything issued so far has drained)
+            tc_commit(accum_bar);                       // this issuer's MMAs have drained
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
         }
     } else {
@@ -189,17 +208,19 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+        const bool two_acc = Cfg::ISSUERS == 2 && my_iters > Cfg::SPLIT;   // a shorter reduction never reaches the second issuer's stages
         if (ok && p.splits == 1) {
             const RowDst d = igemm_row_dst(p, m);
 #pragma unroll 1
             for (int j0 = 0; j0 < BN; j0 += 32) {
-                uint32_t v[32];
+                uint32_t v[32], v2[32];
                 tmem_ld_32cols(trow + j0, v);
+                if (two_acc) tmem_ld_32cols(trow + BN + j0, v2);
                 tmem_ld_wait();
                 float y[32];
 #pragma unroll
                 for (int j = 0; j < 32; ++j) {
-                    y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
+                    y[j] = __uint_as_float(v[j]) + (two_acc ? __uint_as_float(v2[j]) : 0.f) + s_bias[j0 + j];
                     if (p.o.relu) y[j] = fmaxf(y[j], 0.f);
                 }
                 store_row32(p.o, d, k0 + j0, y, smem_base + (uint32_t)(warp & 3) * 4224u);
@@ -209,9 +230,14 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             // buffers are idle now); the cluster-wide sum follows below.
 #pragma unroll 1
             for (int j0 = 0; j0 < BN; j0 += 32) {
-                uint32_t v[32];
+                uint32_t v[32], v2[32];
                 tmem_ld_32cols(trow + j0, v);
+                if (two_acc) tmem_ld_32cols(trow + BN + j0, v2);
                 tmem_ld_wait();
+                if (two_acc) {
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+                }
                 stash_row32<BN>(smem_base, row, j0, v);
             }
         }
@@ -222,7 +248,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         // split reduction, step 2: the CTAs of one output tile form a cluster (one per split); after the
         // cluster barrier each of them sums its share of the channels over all peers' shared memory and stores it.
         cluster_sync_all();
-        if (warp >= 2 && s_abort == 0) {
+        if (warp >= 2 && warp <= 5 && s_abort == 0) {
             const int row = (warp & 3) * 32 + lane;
             cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
         }
