@@ -273,22 +273,27 @@ def run_ours(args):
     layer_ms = [sum(ev[3 * i].elapsed_time(ev[3 * i + 2]) for ev in layer_ev) / args.steps for i in range(n_ops)]
     main_ms = [sum(ev[3 * i + 1].elapsed_time(ev[3 * i + 2]) for ev in layer_ev) / args.steps for i in range(n_ops)]
 
-    # ---------------- the dominant kernel on its own: the conv layer whose main kernel is slowest, re-launched in
-    # place on the activations of the last step, 20 launches back to back between two events (so that host launch
-    # gaps do not count), repeated `steps` times
+    # ---------------- every op on its own, and with it the dominant kernel: op i re-launched in place on the
+    # activations of the last step, 20 launches back to back captured in one CUDA graph (so that neither host launch
+    # cost nor gaps count), the graph replayed several times between events
     dom_reps = 20
     inplace_ms = []
     for i in range(n_ops):
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g):
+            for _ in range(dom_reps):
+                stack.run_op(i, x_dev)
+        g.replay()
         evs = []
         for _ in range(max(3, args.steps // 4)):
             e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
             e0.record()
-            for _ in range(dom_reps):
-                stack.run_op(i, x_dev)
+            g.replay()
             e1.record()
             evs.append((e0, e1))
         barrier()
         inplace_ms.append(sum(a.elapsed_time(b) for a, b in evs) / (len(evs) * dom_reps))
+        del g
     conv_ops = [i for i, op in enumerate(ops) if op.kind == "conv"]
     descs_all = stack.describe()
     # the dominant KERNEL: among the conv ops that are a single kernel launch (input already staged, or DIRECT)

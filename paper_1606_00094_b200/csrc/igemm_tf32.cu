@@ -350,7 +350,14 @@ pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int 
         const int y = yb * t + dy - pad;
         const bool inside = y >= 0 && y < H;
         const float* src = in + (((size_t)n * C + c) * H + (inside ? y : 0)) * W;
-        for (int x = lane; x < W; x += 32) sm_rows[row * W + x] = inside ? __ldg(src + x) : 0.f;
+        for (int x0 = lane; x0 < W; x0 += 256) {                 // eight loads in flight per lane
+            float v[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j) v[j] = (inside && x0 + 32 * j < W) ? __ldg(src + x0 + 32 * j) : 0.f;
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                if (x0 + 32 * j < W) sm_rows[row * W + x0 + 32 * j] = v[j];
+        }
     }
     __syncthreads();
     // write the row of blocks: one warp per block xb, lanes along the packed channels (contiguous 128-byte stores)
