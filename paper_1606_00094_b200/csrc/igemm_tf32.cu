@@ -35,9 +35,10 @@ namespace {
 constexpr int BM = 128;          // pixels per CTA tile (UMMA M)
 constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of fp32)
 constexpr int A_STAGE_BYTES = BM * BKC * 4;
-constexpr int kIgemmThreads = 224;   // warp 0 producer, 1 and 6 MMA issuers, 2..5 epilogue
+constexpr int kIgemmThreads = 352;   // warp 0 producer, 1 and 6 MMA issuers, 2..5 and 7..10 epilogue
 
 using namespace tc;
+
 
 struct IgemmParams {
     int M, stride, pad, S;
@@ -101,9 +102,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t full_bar = bars;                    // STAGES x 8 bytes
     const uint32_t empty_bar = bars + 8 * STAGES;
     const uint32_t accum_bar = bars + 16 * STAGES;
+    const uint32_t recv_bar = accum_bar + 8;           // split reduction: bytes pushed by the cluster peers
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ float s_bias[BN];
+    __shared__ __align__(16) float s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -112,12 +114,14 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const int it_begin = blockIdx.z * p.iters_per_split;
     const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
     const int my_iters = it_end - it_begin;
+    const bool exchange = split_exchange_fits(BN, p.splits, STAGES * Cfg::STAGE_BYTES);   // the same in every CTA
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
         mbar_init(accum_bar, Cfg::ISSUERS);           // one arrival per MMA issuer
+        mbar_init(recv_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
@@ -193,66 +197,147 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
         }
     } else {
-        // ---------------- epilogue: 4 warps, warp w reads TMEM lanes 32*(w%4) .. +31
+        // ---------------- epilogue: 8 warps.  Warp w may read TMEM lanes 32*(w%4) .. +31 only, so warps 2..5 and
+        // 7..10 pair up on the same 32 rows and share the columns in chunks of 32: group 0 takes the even chunks of
+        // a piece of work, group 1 the odd ones.  (One warp per scheduler cannot hide its own instruction latency:
+        // four warps needed about 650 clocks per chunk.)
         const int quarter = warp & 3;
+        const int group = warp >= 7 ? 1 : 0;
         const int row = quarter * 32 + lane;
         const int m = m0 + row;
+        const int etid = threadIdx.x - (group ? 96 : 64);                  // 0 .. 255 over the epilogue threads
         // bias of this tile's channels into shared memory while the main loop runs (0 where there is none)
-        for (int j = threadIdx.x - 64; j < BN; j += 128)
+        for (int j = etid; j < BN; j += 256)
             s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
         if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 4);   // one poller per warp
         __syncwarp();
-        // All 128 epilogue threads meet here whatever their wait returned, then take one common decision:
+        // All epilogue threads meet here whatever their wait returned, then take one common decision:
         // a failed wait has raised the abort flag before returning.
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         const bool two_acc = Cfg::ISSUERS == 2 && my_iters > Cfg::SPLIT;   // a shorter reduction never reaches the second issuer's stages
-        if (ok && p.splits == 1) {
-            const RowDst d = igemm_row_dst(p, m);
-#pragma unroll 1
-            for (int j0 = 0; j0 < BN; j0 += 32) {
-                uint32_t v[32], v2[32];
-                tmem_ld_32cols(trow + j0, v);
-                if (two_acc) tmem_ld_32cols(trow + BN + j0, v2);
+        // 32 accumulator columns of this thread's row (the sum of the two issuers' accumulators)
+        auto load32 = [&](int j0, uint32_t (&v)[32]) {
+            tmem_ld_32cols(trow + j0, v);
+            if (two_acc) {
+                uint32_t v2[32];
+                tmem_ld_32cols(trow + BN + j0, v2);
                 tmem_ld_wait();
-                float y[32];
 #pragma unroll
-                for (int j = 0; j < 32; ++j) {
-                    y[j] = __uint_as_float(v[j]) + (two_acc ? __uint_as_float(v2[j]) : 0.f) + s_bias[j0 + j];
-                    if (p.o.relu) y[j] = fmaxf(y[j], 0.f);
+                for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
+            } else {
+                tmem_ld_wait();
+            }
+        };
+        if (p.splits == 1) {
+            if (ok) {
+                const RowDst d = igemm_row_dst(p, m);
+                const uint32_t row_addr = smem_base + (uint32_t)row * out_tile_row_bytes<BN>();   // the stage buffers are idle now
+                // group 0 takes the first half of the row's chunks, group 1 the second; in the staged layout each
+                // half row leaves as one bulk copy as soon as its thread has written it
+                constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
+                const int c_begin = group ? HALF : 0, c_end = group ? NCH : HALF;
+#pragma unroll 1
+                for (int c = c_begin; c < c_end; ++c) {
+                    uint32_t v[32];
+                    load32(32 * c, v);
+                    float y[32];
+                    bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
+                    if (p.o.packed) out_tile_put32(row_addr, 32 * c, y);
+                    else store_row32(p.o, d, k0 + 32 * c, y, 0u);
                 }
-                store_row32(p.o, d, k0 + j0, y, smem_base + (uint32_t)(warp & 3) * 4224u);
+                if (p.o.packed) {
+                    fence_proxy_async_smem();
+                    out_tile_store_row(p.o, d, k0 + 32 * c_begin, 32 * (c_end - c_begin), row_addr + 128u * (uint32_t)c_begin);
+                    bulk_commit();
+                    bulk_wait_all();
+                }
+            }
+        } else if (exchange) {
+            // split reduction by exchange, see split_share(): partial sums of the channels other CTAs own go into
+            // send blocks while the cluster barrier (every CTA's main loop has ended, its stage buffers are free)
+            // completes; then one bulk copy per peer, and the owner adds what it received to its own accumulator.
+            cluster_arrive();
+            const int rank = (int)cluster_cta_rank();
+            const int per = split_share(BN, p.splits);
+            const int my_w = split_width(BN, per, rank);
+            const uint32_t recv_base = smem_base + 512u * (uint32_t)(per * (p.splits - 1));
+            if (ok) {
+                if (threadIdx.x == 64 && my_w > 0) mbar_expect_tx(recv_bar, 512u * (uint32_t)(my_w * (p.splits - 1)));
+                int turn = 0;
+#pragma unroll 1
+                for (int dst = 0; dst < p.splits; ++dst) {
+                    const int wd = split_width(BN, per, dst);
+                    if (dst == rank || wd == 0) continue;
+                    const uint32_t block = smem_base + 512u * (uint32_t)(per * (dst < rank ? dst : dst - 1));
+#pragma unroll 1
+                    for (int c0 = 0; c0 < wd; c0 += 32, ++turn) {
+                        if ((turn & 1) != group) continue;
+                        uint32_t v[32];
+                        load32(dst * per + c0, v);
+                        xchg_put32(block, wd, row, c0, v);
+                    }
+                }
+                fence_proxy_async_smem();
+            }
+            asm volatile("bar.sync 1, 256;" ::: "memory");
+            cluster_wait();
+            if (threadIdx.x == 64 && s_abort == 0) {
+                for (int dst = 0; dst < p.splits; ++dst) {
+                    const int wd = split_width(BN, per, dst);
+                    if (dst == rank || wd == 0) continue;
+                    const uint32_t block = smem_base + 512u * (uint32_t)(per * (dst < rank ? dst : dst - 1));
+                    const uint32_t slot = smem_base + 512u * (uint32_t)(per * (p.splits - 1))
+                                        + 512u * (uint32_t)(wd * (rank < dst ? rank : rank - 1));
+                    bulk_push_cluster(map_to_cta(slot, (uint32_t)dst), block, 512u * (uint32_t)wd, map_to_cta(recv_bar, (uint32_t)dst));
+                }
+            }
+            if (s_abort == 0 && my_w > 0 && mbar_wait(recv_bar, 0, &s_abort, p.status, 5)) {
+                const RowDst d = igemm_row_dst(p, m);
+#pragma unroll 1
+                for (int c0 = 32 * group; c0 < my_w; c0 += 64) {
+                    uint32_t v[32];
+                    load32(rank * per + c0, v);
+                    float y[32];
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(v[j]);
+                    for (int sl = 0; sl < p.splits - 1; ++sl) xchg_add32(recv_base + 512u * (uint32_t)(my_w * sl), my_w, row, c0, y);
+#pragma unroll
+                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
+                    bias_relu32(v, s_bias + rank * per + c0, p.o.relu != 0, y);
+                    store_row32(p.o, d, k0 + rank * per + c0, y, 0u);
+                }
             }
         } else if (ok) {
-            // split reduction, step 1: park this CTA's partial accumulator in its own shared memory (the stage
-            // buffers are idle now); the cluster-wide sum follows below.
+            // split reduction through remote reads (the exchange blocks do not fit), step 1: park this CTA's partial
+            // accumulator in its own shared memory; the cluster-wide sum follows below.
 #pragma unroll 1
-            for (int j0 = 0; j0 < BN; j0 += 32) {
-                uint32_t v[32], v2[32];
-                tmem_ld_32cols(trow + j0, v);
-                if (two_acc) tmem_ld_32cols(trow + BN + j0, v2);
-                tmem_ld_wait();
-                if (two_acc) {
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(__uint_as_float(v[j]) + __uint_as_float(v2[j]));
-                }
+            for (int j0 = 32 * group; j0 < BN; j0 += 64) {
+                uint32_t v[32];
+                load32(j0, v);
                 stash_row32<BN>(smem_base, row, j0, v);
             }
         }
         tc_fence_before();
     }
+    if (exchange && (warp < 2 || warp == 6)) {      // the other roles' half of the first cluster barrier
+        cluster_arrive();
+        cluster_wait();
+    }
     __syncthreads();
     if (p.splits > 1) {
-        // split reduction, step 2: the CTAs of one output tile form a cluster (one per split); after the
-        // cluster barrier each of them sums its share of the channels over all peers' shared memory and stores it.
-        cluster_sync_all();
-        if (warp >= 2 && warp <= 5 && s_abort == 0) {
-            const int row = (warp & 3) * 32 + lane;
-            cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
+        if (!exchange) {
+            // step 2: after the cluster barrier each CTA sums its share of the channels over all peers' shared
+            // memory and stores it.
+            cluster_sync_all();
+            if (warp >= 2 && warp <= 5 && s_abort == 0) {
+                const int row = (warp & 3) * 32 + lane;
+                cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias, 0u);
+            }
         }
-        cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
+        cluster_sync_all();          // nobody leaves while a peer may still read or write its shared memory
     }
     if (warp == 1) {
         __syncwarp();

@@ -207,11 +207,59 @@ __device__ __forceinline__ void st_shared_v4(uint32_t addr, float a, float b, fl
 {
     asm volatile("st.shared.v4.f32 [%0], {%1, %2, %3, %4};" :: "r"(addr), "f"(a), "f"(b), "f"(c), "f"(d) : "memory");
 }
+__device__ __forceinline__ float4 ld_shared_v4(uint32_t addr)
+{
+    float4 v;
+    asm volatile("ld.shared.v4.f32 {%0, %1, %2, %3}, [%4];" : "=f"(v.x), "=f"(v.y), "=f"(v.z), "=f"(v.w) : "r"(addr) : "memory");
+    return v;
+}
+// the two halves of a cluster barrier: work placed between them overlaps the wait for the slowest CTA
+__device__ __forceinline__ void cluster_arrive() { asm volatile("barrier.cluster.arrive.release;" ::: "memory"); }
+__device__ __forceinline__ void cluster_wait() { asm volatile("barrier.cluster.wait.acquire;" ::: "memory"); }
+
+// ---- bulk copies out of shared memory (asynchronous proxy).  Addresses and sizes are multiples of 16 bytes.
+// Writes made with ordinary stores become visible to the copy engine after this fence.
+__device__ __forceinline__ void fence_proxy_async_smem() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// shared memory of this CTA -> global memory; completion is tracked by the thread's bulk group
+__device__ __forceinline__ void bulk_store_global(void* gdst, uint32_t smem_src, uint32_t bytes)
+{
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+// shared memory of this CTA -> shared memory of a CTA of the cluster (`dst` and `bar` are cluster addresses from
+// map_to_cta); the bytes are counted on the destination CTA's mbarrier `bar`
+__device__ __forceinline__ void bulk_push_cluster(uint32_t dst, uint32_t smem_src, uint32_t bytes, uint32_t bar)
+{
+    asm volatile("cp.async.bulk.shared::cluster.shared::cta.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 :: "r"(dst), "r"(smem_src), "r"(bytes), "r"(bar) : "memory");
+}
+
 __device__ __forceinline__ float round_to_tf32(float x)
 {
     uint32_t r;
     asm("cvt.rna.tf32.f32 %0, %1;" : "=r"(r) : "f"(x));
     return __uint_as_float(r);
+}
+
+// y[0..31] = acc[0..31] + bias[0..31], then ReLU if asked.  The bias (shared memory, 16-byte aligned, the same
+// address in every lane) is read four values per load: a broadcast load costs about seven issue slots of the
+// shared-memory pipe whatever its width, and one per element was a third of the epilogue's time.
+__device__ __forceinline__ void bias_relu32(const uint32_t (&v)[32], const float* bias32, bool relu, float (&y)[32])
+{
+    const float4* b4 = reinterpret_cast<const float4*>(bias32);
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const float4 b = b4[g];
+        y[4 * g] = __uint_as_float(v[4 * g]) + b.x;
+        y[4 * g + 1] = __uint_as_float(v[4 * g + 1]) + b.y;
+        y[4 * g + 2] = __uint_as_float(v[4 * g + 2]) + b.z;
+        y[4 * g + 3] = __uint_as_float(v[4 * g + 3]) + b.w;
+    }
+    if (relu) {
+#pragma unroll
+        for (int j = 0; j < 32; ++j) y[j] = fmaxf(y[j], 0.f);
+    }
 }
 
 // ---- where a tensor-core kernel writes its output tile (fused bias + ReLU epilogue, Section 2 of the paper)
@@ -305,12 +353,65 @@ __device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int row, ui
                 for (int j = 0; j < 32; ++j) y[j] += x[j];
             }
         }
+        {
+            uint32_t v[32];
 #pragma unroll
-        for (int j = 0; j < 32; ++j) {
-            y[j] += s_bias[c0 + j];
-            if (o.relu) y[j] = fmaxf(y[j], 0.f);
+            for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
+            bias_relu32(v, s_bias + c0, o.relu != 0, y);
         }
         store_row32(o, d, k0 + c0, y, tile);
+    }
+}
+
+// ---- staged-layout output through shared memory: every epilogue thread lays its output row down in a row-major
+// tile (row stride BN*4 + 16 bytes, which keeps the 16-byte stores of a quarter warp on distinct banks) and then
+// hands that row to the copy engine as one bulk copy to global memory - 128 row copies per tile instead of
+// thousands of scattered 32-byte stores.
+template <int BN> __host__ __device__ constexpr uint32_t out_tile_row_bytes() { return BN * 4 + 16; }
+__device__ __forceinline__ void out_tile_put32(uint32_t row_addr, int j0, const float (&y)[32])
+{
+    const uint32_t a = row_addr + (uint32_t)j0 * 4u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+        st_shared_v4(a + 16u * g, round_to_tf32(y[4 * g]), round_to_tf32(y[4 * g + 1]), round_to_tf32(y[4 * g + 2]),
+                     round_to_tf32(y[4 * g + 3]));
+}
+// the row's channels [k0, k0 + width) -> global; the caller commits and waits for the bulk group
+__device__ __forceinline__ void out_tile_store_row(const OutSpec& o, const RowDst& d, int k0, int width, uint32_t row_addr)
+{
+    const int w = min(width, o.Cp - k0);
+    if (d.valid && w > 0) bulk_store_global(o.out + d.base + k0, row_addr, (uint32_t)w * 4u);
+}
+
+// ---- split reduction by exchange: each CTA of the cluster owns `per` consecutive channels of the tile (the last
+// owner possibly fewer) and receives the other CTAs' partial sums of those channels as one bulk copy per peer from
+// shared memory to shared memory.  Exchange blocks are row-major [128 rows][w channels] with the 16-byte pieces of
+// every 128-byte group XOR-swizzled by (row & 7): thread-per-row accesses then stay free of bank conflicts without
+// padding, and sender and receiver use the same mapping.
+__host__ __device__ constexpr int split_share(int BN, int splits) { return ((((BN + splits - 1) / splits) + 31) / 32) * 32; }
+__host__ __device__ constexpr int split_width(int BN, int per, int rank)
+{
+    return BN - rank * per <= 0 ? 0 : (BN - rank * per < per ? BN - rank * per : per);
+}
+__host__ __device__ constexpr bool split_exchange_fits(int BN, int splits, int stage_region_bytes)
+{
+    return splits > 1 && 2 * 512 * split_share(BN, splits) * (splits - 1) <= stage_region_bytes;
+}
+__device__ __forceinline__ void xchg_put32(uint32_t block, int w, int row, int c0, const uint32_t (&v)[32])
+{
+    const uint32_t a = block + (uint32_t)(row * w + c0) * 4u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g)
+        st_shared_v4(a + (uint32_t)((g ^ (row & 7)) << 4), __uint_as_float(v[4 * g]), __uint_as_float(v[4 * g + 1]),
+                     __uint_as_float(v[4 * g + 2]), __uint_as_float(v[4 * g + 3]));
+}
+__device__ __forceinline__ void xchg_add32(uint32_t block, int w, int row, int c0, float (&y)[32])
+{
+    const uint32_t a = block + (uint32_t)(row * w + c0) * 4u;
+#pragma unroll
+    for (int g = 0; g < 8; ++g) {
+        const float4 t = ld_shared_v4(a + (uint32_t)((g ^ (row & 7)) << 4));
+        y[4 * g] += t.x; y[4 * g + 1] += t.y; y[4 * g + 2] += t.z; y[4 * g + 3] += t.w;
     }
 }
 

@@ -26,7 +26,7 @@ namespace halo {
 
 using namespace tc;
 
-constexpr int kThreads = 224;      // warp 0 producer, 1 and 6 MMA issuers, 2..5 epilogue
+constexpr int kThreads = 352;      // warp 0 producer, 1 and 6 MMA issuers, 2..5 and 7..10 epilogue
 constexpr int kMaxBStages = 8;
 constexpr int kASlots = 2;
 constexpr int kSmemBudget = 200 * 1024;
@@ -88,7 +88,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t accum_bar = b_empty + 8 * kMaxBStages;
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
-    __shared__ float s_bias[BN];
+    __shared__ __align__(16) float s_bias[BN];
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
@@ -211,35 +211,54 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 15);
         }
     } else {
-        // ---------------- epilogue
+        // ---------------- epilogue: 8 warps.  Warp w may read TMEM lanes 32*(w%4) .. +31 only, so warps 2..5 and
+        // 7..10 pair up on the same 32 rows: with several accumulators the two groups take alternate accumulators,
+        // with one they take the two halves of its columns.
         const int quarter = warp & 3;
+        const int group = warp >= 7 ? 1 : 0;
         const int row = quarter * 32 + lane;
-        for (int j = threadIdx.x - 64; j < BN; j += 128)
+        const int etid = threadIdx.x - (group ? 96 : 64);                  // 0 .. 255 over the epilogue threads
+        for (int j = etid; j < BN; j += 256)
             s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
         if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 16);   // one poller per warp
         __syncwarp();
-        asm volatile("bar.sync 1, 128;" ::: "memory");
+        asm volatile("bar.sync 1, 256;" ::: "memory");
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         if (ok && p.splits == 1) {
+            constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
+            const int c_begin = (NACC == 1 && group) ? HALF : 0, c_end = (NACC == 1 && !group) ? HALF : NCH;
+            // Staged layout: rows go through shared memory (the operand buffers are idle now) and leave as bulk
+            // copies; every thread owns the same row slot of each of the `nbuf` tile buffers that fit, so only its
+            // own earlier copy has to have been read before it overwrites a slot.
+            constexpr uint32_t TILE_BYTES = 128u * out_tile_row_bytes<BN>();
+            const int nbuf = (int)((uint32_t)(kASlots * p.a_slot_bytes + p.b_stages * Cfg::B_STAGE_BYTES) / TILE_BYTES);
+            const bool bulk = p.o.packed && nbuf >= (NACC == 1 ? 1 : 2);      // with several accumulators: a buffer per group
+            int turn = 0;
 #pragma unroll 1
-            for (int acc = 0; acc < NACC; ++acc) {
+            for (int acc = (NACC == 1 ? 0 : group); acc < NACC; acc += (NACC == 1 ? 1 : 2), ++turn) {
                 const RowDst d = halo_row_dst(p, f0 + acc * 128 + row);
+                const uint32_t row_addr = smem_base + (NACC == 1 ? 0u : (uint32_t)group * TILE_BYTES)
+                                        + (uint32_t)row * out_tile_row_bytes<BN>();
+                if (bulk && turn > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 #pragma unroll 1
-                for (int j0 = 0; j0 < BN; j0 += 32) {
+                for (int c = c_begin; c < c_end; ++c) {
                     uint32_t v[32];
-                    tmem_ld_32cols(trow + acc * BN + j0, v);
+                    tmem_ld_32cols(trow + acc * BN + 32 * c, v);
                     tmem_ld_wait();
                     float y[32];
-#pragma unroll
-                    for (int j = 0; j < 32; ++j) {
-                        y[j] = __uint_as_float(v[j]) + s_bias[j0 + j];
-                        if (p.o.relu) y[j] = fmaxf(y[j], 0.f);
-                    }
-                    store_row32(p.o, d, k0 + j0, y, smem_base + (uint32_t)(warp & 3) * 4224u);
+                    bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
+                    if (bulk) out_tile_put32(row_addr, 32 * c, y);
+                    else store_row32(p.o, d, k0 + 32 * c, y, 0u);
+                }
+                if (bulk) {
+                    fence_proxy_async_smem();
+                    out_tile_store_row(p.o, d, k0 + 32 * c_begin, 32 * (c_end - c_begin), row_addr + 128u * (uint32_t)c_begin);
+                    bulk_commit();
                 }
             }
+            if (bulk) bulk_wait_all();
         }
         tc_fence_before();
     }
