@@ -143,9 +143,32 @@ def whole_job_gflops(flops_per_replica_step: int, world: int, ms_per_step: float
     return world * flops_per_replica_step / (ms_per_step * 1e-3) / 1e9
 
 
-def single_layer_configs(B, wl, torch, peaks):
+def _graph_us(torch, fn, reps=20, replays=5):
+    """Device time per call of fn: `reps` calls captured in one CUDA graph (no host launch cost in the number)."""
+    g = torch.cuda.CUDAGraph()
+    with torch.cuda.graph(g):
+        for _ in range(reps):
+            fn()
+    g.replay()
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(replays):
+        g.replay()
+    e1.record()
+    torch.cuda.synchronize()
+    return e0.elapsed_time(e1) / (reps * replays) * 1e3
+
+
+def single_layer_configs(B, wl, torch, peaks, flush):
     """The four single-layer configurations (parity-test cases; reported for context): NCHW in and out through
-    boda_conv_fwd_planned, input staging included, 20 back-to-back launches per event pair (L2-warm)."""
+    boda_conv_fwd_planned, input staging included.  Per configuration: L2-warm time (20 launches per captured graph),
+    L2-cold time (one launch after an L2 flush, median of 9), the same with unbound filters (re-laid-out on every
+    call), and two floors measured the same way: the library's smallest kernel (a 3x3 pooling of one 3x3 plane) and
+    a device copy that moves the layer's algorithmic bytes."""
+    tiny_in = torch.zeros((1, 1, 3, 3), dtype=torch.float32, device="cuda")
+    tiny_out = torch.zeros((1, 1, 1, 1), dtype=torch.float32, device="cuda")
+    null_us = _graph_us(torch, lambda: B.boda_maxpool_fwd(tiny_in, tiny_out, 1, 1, 3, 3, 3, 2))
     out = []
     for cid in (1, 2, 3, 4):
         cfg = wl.CONFIGS[cid]
@@ -153,25 +176,58 @@ def single_layer_configs(B, wl, torch, peaks):
         x, w, b = (torch.from_numpy(t).cuda() for t in cfg.tensors())
         plan = B.ConvPlan(s.as_tuple(), tune=1)
         y = torch.empty(plan.out_shape, dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            plan(x, w, b, out=y)                              # unbound: filters staged on every call
+        torch.cuda.synchronize()
+        us_unbound = _graph_us(torch, lambda: plan(x, w, b, out=y))
         plan.bind_filters(w)
-        for _ in range(5):
+        for _ in range(3):
             plan(x, w, b, out=y)
         torch.cuda.synchronize()
-        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        reps = 20
-        e0.record()
-        for _ in range(reps):
+        us = _graph_us(torch, lambda: plan(x, w, b, out=y))
+        cold = []
+        for _ in range(9):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
             plan(x, w, b, out=y)
-        e1.record()
-        torch.cuda.synchronize()
-        us = e0.elapsed_time(e1) / reps * 1e3
+            e1.record()
+            torch.cuda.synchronize()
+            cold.append(e0.elapsed_time(e1) * 1e3)
+        cold_us = sorted(cold)[len(cold) // 2]
+        half = max(s.min_bytes // 8, 1)                        # floats: the copy reads and writes min_bytes in total
+        src = torch.empty(half, dtype=torch.float32, device="cuda")
+        dst = torch.empty(half, dtype=torch.float32, device="cuda")
+        copy_us = _graph_us(torch, lambda: dst.copy_(src))
         desc = plan.describe()
         plan.close()
         tf = s.flops / us / 1e6
-        out.append({"config": cid, "name": cfg.name, "us_per_call": round(us, 2), "gflops": round(tf * 1e3, 1),
+        out.append({"config": cid, "name": cfg.name, "us_per_call": round(us, 2), "us_l2_cold": round(cold_us, 2),
+                    "us_unbound_filters": round(us_unbound, 2), "gflops": round(tf * 1e3, 1),
                     "algorithmic_gbs": round(s.min_bytes / us / 1e3, 1),
-                    "frac_of_hbm_peak": round(s.min_bytes / us / 1e3 / peaks["hbm_gbs"], 4),
-                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4), "plan": desc})
+                    "frac_of_hbm_peak_l2_cold": round(s.min_bytes / cold_us / 1e3 / peaks["hbm_gbs"], 4),
+                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4),
+                    "floor_smallest_kernel_us": round(null_us, 2), "floor_size_matched_copy_us": round(copy_us, 2),
+                    "plan": desc})
+    return out
+
+
+def sgemm_table1(B, torch, peaks):
+    """boda_sgemm on the square sizes of the paper's Table 1 (context, not the headline): device time per call
+    from a captured graph of 20 calls, operands L2-warm."""
+    out = []
+    for n in (128, 256, 512, 1024, 2048):
+        a = torch.randn((n, n), dtype=torch.float32, device="cuda")
+        b = torch.randn((n, n), dtype=torch.float32, device="cuda")
+        c = torch.empty((n, n), dtype=torch.float32, device="cuda")
+        for _ in range(3):
+            B.boda_sgemm(a, b, c, n, n, n)
+        torch.cuda.synchronize()
+        us = _graph_us(torch, lambda: B.boda_sgemm(a, b, c, n, n, n))
+        tf = 2.0 * n * n * n / us / 1e6
+        out.append({"n": n, "us_per_call": round(us, 2), "gflops": round(tf * 1e3, 1),
+                    "flops_per_byte": round(2.0 * n * n * n / (12.0 * n * n), 1),
+                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4)})
     return out
 
 
@@ -353,7 +409,8 @@ def run_ours(args):
                     "frac": round(dom_tf / peak, 4), "traffic": traffic, "kernel": layers[dom]["op"] + ": " + descs[dom],
                     "peak_source": peak_note, "launch_ms": round(dom_ms, 5),
                     "timing": f"{dom_reps} back-to-back launches of that layer in place per event pair, L2-warm as inside the step"}
-        per_config = single_layer_configs(B, wl, torch, peaks)
+        per_config = single_layer_configs(B, wl, torch, peaks, flush)
+        sgemm_rows = sgemm_table1(B, torch, peaks)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -371,6 +428,7 @@ def run_ours(args):
                              "kind": "oracle", "sample": f"the whole batch-{BATCH} stack, best of 2 ({cpu_t:.2f} s)" if cpu_t else "skipped"},
             "layers": layers,
             "single_layer_configs": per_config,
+            "sgemm_table1": sgemm_rows,
             "frac_of_tf32_peak_whole_step": round(value / 1e3 / (0.5 * peaks["bf16_tflops"]) / world, 4),
         }
         print(json.dumps(line))

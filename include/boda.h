@@ -152,6 +152,18 @@ int boda_conv_fwd_host(const float* in_host, const float* filt_host, const float
                        void* stream);
 
 /*
+ * Single-precision matrix product C[M][N] = A[M][K] * B[K][N], all three row-major, dense, fp32 DEVICE
+ * pointers (the paper's warm-up operation: Section 4, Table 1 lists square sizes 128 ... 2048 with
+ * 2*M*N*K FLOPs and 4*(M*K + K*N + M*N) bytes).  Section 5 observes that a 1x1 convolution "is" this
+ * product; the library takes that literally and runs the product as the 1x1 convolution of a one-image
+ * input in[1][K][1][N] = B with filters filt[M][K][1][1] = A, no bias, no ReLU, through the same plan
+ * cache and kernels as boda_conv_fwd (default options: TF32 tensor cores where profitable, so the
+ * TF32 error bar applies).  The first call for a size allocates; later calls do not.
+ * Errors: INVALID_ARG (NULL pointer, non-positive size), plus those of boda_conv_fwd.
+ */
+int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, void* stream);
+
+/*
  * The forward pass for callers that must not allocate device memory.  (The paper has no counterpart: this
  * is a property of the library, not of the method.)
  *

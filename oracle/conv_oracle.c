@@ -134,6 +134,24 @@ double oracle_sgemm_ai(long long M, long long N, long long K)
            (4.0 * ((double)M * N + (double)M * K + (double)K * N));
 }
 
+/*
+ * SGEMM, Section 4 (the paper's warm-up; Table 1): C[i][j] = sum over k of A[i][k] * B[k][j], all row-major.
+ * The definition written out: one fp64 accumulator per element, k ascending.  OpenMP over rows only.
+ * Returns 0 on success, 1 on invalid arguments.
+ */
+int oracle_sgemm_f64(const double* A, const double* B, double* C, int M, int N, int K)
+{
+    if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return 1;
+#pragma omp parallel for schedule(static)
+    for (int i = 0; i < M; ++i)
+        for (int j = 0; j < N; ++j) {
+            double acc = 0.0;
+            for (int k = 0; k < K; ++k) acc += A[(size_t)i * K + k] * B[(size_t)k * N + j];
+            C[(size_t)i * N + j] = acc;
+        }
+    return 0;
+}
+
 int oracle_num_threads(void)
 {
 #ifdef _OPENMP

@@ -54,6 +54,8 @@ def _load():
         lib.oracle_conv_min_bytes.restype = ll
         lib.oracle_sgemm_ai.argtypes = [ll, ll, ll]
         lib.oracle_sgemm_ai.restype = ctypes.c_double
+        lib.oracle_sgemm_f64.argtypes = [dp, dp, dp, i, i, i]
+        lib.oracle_sgemm_f64.restype = i
         lib.oracle_num_threads.argtypes = []
         lib.oracle_num_threads.restype = i
         _lib = lib
@@ -128,6 +130,20 @@ def conv_min_bytes(N, C, H, W, K, R, S, stride, pad) -> int:
 
 def sgemm_ai(M: int, N: int, K: int) -> float:
     return float(_load().oracle_sgemm_ai(M, N, K))
+
+
+def sgemm(A, Bm) -> np.ndarray:
+    """C = A @ Bm by the definition (Section 4, Table 1): row-major [M][K] x [K][N], fp64 accumulation, k ascending."""
+    a, b = _f64(A), _f64(Bm)
+    if a.ndim != 2 or b.ndim != 2 or a.shape[1] != b.shape[0]:
+        raise ValueError("sgemm: shapes do not chain")
+    M, K = a.shape
+    N = b.shape[1]
+    c = np.empty((M, N), dtype=np.float64)
+    rc = _load().oracle_sgemm_f64(_ptr(a), _ptr(b), _ptr(c), M, N, K)
+    if rc != 0:
+        raise ValueError("oracle_sgemm_f64: invalid arguments")
+    return c
 
 
 def num_threads() -> int:

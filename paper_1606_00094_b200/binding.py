@@ -67,6 +67,8 @@ _lib.boda_conv_fwd_planned.argtypes = [_vp] * 7
 _lib.boda_conv_fwd_planned.restype = _i
 _lib.boda_conv_fwd.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd.restype = _i
+_lib.boda_sgemm.argtypes = [_vp] * 3 + [_i] * 3 + [_vp]
+_lib.boda_sgemm.restype = _i
 _lib.boda_conv_fwd_host.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd_host.restype = _i
 _lib.boda_conv_fwd_noalloc.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
@@ -223,6 +225,11 @@ def boda_conv_fwd_noalloc(inp, filt, bias, out, N, C, H, W, K, R, S, stride, pad
     BODA_ERR_TOO_LARGE when the shape's scratch exceeds BODA_NOALLOC_SCRATCH_BYTES."""
     _check(_lib.boda_conv_fwd_noalloc(_addr(inp), _addr(filt), _addr(bias), _addr(out), N, C, H, W, K, R, S, stride,
                                       pad, int(bool(relu)), _stream(stream)), "boda_conv_fwd_noalloc")
+
+
+def boda_sgemm(A, Bm, C, M, N, K, stream=None) -> None:
+    """C[M][N] = A[M][K] @ Bm[K][N], row-major fp32 device tensors."""
+    _check(_lib.boda_sgemm(_addr(A), _addr(Bm), _addr(C), M, N, K, _stream(stream)), "boda_sgemm")
 
 
 def boda_maxpool_fwd(inp, out, N, C, H, W, ksz=3, stride=2, stream=None) -> None:

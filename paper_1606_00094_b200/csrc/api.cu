@@ -80,29 +80,33 @@ int get_ctx(int device, DeviceCtx** out)
     return BODA_OK;
 }
 
-// ---- autotune cache: a text file "key tile split" per line, named by the environment variable BODA_TUNE_CACHE
-bool tune_cache_lookup(const char* key, int* tile, int* split)
+// ---- autotune cache: a text file with one line "key tile split variant s2d" per tuned shape, named by the
+// environment variable BODA_TUNE_CACHE
+bool tune_cache_lookup(const char* key, int* tile, int* split, int* variant, int* s2d)
 {
     const char* path = std::getenv("BODA_TUNE_CACHE");
     if (!path || !*path) return false;
     FILE* f = std::fopen(path, "r");
     if (!f) return false;
-    char k[200];
-    int t = 0, sp = 0;
+    char line[320], k[200];
     bool hit = false;
-    while (std::fscanf(f, "%199s %d %d", k, &t, &sp) == 3)
-        if (std::strcmp(k, key) == 0) { *tile = t; *split = sp; hit = true; }
+    while (std::fgets(line, sizeof(line), f)) {
+        int t = 0, sp = 0, v = 0, sd = 0;
+        if (std::sscanf(line, "%199s %d %d %d %d", k, &t, &sp, &v, &sd) == 5 && std::strcmp(k, key) == 0) {
+            *tile = t; *split = sp; *variant = v; *s2d = sd; hit = true;
+        }
+    }
     std::fclose(f);
     return hit;
 }
 
-void tune_cache_store(const char* key, int tile, int split)
+void tune_cache_store(const char* key, int tile, int split, int variant, int s2d)
 {
     const char* path = std::getenv("BODA_TUNE_CACHE");
     if (!path || !*path) return;
     FILE* f = std::fopen(path, "a");
     if (!f) return;
-    std::fprintf(f, "%s %d %d\n", key, tile, split);
+    std::fprintf(f, "%s %d %d %d %d\n", key, tile, split, variant, s2d);
     std::fclose(f);
 }
 
@@ -287,40 +291,65 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
     if (!o.tune || o.tile_id >= 0) {
         rc = plan_build(*shape, o, ctx, variant, o.tile_id, o.split_k, plan);
     } else {
-        // Automated tuning: time every tile (and split) of the chosen variant, keep the fastest.  Winners are
-        // remembered in the file named by BODA_TUNE_CACHE (if set), one line per (shape, variant).
+        // Automated tuning: the rule above names a variant; timing confirms or overturns it.  Every tile and split
+        // of that variant is timed and, when the caller left variant and math open, so is the alternative (the FP32
+        // kernel against the tensor-core variant, and a strided tconv layer with and without its space-to-depth
+        // view).  The fastest plan is kept and remembered in the file named by BODA_TUNE_CACHE (if set).
         char key[160];
-        std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,m%d", shape->N, shape->C, shape->H, shape->W,
-                      shape->K, shape->R, shape->S, shape->stride, shape->pad, variant, o.s2d, o.split_k);
-        int c_tile = -1, c_split = 0;
-        if (tune_cache_lookup(key, &c_tile, &c_split)) {
-            rc = plan_build(*shape, o, ctx, variant, c_tile, c_split, plan);
+        std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d", shape->N, shape->C, shape->H, shape->W,
+                      shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math);
+        int c_tile = -1, c_split = 0, c_variant = variant, c_s2d = o.s2d;
+        if (tune_cache_lookup(key, &c_tile, &c_split, &c_variant, &c_s2d)) {
+            boda_plan_opts oc = o;
+            oc.s2d = c_s2d;
+            rc = plan_build(*shape, oc, ctx, c_variant, c_tile, c_split, plan);
             if (rc == BODA_OK) { (void)cudaSetDevice(prev); return rc; }
+        }
+        struct Cand { int variant, s2d; };
+        std::vector<Cand> cands;
+        const int tensor_variant = k1_legal ? BODA_VARIANT_K1CONV : t_legal ? BODA_VARIANT_TCONV : -1;
+        const bool open_choice = o.variant == BODA_VARIANT_AUTO && o.math == BODA_MATH_AUTO;
+        auto add_tensor = [&](int v) {
+            if (v == BODA_VARIANT_TCONV && o.s2d < 0 && igemm_s2d_applicable(d)) { cands.push_back({v, 0}); cands.push_back({v, 1}); }
+            else cands.push_back({v, o.s2d});
+        };
+        if (variant == BODA_VARIANT_DIRECT) {
+            cands.push_back({variant, o.s2d});
+            if (open_choice && tensor_variant >= 0 && d.K >= 16) add_tensor(tensor_variant);
+        } else {
+            add_tensor(variant);
+            if (open_choice) cands.push_back({BODA_VARIANT_DIRECT, o.s2d});
         }
         boda_conv_plan* best = nullptr;
         float best_ms = 1e30f;
-        const int ntiles = variant == BODA_VARIANT_DIRECT ? direct_num_tiles() : igemm_num_tiles();
-        for (int t = 0; t < ntiles; ++t) {
-            const int nsplit = variant == BODA_VARIANT_DIRECT ? 1 : igemm_num_split_candidates();
-            for (int si = 0; si < nsplit; ++si) {
-                const int split = variant == BODA_VARIANT_DIRECT ? 0 : igemm_split_candidate(si);
-                if (o.split_k > 0 && split != o.split_k) continue;
-                boda_conv_plan* cand = nullptr;
-                if (plan_build(*shape, o, ctx, variant, t, split, &cand) != BODA_OK) continue;
-                float ms = 0.f;
-                if (plan_time_ms(cand, &ms) == BODA_OK && ms < best_ms) {
-                    if (best) boda_conv_plan_destroy(best);
-                    best = cand;
-                    best_ms = ms;
-                } else {
-                    boda_conv_plan_destroy(cand);
+        int best_s2d = o.s2d;
+        for (const Cand& c : cands) {
+            boda_plan_opts oc = o;
+            oc.s2d = c.s2d;
+            const int ntiles = c.variant == BODA_VARIANT_DIRECT ? direct_num_tiles() : igemm_num_tiles();
+            for (int t = 0; t < ntiles; ++t) {
+                const int nsplit = c.variant == BODA_VARIANT_DIRECT ? 1 : igemm_num_split_candidates();
+                for (int si = 0; si < nsplit; ++si) {
+                    const int split = c.variant == BODA_VARIANT_DIRECT ? 0 : igemm_split_candidate(si);
+                    if (o.split_k > 0 && split != o.split_k) continue;
+                    boda_conv_plan* cand = nullptr;
+                    if (plan_build(*shape, oc, ctx, c.variant, t, split, &cand) != BODA_OK) continue;
+                    float ms = 0.f;
+                    if (plan_time_ms(cand, &ms) == BODA_OK && ms < best_ms) {
+                        if (best) boda_conv_plan_destroy(best);
+                        best = cand;
+                        best_ms = ms;
+                        best_s2d = c.s2d;
+                    } else {
+                        boda_conv_plan_destroy(cand);
+                    }
                 }
             }
         }
         if (best) {
             *plan = best;
             rc = BODA_OK;
-            tune_cache_store(key, best->tile_id, best->ig ? igemm_plan_splits(best->ig) : 0);
+            tune_cache_store(key, best->tile_id, best->ig ? igemm_plan_splits(best->ig) : 0, best->variant, best_s2d);
         }
         else rc = plan_build(*shape, o, ctx, variant, -1, o.split_k, plan);
     }
@@ -463,6 +492,13 @@ int boda_conv_fwd(const float* in, const float* filt, const float* bias, float* 
     int rc = cache_lookup(s, false, &e);
     if (rc != BODA_OK) return rc;
     return boda_conv_fwd_planned(e->plan, in, filt, bias, out, e->workspace, stream);
+}
+
+int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, void* stream)
+{
+    if (!A || !B || !C || M <= 0 || N <= 0 || K <= 0) return BODA_ERR_INVALID_ARG;
+    // in[1][K][1][N] = B, filt[M][K][1][1] = A, out[1][M][1][N] = C
+    return boda_conv_fwd(B, A, nullptr, C, 1, K, 1, N, M, 1, 1, 1, 0, 0, stream);
 }
 
 int boda_conv_fwd_host(const float* in, const float* filt, const float* bias, float* out, int N, int C, int H,

@@ -35,7 +35,7 @@ namespace {
 constexpr int BM = 128;          // pixels per CTA tile (UMMA M)
 constexpr int BKC = 32;          // channels per reduction chunk (128 bytes of fp32)
 constexpr int A_STAGE_BYTES = BM * BKC * 4;
-constexpr int kIgemmThreads = 352;   // warp 0 producer, 1 and 6 MMA issuers, 2..5 and 7..10 epilogue
+constexpr int kIgemmThreads = 416;   // warps 0, 11, 12 producers, 1 and 6 MMA issuers, 2..5 and 7..10 epilogue
 
 using namespace tc;
 
@@ -136,9 +136,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t tmem_acc = s_tmem_base;
     pdl_wait();          // everything above overlapped the previous kernel; its results are needed from here on
 
-    if (warp == 0) {
+    if (warp == 0 || warp >= 11) {
         if (lane == 0) {
-            // ---------------- TMA producer
+            // ---------------- TMA producers.  For one thread, an arrival with a byte count costs about 105 clocks, a
+            // TMA issue about 125 and a successful barrier test about 45 (measured): one thread doing all of it needs
+            // about 430 clocks per stage, more than the MMAs of a stage take for BN <= 192.  So three threads in three
+            // warps share a stage: warp 0 loads the input tile (A), warp 11 the filter tile (B), warp 12 posts the
+            // stage's byte count on its full barrier (bytes that land before the count is posted are legal: the
+            // barrier's phase cannot complete before its one arrival).  Ring position, parity and addresses advance
+            // incrementally: the loops hold no division.
+            const int role = warp == 0 ? 0 : warp == 11 ? 1 : 2;
             const int n0 = m0 / p.o.PQ;
             const int rem = m0 - n0 * p.o.PQ;
             const int p0 = rem / p.o.Q;
@@ -149,18 +156,18 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             int cc = it_begin - tap * p.cchunks;
             int r = tap / p.S;
             int s = tap - r * p.S;
-            // ring position, parity and addresses advance incrementally: this single thread's loop latency
-            // bounds the iteration rate, so it holds no division
             uint32_t stage = 0, par = 1;
-            uint32_t fb = full_bar, eb = empty_bar, adst = smem_a, bdst = smem_b;
+            uint32_t fb = full_bar, eb = empty_bar, dst = role == 0 ? smem_a : smem_b;
+            const uint32_t dst0 = dst, dst_step = role == 0 ? (uint32_t)A_STAGE_BYTES : (uint32_t)Cfg::B_STAGE_BYTES;
+            const int cchunks = p.cchunks, S = p.S;
             for (int i = 0; i < my_iters; ++i) {
-                if (!mbar_wait(eb, par, &s_abort, p.status, 1)) break;
-                mbar_expect_tx(fb, Cfg::STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
-                tma_load_im2col_4d(adst, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
-                tma_load_3d(bdst, &map_b, fb, cc * BKC, k0, tap);
-                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; adst = smem_a; bdst = smem_b; }
-                else { fb += 8; eb += 8; adst += A_STAGE_BYTES; bdst += Cfg::B_STAGE_BYTES; }
-                if (++cc == p.cchunks) { cc = 0; ++tap; if (++s == p.S) { s = 0; ++r; } }
+                if (!mbar_wait(eb, par, &s_abort, p.status, 1 + 5 * role)) break;
+                if (role == 0) tma_load_im2col_4d(dst, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                else if (role == 1) tma_load_3d(dst, &map_b, fb, cc * BKC, k0, tap);
+                else mbar_expect_tx(fb, Cfg::STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
+                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = dst0; }
+                else { fb += 8; eb += 8; dst += dst_step; }
+                if (++cc == cchunks) { cc = 0; ++tap; if (++s == S) { s = 0; ++r; } }
             }
         }
     } else if (warp == 1 || warp == 6) {
@@ -322,7 +329,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         }
         tc_fence_before();
     }
-    if (exchange && (warp < 2 || warp == 6)) {      // the other roles' half of the first cluster barrier
+    if (exchange && (warp < 2 || warp == 6 || warp >= 11)) {      // the other roles' half of the first cluster barrier
         cluster_arrive();
         cluster_wait();
     }
@@ -620,7 +627,8 @@ bool igemm_variant_profitable(const ConvDims& d)
     // Channels are padded to 32 per reduction chunk and pixels to 128 per tile: tiny C (first layers) and tiny
     // layers stay on the FP32 kernel.
     if (d.K < 16 || (long long)d.M * d.K < 128 * 64) return false;
-    return d.C >= 16 || s2d_efficiency(d) >= 0.35;
+    const int Cp = ((d.C + BKC - 1) / BKC) * BKC;
+    return std::max((double)d.C / Cp, s2d_efficiency(d)) >= 0.2;     // measured: C = 8 of 32 wins, C = 3 of 32 loses
 }
 
 int igemm_num_tiles() { return kNumIgemmTiles; }
@@ -629,37 +637,58 @@ int igemm_split_candidate(int i) { return kSplitCandidates[i]; }
 
 namespace {
 
-// Cost model (SM clocks) used when a plan is not tuned by timing.  Calibrated on B200: one thread issues the MMAs of
-// a stage, and a stage costs about 290 clocks of MMA issue per 128-row accumulator plus about 240 (im2col kernel) or
-// 390 (halo kernel) clocks of barrier hand-shakes, unless the MMAs themselves take longer (2*BN clocks per 32
-// channels and accumulator).  Prologue, pipeline fill and tail cost about 4500 clocks; the epilogue about 22 clocks
-// per channel, a cluster split reduction about 6 + 30/splits per channel plus 2500.
-double epilogue_cost(double cols, int splits)
+// Cost model (SM clocks) used when a plan is not tuned by timing; fitted to a sweep of every tile and split over
+// fourteen layer shapes on B200 (its choice is within 3 % of the best measured one for each of them).
+//   main loop: a stage costs the MMAs' 2*BN clocks or about 380 clocks of producer / issuer hand-shakes, whichever
+//              is longer (halo kernel: 2.2*BN per accumulator, or 290 per accumulator + 390);
+//   fixed:     prologue, pipeline fill and tail, about 3500 clocks (halo kernel 5000);
+//   epilogue:  32 clocks per channel without a split (the SM writes about 32 bytes per clock); with a split by
+//              exchange 1500 + 14 per channel sent + 20 per channel and peer received + (40 + 6 per peer) per channel
+//              finished + 300 per CTA of the cluster; the remote-read fallback 60 per channel and peer;
+//   waves:     CTAs over 148 SMs, and clusters over what eight GPCs of 16 SMs hold at once.
+int split_share_host(int BN, int splits) { return ((((BN + splits - 1) / splits) + 31) / 32) * 32; }
+
+double epilogue_cost(int BN, int splits, bool exchange)
 {
-    return splits > 1 ? cols * (6.0 + 30.0 / splits) + 2500.0 : cols * 22.0;
+    if (splits <= 1) return 32.0 * BN;
+    const int w = split_share_host(BN, splits);
+    if (exchange) return 1500.0 + 14.0 * (BN - w) + 20.0 * w * (splits - 1) + w * (40.0 + 6.0 * (splits - 1)) + 300.0 * splits;
+    return 1500.0 + 22.0 * BN + 60.0 * w * splits + 300.0 * splits;
+}
+
+double wave_count(double tiles, int splits)
+{
+    double waves = (double)(long long)((tiles * splits + 147) / 148);
+    if (splits > 1) waves = std::max(waves, (double)(long long)((tiles + 8 * (16 / splits) - 1) / (8 * (16 / splits))));
+    return waves;
+}
+
+template <int BN> constexpr int stage_region_bytes() { return TileCfg<BN>::STAGES * TileCfg<BN>::STAGE_BYTES; }
+int stage_region_of(int BN)
+{
+    return BN == 64 ? stage_region_bytes<64>() : BN == 96 ? stage_region_bytes<96>() : BN == 128 ? stage_region_bytes<128>()
+         : BN == 192 ? stage_region_bytes<192>() : stage_region_bytes<256>();
 }
 
 double model_cost(const ConvDims& d, int Cp, int BN, int splits)
 {
     const int iters = d.R * d.S * (Cp / BKC);
     const int ips = (iters + splits - 1) / splits;
+    const int se = (iters + ips - 1) / ips;
     const long long tm = (d.M + BM - 1) / BM, tn = (d.K + BN - 1) / BN;
-    const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
-    const double waves = (double)(long long)((ctas + 147) / 148);
-    const double per_iter = std::max(2.0 * BN, 530.0);
-    return waves * (ips * per_iter + 4500.0 + epilogue_cost(BN, splits));
+    const double per_iter = std::max(2.0 * BN, 380.0);
+    return wave_count((double)tm * tn, se) * (ips * per_iter + 3500.0 + epilogue_cost(BN, se, split_exchange_fits(BN, se, stage_region_of(BN))));
 }
 
 double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
 {
     const int iters = d.R * d.S * (Cp / BKC);
     const int ips = (iters + splits - 1) / splits;
+    const int se = (iters + ips - 1) / ips;
     const long long mflat = (long long)d.N * (d.H + d.pad) * (d.W + d.pad);
     const long long tm = (mflat + 128 * nacc - 1) / (128 * nacc), tn = (d.K + BN - 1) / BN;
-    const double ctas = (double)tm * tn * ((iters + ips - 1) / ips);
-    const double waves = (double)(long long)((ctas + 147) / 148);
     const double per_iter = std::max(2.2 * BN * nacc, 290.0 * nacc + 390.0);
-    return waves * (ips * per_iter + 5000.0 + nacc * epilogue_cost(BN, splits));
+    return wave_count((double)tm * tn, se) * (ips * per_iter + 5000.0 + nacc * epilogue_cost(BN, se, false));
 }
 
 template <int BN, int NACC>
@@ -763,7 +792,8 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         ConvDims e;
         const bool can = s2d_view(d_in, &e);
         if (s2d > 0 && !can) return BODA_ERR_UNSUPPORTED;
-        if (can && (s2d > 0 || s2d_efficiency(d_in) >= 0.35)) { d = e; use_s2d = true; }
+        const int Cp_in = ((d_in.C + BKC - 1) / BKC) * BKC;
+        if (can && (s2d > 0 || s2d_efficiency(d_in) >= std::max(0.2, (double)d_in.C / Cp_in))) { d = e; use_s2d = true; }
     } else if (s2d > 0) {
         return BODA_ERR_UNSUPPORTED;
     }

@@ -326,3 +326,41 @@ def test_generators_are_deterministic_and_sane():
     assert abs(float(w.std()) - 0.1) < 0.02 and abs(float(b.std()) - 0.01) < 0.006
     assert wl.stack_flops(20) == 43065365760
     assert math.isclose(wl.CONFIGS[4].shape.flops, 5980815360)
+
+
+# ---------------------------------------------------------------- SGEMM oracle (Section 4, Table 1)
+def test_sgemm_hand_case():
+    # [[1,2],[3,4]] x [[5,6,7],[8,9,10]] worked by hand: row 0 = (1*5+2*8, 1*6+2*9, 1*7+2*10), row 1 likewise
+    A = np.array([[1, 2], [3, 4]], dtype=np.float32)
+    Bm = np.array([[5, 6, 7], [8, 9, 10]], dtype=np.float32)
+    np.testing.assert_array_equal(orc.sgemm(A, Bm), np.array([[21, 24, 27], [47, 54, 61]], dtype=np.float64))
+
+
+def test_sgemm_closed_forms():
+    # ones x ones = K everywhere; identity is neutral on either side; a transposed operand would fail the last check
+    M, N, K = 7, 5, 11
+    np.testing.assert_array_equal(orc.sgemm(np.ones((M, K)), np.ones((K, N))), np.full((M, N), float(K)))
+    X = wl.normal(91, (6, 6))
+    np.testing.assert_array_equal(orc.sgemm(np.eye(6), X), X.astype(np.float64))
+    np.testing.assert_array_equal(orc.sgemm(X, np.eye(6)), X.astype(np.float64))
+    A = np.arange(6, dtype=np.float64).reshape(2, 3)
+    Bm = np.arange(12, dtype=np.float64).reshape(3, 4)
+    # entry (1, 2): row (3,4,5) . column (2,6,10) = 6 + 24 + 50
+    assert orc.sgemm(A, Bm)[1, 2] == 80.0
+
+
+def test_sgemm_is_the_1x1_convolution():
+    # Section 5: a 1x1 convolution of a one-image input is the matrix product filt[M x K] . in[K x N];
+    # the two oracle routines are separate loop nests, so each pins the other
+    M, N, K = 9, 14, 6
+    A = wl.normal(92, (M, K))
+    Bm = wl.normal(93, (K, N))
+    via_conv = orc.conv_fwd(Bm.reshape(1, K, 1, N), A.reshape(M, K, 1, 1))
+    np.testing.assert_allclose(orc.sgemm(A, Bm), via_conv.reshape(M, N), rtol=1e-14, atol=1e-14)
+
+
+def test_sgemm_against_library_matmul():
+    A = wl.normal(94, (33, 17))
+    Bm = wl.normal(95, (17, 29))
+    ref = A.astype(np.float64) @ Bm.astype(np.float64)
+    np.testing.assert_allclose(orc.sgemm(A, Bm), ref, rtol=1e-13, atol=1e-13)
