@@ -201,8 +201,17 @@ def single_layer_configs(B, wl, torch, peaks, flush):
         copy_us = _graph_us(torch, lambda: dst.copy_(src))
         desc = plan.describe()
         plan.close()
+        # the same layer in the error-compensated TF32 mode (FP32 accuracy from the tensor cores)
+        plan3 = B.ConvPlan(s.as_tuple(), math=B.BODA_MATH_TF32X3, tune=1)
+        plan3.bind_filters(w)
+        for _ in range(3):
+            plan3(x, w, b, out=y)
+        torch.cuda.synchronize()
+        us_x3 = _graph_us(torch, lambda: plan3(x, w, b, out=y))
+        desc_x3 = plan3.describe()
+        plan3.close()
         tf = s.flops / us / 1e6
-        out.append({"config": cid, "name": cfg.name, "us_per_call": round(us, 2), "us_l2_cold": round(cold_us, 2),
+        out.append({"config": cid, "us_tf32x3": round(us_x3, 2), "plan_tf32x3": desc_x3, "name": cfg.name, "us_per_call": round(us, 2), "us_l2_cold": round(cold_us, 2),
                     "us_unbound_filters": round(us_unbound, 2), "gflops": round(tf * 1e3, 1),
                     "algorithmic_gbs": round(s.min_bytes / us / 1e3, 1),
                     "frac_of_hbm_peak_l2_cold": round(s.min_bytes / cold_us / 1e3 / peaks["hbm_gbs"], 4),

@@ -55,7 +55,14 @@ enum { BODA_VARIANT_AUTO = -1, BODA_VARIANT_DIRECT = 0, BODA_VARIANT_K1CONV = 1,
 /* Arithmetic the plan may use. */
 enum { BODA_MATH_AUTO = 0,       /* TF32 tensor cores where a tensor-core variant applies */
        BODA_MATH_FP32 = 1,       /* FP32 FMA only (DIRECT); relative L2 error vs fp64 <= 1e-5 */
-       BODA_MATH_TF32 = 2 };     /* TF32 operands, fp32 accumulate; relative L2 error <= 5e-3 */
+       BODA_MATH_TF32 = 2,       /* TF32 operands, fp32 accumulate; relative L2 error <= 5e-3 */
+       BODA_MATH_TF32X3 = 3 };   /* error-compensated TF32 on the tensor cores: every operand is split into a TF32
+                                    value and a TF32 remainder, and each product is formed as hi*hi + lo*hi + hi*lo
+                                    (three tensor-core products, fp32 accumulate); meets the FP32 bar (<= 1e-5) at
+                                    about a third of the TF32 rate.  The paper names reduced and mixed precision as
+                                    the next step (Sections 2 and 6); this is the mode for callers who need FP32
+                                    accuracy from the tensor cores.  NCHW in and out only; K1CONV and TCONV (im2col
+                                    kernel); where no tensor-core variant is legal the FP32 kernel runs instead. */
 
 typedef struct boda_conv_shape {
     int N, C, H, W;              /* input  [N][C][H][W] */

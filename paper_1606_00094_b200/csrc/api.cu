@@ -169,7 +169,7 @@ bool conv_plan_input_geometry(const boda_conv_plan* p, int* Hp, int* Wp, int* Cp
     return p->ig ? igemm_plan_input_geometry(p->ig, Hp, Wp, Cp) : false;
 }
 
-bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr; }
+bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && p->math != BODA_MATH_TF32X3; }
 
 int conv_plan_set_io(boda_conv_plan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
@@ -242,8 +242,8 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
         if (e != cudaSuccess) rc = record_cuda_error(e, "tap table upload");
         p->ws_bytes = 0;
     } else {
-        p->math = BODA_MATH_TF32;
-        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig);
+        p->math = o.math == BODA_MATH_TF32X3 ? BODA_MATH_TF32X3 : BODA_MATH_TF32;
+        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig, o.math == BODA_MATH_TF32X3);
         if (rc == BODA_OK) { p->tile_id = igemm_plan_tile(p->ig); p->ws_bytes = igemm_plan_workspace_bytes(p->ig); }
     }
     if (rc != BODA_OK) { boda_conv_plan_destroy(p); return rc; }
@@ -259,7 +259,7 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
     boda_plan_opts o;
     boda_plan_opts_default(&o);
     if (opts) o = *opts;
-    if (o.math < BODA_MATH_AUTO || o.math > BODA_MATH_TF32) return BODA_ERR_INVALID_ARG;
+    if (o.math < BODA_MATH_AUTO || o.math > BODA_MATH_TF32X3) return BODA_ERR_INVALID_ARG;
     if (o.variant < BODA_VARIANT_AUTO || o.variant > BODA_VARIANT_TCONV) return BODA_ERR_INVALID_ARG;
 
     std::lock_guard<std::mutex> lock(g_mutex);
@@ -278,6 +278,8 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
     int variant = o.variant;
     if (variant == BODA_VARIANT_AUTO) {
         if (o.math == BODA_MATH_FP32) variant = BODA_VARIANT_DIRECT;
+        else if (o.math == BODA_MATH_TF32X3 && d.K >= 16 && (k1_legal || t_legal) && o.s2d <= 0)
+            variant = k1_legal ? BODA_VARIANT_K1CONV : BODA_VARIANT_TCONV;   // FP32-accurate either way: the tensor cores if legal
         else if (k1_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_K1CONV;
         else if (t_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_TCONV;
         else variant = BODA_VARIANT_DIRECT;
@@ -367,7 +369,8 @@ int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
     } else {
         char tmp[160];
         igemm_plan_describe(p->ig, tmp, sizeof(tmp));
-        std::snprintf(buf, n, "variant=%s %s math=tf32 workspace=%zu", vn[p->variant], tmp, p->ws_bytes);
+        std::snprintf(buf, n, "variant=%s %s math=%s workspace=%zu", vn[p->variant], tmp,
+                      p->math == BODA_MATH_TF32X3 ? "tf32x3" : "tf32", p->ws_bytes);
     }
     return BODA_OK;
 }

@@ -43,7 +43,9 @@ using namespace tc;
 struct IgemmParams {
     int M, stride, pad, S;
     int cchunks;                 // Cp / 32
-    int iters_total;             // taps * cchunks
+    int terms;                   // 1: TF32.  3: error-compensated TF32 (each chunk as hi*hi, lo*hi, hi*lo)
+    int lo_off;                  // channel offset of the low parts in the staged operands (Cp)
+    int iters_total;             // taps * cchunks * terms
     int iters_per_split;
     int splits;
     const float* bias;
@@ -152,8 +154,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int q0 = rem - p0 * p.o.Q;
             const int w0 = q0 * p.stride - p.pad;
             const int h0 = p0 * p.stride - p.pad;
-            int tap = it_begin / p.cchunks;
-            int cc = it_begin - tap * p.cchunks;
+            const int terms = p.terms;
+            const int chunk0 = it_begin / terms;
+            int term = it_begin - chunk0 * terms;
+            int tap = chunk0 / p.cchunks;
+            int cc = chunk0 - tap * p.cchunks;
             int r = tap / p.S;
             int s = tap - r * p.S;
             uint32_t stage = 0, par = 1;
@@ -162,12 +167,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int cchunks = p.cchunks, S = p.S;
             for (int i = 0; i < my_iters; ++i) {
                 if (!mbar_wait(eb, par, &s_abort, p.status, 1 + 5 * role)) break;
-                if (role == 0) tma_load_im2col_4d(dst, &map_a, fb, cc * BKC, w0, h0, n0, (uint16_t)s, (uint16_t)r);
-                else if (role == 1) tma_load_3d(dst, &map_b, fb, cc * BKC, k0, tap);
+                // error-compensated mode: term 0 = hi * hi, term 1 = lo(input) * hi(filter), term 2 = hi(input) * lo(filter)
+                if (role == 0) tma_load_im2col_4d(dst, &map_a, fb, cc * BKC + (term == 1 ? p.lo_off : 0), w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                else if (role == 1) tma_load_3d(dst, &map_b, fb, cc * BKC + (term == 2 ? p.lo_off : 0), k0, tap);
                 else mbar_expect_tx(fb, Cfg::STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
                 if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = dst0; }
                 else { fb += 8; eb += 8; dst += dst_step; }
-                if (++cc == cchunks) { cc = 0; ++tap; if (++s == S) { s = 0; ++r; } }
+                if (++term == terms) {
+                    term = 0;
+                    if (++cc == cchunks) { cc = 0; ++tap; if (++s == S) { s = 0; ++r; } }
+                }
             }
         }
     } else if (warp == 1 || warp == 6) {
@@ -364,8 +373,10 @@ __device__ __forceinline__ float round_tf32(float x)
     return __uint_as_float(r);
 }
 
+// With `split` the row holds 2*Cp values: the TF32-rounded value hi at channel c and the rounded remainder
+// lo = rna(x - hi) at channel Cp + c (error-compensated mode: x = hi + lo up to 2^-22 relative).
 __global__ void __launch_bounds__(256)
-pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int C, int Cp, int HW)
+pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int C, int Cp, int HW, int split)
 {
     __shared__ float tile[32][33];
     pdl_launch_dependents();
@@ -374,7 +385,8 @@ pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int
     const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
     const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;          // 32 x 8
     const float* src = in + (size_t)n * C * HW;
-    float* dst = xp + (size_t)n * HW * Cp;
+    const int Cs = split ? 2 * Cp : Cp;
+    float* dst = xp + (size_t)n * HW * Cs;
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int c = c0 + ty + 8 * i, hw = hw0 + tx;
@@ -384,24 +396,33 @@ pack_input_nhwc_kernel(const float* __restrict__ in, float* __restrict__ xp, int
 #pragma unroll
     for (int i = 0; i < 4; ++i) {
         const int hw = hw0 + ty + 8 * i, c = c0 + tx;
-        if (hw < HW) dst[(size_t)hw * Cp + c] = round_tf32(tile[tx][ty + 8 * i]);
+        if (hw < HW) {
+            const float x = tile[tx][ty + 8 * i];
+            const float hi = round_tf32(x);
+            dst[(size_t)hw * Cs + c] = hi;
+            if (split) dst[(size_t)hw * Cs + Cp + c] = round_tf32(x - hi);
+        }
     }
 }
 
 // filters KCRS -> [R*S][K][Cp], TF32-rounded, zero in the padded channels
 __global__ void __launch_bounds__(256)
-pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int Cp, int RS)
+pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int C, int Cp, int RS, int split)
 {
     pdl_launch_dependents();
     pdl_wait();
     const long long total = (long long)RS * K * Cp;
+    const int Cs = split ? 2 * Cp : Cp;
     for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
          idx += (long long)gridDim.x * blockDim.x) {
         const int c = (int)(idx % Cp);
         const long long t = idx / Cp;
         const int k = (int)(t % K);
         const int tap = (int)(t / K);
-        wp[idx] = c < C ? round_tf32(__ldg(filt + ((size_t)k * C + c) * RS + tap)) : 0.f;
+        const float x = c < C ? __ldg(filt + ((size_t)k * C + c) * RS + tap) : 0.f;
+        const float hi = round_tf32(x);
+        wp[t * Cs + c] = hi;
+        if (split) wp[t * Cs + Cp + c] = round_tf32(x - hi);         // see pack_input_nhwc_kernel
     }
 }
 
@@ -540,6 +561,8 @@ struct IgemmPlan {
     int tile_id = 0;
     int BN = 128;
     int Cp = 0;
+    int terms = 1;                   // 3: error-compensated TF32, staged operands hold hi and lo parts (2*Cp channels)
+    int Cs() const { return terms == 3 ? 2 * Cp : Cp; }
     int splits = 1;
     int iters_total = 0, iters_per_split = 0;
     int tiles_m = 0, tiles_n = 0;
@@ -745,8 +768,9 @@ int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 int encode_map_a(IgemmPlan* p, const void* xp)
 {
     const ConvDims& d = p->d;
-    const cuuint64_t dims[4] = {(cuuint64_t)p->Cp, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
-    const cuuint64_t strides[3] = {(cuuint64_t)p->Cp * 4, (cuuint64_t)d.W * p->Cp * 4, (cuuint64_t)d.H * d.W * p->Cp * 4};
+    const cuuint64_t Cs = (cuuint64_t)p->Cs();
+    const cuuint64_t dims[4] = {Cs, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
+    const cuuint64_t strides[3] = {Cs * 4, (cuuint64_t)d.W * Cs * 4, (cuuint64_t)d.H * d.W * Cs * 4};
     const int lower[2] = {-d.pad, -d.pad};                                 // W, H
     const int upper[2] = {d.pad - (d.S - 1), d.pad - (d.R - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)d.stride, (cuuint32_t)d.stride, 1};
@@ -765,8 +789,9 @@ int encode_map_a(IgemmPlan* p, const void* xp)
 int encode_map_b(IgemmPlan* p)
 {
     const ConvDims& d = p->d;
-    const cuuint64_t dims[3] = {(cuuint64_t)p->Cp, (cuuint64_t)d.K, (cuuint64_t)(d.R * d.S)};
-    const cuuint64_t strides[2] = {(cuuint64_t)p->Cp * 4, (cuuint64_t)d.K * p->Cp * 4};
+    const cuuint64_t Cs = (cuuint64_t)p->Cs();
+    const cuuint64_t dims[3] = {Cs, (cuuint64_t)d.K, (cuuint64_t)(d.R * d.S)};
+    const cuuint64_t strides[2] = {Cs * 4, (cuuint64_t)d.K * Cs * 4};
     const cuuint32_t box[3] = {BKC, (cuuint32_t)p->BN, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
     CUresult r = g_encode_tiled(&p->map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, dims, strides, box, estr,
@@ -782,13 +807,14 @@ int encode_map_b(IgemmPlan* p)
 
 }  // namespace
 
-int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out)
+int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out, bool x3)
 {
     if (!igemm_variant_legal(d_in, variant)) return BODA_ERR_UNSUPPORTED;
     // strided tconv layers may run as their stride-1 space-to-depth view
     ConvDims d = d_in;
     bool use_s2d = false;
-    if (variant == BODA_VARIANT_TCONV && s2d != 0) {
+    if (x3 && s2d > 0) return BODA_ERR_UNSUPPORTED;      // the error-compensated mode runs on the im2col kernel only
+    if (variant == BODA_VARIANT_TCONV && s2d != 0 && !x3) {
         ConvDims e;
         const bool can = s2d_view(d_in, &e);
         if (s2d > 0 && !can) return BODA_ERR_UNSUPPORTED;
@@ -820,18 +846,19 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->variant = variant;
     p->d_status = d_status;
     p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
-    p->iters_total = d.R * d.S * (p->Cp / BKC);
+    p->terms = x3 ? 3 : 1;
+    p->iters_total = d.R * d.S * (p->Cp / BKC) * p->terms;
     // tile and split: forced, or the minimum of the cost model
     double best = 1e300;
     int best_t = 2, best_s = 1;
     for (int t = 0; t < kNumIgemmTiles; ++t) {
         if (tile_id >= 0 && t != tile_id) continue;
         const int nacc = kTileNacc[t];
-        if (nacc > 0 && (variant != BODA_VARIANT_TCONV || !halo_geometry(d, kTileBN[t], nacc, nullptr))) continue;
+        if (nacc > 0 && (x3 || variant != BODA_VARIANT_TCONV || !halo_geometry(d, kTileBN[t], nacc, nullptr))) continue;
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
             if (s > p->iters_total) continue;
-            const double c = nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp, kTileBN[t], s);
+            const double c = nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms, kTileBN[t], s);
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
     }
@@ -840,7 +867,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->tile_id = best_t;
     p->BN = kTileBN[best_t];
     p->nacc = kTileNacc[best_t];
-    if (p->nacc > 0 && (variant != BODA_VARIANT_TCONV || !halo_geometry(d, p->BN, p->nacc, p))) { delete p; return BODA_ERR_UNSUPPORTED; }
+    if (p->nacc > 0 && (x3 || variant != BODA_VARIANT_TCONV || !halo_geometry(d, p->BN, p->nacc, p))) { delete p; return BODA_ERR_UNSUPPORTED; }
     p->iters_per_split = (p->iters_total + best_s - 1) / best_s;
     p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;   // no empty split
     p->tiles_n = (d.K + p->BN - 1) / p->BN;
@@ -851,11 +878,11 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     } else {
         p->tiles_m = (d.M + BM - 1) / BM;
-        p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
+        p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cs() * 4) + 1023) & ~(size_t)1023;
         p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     }
 
-    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cp * 4);
+    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cs() * 4);
     if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
     rc = encode_map_b(p);
     if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -882,7 +909,7 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
                       p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits);
         return;
     }
-    std::snprintf(buf, n, "%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->BN, p->tile_id,
+    std::snprintf(buf, n, "%s%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->terms == 3 ? "x3 " : "", p->BN, p->tile_id,
                   p->BN == 64 ? TileCfg<64>::STAGES : p->BN == 96 ? TileCfg<96>::STAGES : p->BN == 128 ? TileCfg<128>::STAGES
                   : p->BN == 192 ? TileCfg<192>::STAGES : TileCfg<256>::STAGES,
                   p->splits, p->tiles_m, p->tiles_n, p->splits);
@@ -899,7 +926,7 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
                                     o.S, o.stride, d.R, d.S, p->Cp));
     } else {
         BODA_CUDA_TRY(launch_kernel(pack_filters_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.C, p->Cp,
-                                    d.R * d.S));
+                                    d.R * d.S, p->terms == 3 ? 1 : 0));
     }
     count_launch();
     return BODA_OK;
@@ -928,7 +955,7 @@ static OutSpec make_out_spec(const IgemmPlan* p, float* out)
 
 bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 {
-    if (p->s2d) return false;                       // the space-to-depth staging reads NCHW only
+    if (p->s2d || p->terms == 3) return false;      // space-to-depth staging and the hi/lo operand split read NCHW only
     if (p->nacc > 0) { *Hp = p->Hp; *Wp = p->Wp; } else { *Hp = p->d.H; *Wp = p->d.W; }
     *Cp = p->Cp;
     return true;
@@ -937,6 +964,7 @@ bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
     if (in_packed && p->s2d) return BODA_ERR_UNSUPPORTED;
+    if ((in_packed || out_packed) && p->terms == 3) return BODA_ERR_UNSUPPORTED;
     if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < p->d.P || oWp < p->d.Q)) return BODA_ERR_INVALID_ARG;
     p->in_packed = in_packed != 0;
     p->out_packed = out_packed ? 1 : 0;
@@ -1002,7 +1030,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     if (!p->s2d && !p->in_packed) {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
-        BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW));
+        BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW, p->terms == 3 ? 1 : 0));
         count_launch();
     }
     if (p->map_a_base != xp) {
@@ -1013,6 +1041,8 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     IgemmParams prm;
     prm.M = d.M; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
     prm.cchunks = p->Cp / BKC;
+    prm.terms = p->terms;
+    prm.lo_off = p->Cp;
     prm.iters_total = p->iters_total;
     prm.iters_per_split = p->iters_per_split;
     prm.splits = p->splits;
@@ -1100,13 +1130,15 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
-        cudaError_t e = launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW);
+        cudaError_t e = launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW, 0);
         if (e != cudaSuccess) { p->d_wp = nullptr; return record_cuda_error(e, "pack_input_nhwc_kernel"); }
         count_launch();
     }
     IgemmParams prm;
     prm.M = d.M; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
     prm.cchunks = p->Cp / BKC;
+    prm.terms = 1;
+    prm.lo_off = 0;
     prm.iters_total = p->iters_total;
     prm.iters_per_split = p->iters_per_split;
     prm.splits = p->splits;

@@ -14,8 +14,10 @@ int igemm_num_tiles();
 int igemm_num_split_candidates();
 int igemm_split_candidate(int i);
 
-// s2d: -1 automatic, 0 never, 1 force the space-to-depth view of a strided tconv layer
-int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out);
+// s2d: -1 automatic, 0 never, 1 force the space-to-depth view of a strided tconv layer.
+// x3: error-compensated TF32 (three tensor-core products per FP32 product; im2col kernel only, NCHW in and out).
+int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out,
+                      bool x3 = false);
 bool igemm_s2d_applicable(const ConvDims& d);
 void igemm_plan_destroy(IgemmPlan* p);
 int igemm_plan_tile(const IgemmPlan* p);
