@@ -341,7 +341,7 @@ def run_ours(args):
     # ---------------- every op on its own, and with it the dominant kernel: op i re-launched in place on the
     # activations of the last step, 20 launches back to back captured in one CUDA graph (so that neither host launch
     # cost nor gaps count), the graph replayed several times between events
-    dom_reps = 20
+    dom_reps = 2 if args.stack_only else 20
     inplace_ms = []
     for i in range(n_ops):
         g = torch.cuda.CUDAGraph()
@@ -417,9 +417,9 @@ def run_ours(args):
         roofline = {"bound": bound, "achieved": round(dom_tf, 3), "peak": round(peak, 2), "unit": "TFLOP/s",
                     "frac": round(dom_tf / peak, 4), "traffic": traffic, "kernel": layers[dom]["op"] + ": " + descs[dom],
                     "peak_source": peak_note, "launch_ms": round(dom_ms, 5),
-                    "timing": f"{dom_reps} back-to-back launches of that layer in place per event pair, L2-warm as inside the step"}
-        per_config = single_layer_configs(B, wl, torch, peaks, flush)
-        sgemm_rows = sgemm_table1(B, torch, peaks)
+                    "timing": f"{dom_reps} launches of that layer in place, back to back in one captured graph, per event pair; L2-warm as inside the step"}
+        per_config = [] if args.stack_only else single_layer_configs(B, wl, torch, peaks, flush)
+        sgemm_rows = [] if args.stack_only else sgemm_table1(B, torch, peaks)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
@@ -454,6 +454,8 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--tune", type=int, default=1, help="time candidate tiles when planning (default on)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--stack-only", action="store_true",
+                    help="skip the single-layer, SGEMM and per-op context measurements (short launch lists for profiling)")
     args = ap.parse_args()
     if args.impl == "reference":
         run_reference(args)

@@ -89,7 +89,9 @@ __device__ __forceinline__ RowDst igemm_row_dst(const IgemmParams& p, int m)
 }
 
 // ------------------------------------------------------------------------------------------------
-template <int BN>
+// X3: the error-compensated mode (three reduction steps per channel chunk); a compile-time switch because the
+// producers' loops set the pace of the main loop and every instruction in them shows in the layer's time.
+template <int BN, bool X3>
 __global__ void __launch_bounds__(kIgemmThreads, 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const IgemmParams p)
@@ -147,35 +149,64 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             // stage's byte count on its full barrier (bytes that land before the count is posted are legal: the
             // barrier's phase cannot complete before its one arrival).  Ring position, parity and addresses advance
             // incrementally: the loops hold no division.
-            const int role = warp == 0 ? 0 : warp == 11 ? 1 : 2;
-            const int n0 = m0 / p.o.PQ;
-            const int rem = m0 - n0 * p.o.PQ;
-            const int p0 = rem / p.o.Q;
-            const int q0 = rem - p0 * p.o.Q;
-            const int w0 = q0 * p.stride - p.pad;
-            const int h0 = p0 * p.stride - p.pad;
-            const int terms = p.terms;
+            // Each role has its own loop with nothing in it that the role does not need: a handful of extra
+            // integer instructions per stage in these loops cost a microsecond per layer (measured).
+            constexpr int terms = X3 ? 3 : 1;
             const int chunk0 = it_begin / terms;
             int term = it_begin - chunk0 * terms;
             int tap = chunk0 / p.cchunks;
-            int cc = chunk0 - tap * p.cchunks;
-            int r = tap / p.S;
-            int s = tap - r * p.S;
+            int cx = (chunk0 - tap * p.cchunks) * BKC;                 // first channel of the chunk
+            const int cend = p.cchunks * BKC;
             uint32_t stage = 0, par = 1;
-            uint32_t fb = full_bar, eb = empty_bar, dst = role == 0 ? smem_a : smem_b;
-            const uint32_t dst0 = dst, dst_step = role == 0 ? (uint32_t)A_STAGE_BYTES : (uint32_t)Cfg::B_STAGE_BYTES;
-            const int cchunks = p.cchunks, S = p.S;
-            for (int i = 0; i < my_iters; ++i) {
-                if (!mbar_wait(eb, par, &s_abort, p.status, 1 + 5 * role)) break;
-                // error-compensated mode: term 0 = hi * hi, term 1 = lo(input) * hi(filter), term 2 = hi(input) * lo(filter)
-                if (role == 0) tma_load_im2col_4d(dst, &map_a, fb, cc * BKC + (term == 1 ? p.lo_off : 0), w0, h0, n0, (uint16_t)s, (uint16_t)r);
-                else if (role == 1) tma_load_3d(dst, &map_b, fb, cc * BKC + (term == 2 ? p.lo_off : 0), k0, tap);
-                else mbar_expect_tx(fb, Cfg::STAGE_BYTES + ((i == 0 && (blockIdx.x | blockIdx.y | blockIdx.z) == 0) ? (uint32_t)p.tx_extra : 0u));
-                if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = dst0; }
-                else { fb += 8; eb += 8; dst += dst_step; }
-                if (++term == terms) {
-                    term = 0;
-                    if (++cc == cchunks) { cc = 0; ++tap; if (++s == S) { s = 0; ++r; } }
+            uint32_t fb = full_bar, eb = empty_bar;
+            if (warp == 0) {
+                // input tiles (A).  error-compensated mode: term 0 = hi * hi, term 1 = lo(input) * hi(filter),
+                // term 2 = hi(input) * lo(filter)
+                const int n0 = m0 / p.o.PQ;
+                const int rem = m0 - n0 * p.o.PQ;
+                const int p0 = rem / p.o.Q;
+                const int q0 = rem - p0 * p.o.Q;
+                const int w0 = q0 * p.stride - p.pad;
+                const int h0 = p0 * p.stride - p.pad;
+                const int S = p.S, lo_off = p.lo_off;
+                int r = tap / S;
+                int s = tap - r * S;
+                uint32_t dst = smem_a;
+                for (int i = 0; i < my_iters; ++i) {
+                    if (!mbar_wait(eb, par, &s_abort, p.status, 1)) break;
+                    tma_load_im2col_4d(dst, &map_a, fb, cx + ((X3 && term == 1) ? lo_off : 0), w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                    if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = smem_a; }
+                    else { fb += 8; eb += 8; dst += A_STAGE_BYTES; }
+                    if (!X3 || ++term == terms) {
+                        term = 0;
+                        cx += BKC;
+                        if (cx == cend) { cx = 0; if (++s == S) { s = 0; ++r; } }
+                    }
+                }
+            } else if (warp == 11) {
+                // filter tiles (B)
+                const int lo_off = p.lo_off;
+                uint32_t dst = smem_b;
+                for (int i = 0; i < my_iters; ++i) {
+                    if (!mbar_wait(eb, par, &s_abort, p.status, 6)) break;
+                    tma_load_3d(dst, &map_b, fb, cx + ((X3 && term == 2) ? lo_off : 0), k0, tap);
+                    if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = smem_b; }
+                    else { fb += 8; eb += 8; dst += Cfg::B_STAGE_BYTES; }
+                    if (!X3 || ++term == terms) {
+                        term = 0;
+                        cx += BKC;
+                        if (cx == cend) { cx = 0; ++tap; }
+                    }
+                }
+            } else {
+                // byte counts
+                uint32_t bytes = Cfg::STAGE_BYTES + ((blockIdx.x | blockIdx.y | blockIdx.z) == 0 ? (uint32_t)p.tx_extra : 0u);
+                for (int i = 0; i < my_iters; ++i) {
+                    if (!mbar_wait(eb, par, &s_abort, p.status, 11)) break;
+                    mbar_expect_tx(fb, bytes);
+                    bytes = Cfg::STAGE_BYTES;
+                    if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; }
+                    else { fb += 8; eb += 8; }
                 }
             }
         }
@@ -192,22 +223,27 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             bool ok = true;
             uint32_t par = 0;
             int stage = lo;
-            const uint64_t da0 = smem_desc_k_sw128(smem_a), db0 = smem_desc_k_sw128(smem_b);
             const uint32_t my_acc = tmem_acc + (uint32_t)(me * BN);
+            // barrier addresses and operand descriptors of the owned stages advance incrementally, like the producers'
+            const uint64_t da_lo = smem_desc_k_sw128(smem_a) + (uint64_t)lo * (A_STAGE_BYTES >> 4);
+            const uint64_t db_lo = smem_desc_k_sw128(smem_b) + (uint64_t)lo * (Cfg::B_STAGE_BYTES >> 4);
+            const uint32_t fb_lo = full_bar + 8 * lo, eb_lo = empty_bar + 8 * lo;
+            const int skip = STAGES - (hi - lo);         // iterations that belong to the other issuer per ring turn
+            uint64_t da = da_lo, db = db_lo;
+            uint32_t fb = fb_lo, eb = eb_lo;
             uint32_t accumulate = 0;
             for (int i = lo; i < my_iters;) {
-                ok = mbar_wait(full_bar + 8 * stage, par, &s_abort, p.status, 2);
+                ok = mbar_wait(fb, par, &s_abort, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
-                const uint64_t da = da0 + (uint64_t)stage * (A_STAGE_BYTES >> 4);
-                const uint64_t db = db0 + (uint64_t)stage * (Cfg::B_STAGE_BYTES >> 4);
 #pragma unroll
                 for (int k = 0; k < BKC / 8; ++k)       // 8 TF32 values = 32 bytes = 2 descriptor units per step
                     umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
                 accumulate = 1u;
-                tc_commit(empty_bar + 8 * stage);       // frees the stage once these MMAs have read it
-                ++stage; ++i;
-                if (stage == hi) { stage = lo; i += STAGES - (hi - lo); par ^= 1u; }
+                tc_commit(eb);                          // frees the stage once these MMAs have read it
+                ++i;
+                if (++stage == hi) { stage = lo; i += skip; par ^= 1u; da = da_lo; db = db_lo; fb = fb_lo; eb = eb_lo; }
+                else { da += A_STAGE_BYTES >> 4; db += Cfg::B_STAGE_BYTES >> 4; fb += 8; eb += 8; }
             }
             tc_commit(accum_bar);                       // this issuer's MMAs have drained
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
@@ -749,20 +785,25 @@ int encode_map_a_halo(IgemmPlan* p, const void* xs)
     return BODA_OK;
 }
 
-template <int BN>
-int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
+template <int BN, bool X3>
+int launch_bn_mode(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 {
     using Cfg = TileCfg<BN>;
     static bool attr_set = false;
     if (!attr_set) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(igemm_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
+        BODA_CUDA_TRY(cudaFuncSetAttribute(igemm_tf32_kernel<BN, X3>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
         attr_set = true;
     }
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
+    BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN, X3>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
                                 p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
+}
+template <int BN>
+int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
+{
+    return prm.terms == 3 ? launch_bn_mode<BN, true>(p, prm, stream) : launch_bn_mode<BN, false>(p, prm, stream);
 }
 
 int encode_map_a(IgemmPlan* p, const void* xp)

@@ -33,11 +33,11 @@ def main() -> None:
     ap.add_argument("--split", type=int, default=0)
     ap.add_argument("--tune", type=int, default=0)
     ap.add_argument("--variant", default="auto", choices=["auto", "direct", "k1conv", "tconv"])
-    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32"])
+    ap.add_argument("--math", default="auto", choices=["auto", "fp32", "tf32", "tf32x3"])
     args = ap.parse_args()
     s = layer_shape(args.layer, args.batch)
     variant = {"auto": -1, "direct": 0, "k1conv": 1, "tconv": 2}[args.variant]
-    math = {"auto": 0, "fp32": 1, "tf32": 2}[args.math]
+    math = {"auto": 0, "fp32": 1, "tf32": 2, "tf32x3": 3}[args.math]
     plan = B.ConvPlan(s.as_tuple(), math=math, variant=variant, tile_id=args.tile, split_k=args.split, tune=args.tune)
     x = torch.from_numpy(wl.half_normal(1, (s.N, s.C, s.H, s.W))).cuda()
     w = torch.from_numpy(wl.normal(2, (s.K, s.C, s.R, s.S), 0.0, (2.0 / (s.C * s.R * s.S)) ** 0.5)).cuda()
