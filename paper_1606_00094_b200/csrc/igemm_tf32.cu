@@ -63,11 +63,11 @@ template <int BN> struct TileCfg {
 #endif
     // MMA issuers: two for the narrower tiles, where one thread's issue cost (about 530 clocks per stage) exceeds
     // the MMA work of a stage (2*BN clocks); one for BN = 256, which is bound by the tensor pipe either way.
-    // Each issuer OWNS a contiguous set of ring stages ([0, SPLIT) and [SPLIT, STAGES)) and walks it in order, so
-    // every barrier has one waiter and a wait can never alias a phase that its issuer has not seen yet.
+    // The issuers take alternate reduction steps (even / odd), so that one issues while the other's MMAs run.  Every
+    // stage has one full barrier per issuer: with an odd number of stages a stage changes hands on every turn of the
+    // ring, and a barrier shared by both issuers could be read one phase early by the issuer that runs ahead.
     static constexpr int ISSUERS = BN <= BODA_IGEMM_DUAL_ISSUE_MAX_BN ? 2 : 1;
     static constexpr int STAGES = (200 * 1024) / STAGE_BYTES > 8 ? 8 : (200 * 1024) / STAGE_BYTES;
-    static constexpr int SPLIT = ISSUERS == 2 ? (STAGES + 1) / 2 : STAGES;   // first stage of the second issuer
     static_assert(STAGES >= 2, "both issuers need a stage");
     static constexpr int ACC_COLS = ISSUERS * BN;                                         // one accumulator per issuer
     static constexpr int TMEM_COLS = ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
@@ -103,9 +103,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t smem_a = smem_base;
     const uint32_t smem_b = smem_base + STAGES * A_STAGE_BYTES;
     const uint32_t bars = smem_base + STAGES * Cfg::STAGE_BYTES;
-    const uint32_t full_bar = bars;                    // STAGES x 8 bytes
-    const uint32_t empty_bar = bars + 8 * STAGES;
-    const uint32_t accum_bar = bars + 16 * STAGES;
+    const uint32_t full_bar = bars;                    // STAGES x 2 x 8 bytes: [stage][issuer]
+    const uint32_t empty_bar = bars + 16 * STAGES;
+    const uint32_t accum_bar = bars + 24 * STAGES;
     const uint32_t recv_bar = accum_bar + 8;           // split reduction: bytes pushed by the cluster peers
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
@@ -123,7 +123,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
         s_abort = 0;
-        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 8 * s, 1); mbar_init(empty_bar + 8 * s, 1); }
+        for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 16 * s, 1); mbar_init(full_bar + 16 * s + 8, 1); mbar_init(empty_bar + 8 * s, 1); }
         mbar_init(accum_bar, Cfg::ISSUERS);           // one arrival per MMA issuer
         mbar_init(recv_bar, 1);
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
@@ -158,7 +158,9 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             int cx = (chunk0 - tap * p.cchunks) * BKC;                 // first channel of the chunk
             const int cend = p.cchunks * BKC;
             uint32_t stage = 0, par = 1;
-            uint32_t fb = full_bar, eb = empty_bar;
+            // full barrier of local reduction step i: [stage][i & 1] with two issuers, [stage][0] with one
+            constexpr uint32_t FLIP = Cfg::ISSUERS == 2 ? 8u : 0u;
+            uint32_t fb = full_bar, eb = empty_bar, fsel = 0;      // fb: the stage's pair of full barriers; fsel: which of them
             if (warp == 0) {
                 // input tiles (A).  error-compensated mode: term 0 = hi * hi, term 1 = lo(input) * hi(filter),
                 // term 2 = hi(input) * lo(filter)
@@ -174,9 +176,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 uint32_t dst = smem_a;
                 for (int i = 0; i < my_iters; ++i) {
                     if (!mbar_wait(eb, par, &s_abort, p.status, 1)) break;
-                    tma_load_im2col_4d(dst, &map_a, fb, cx + ((X3 && term == 1) ? lo_off : 0), w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                    tma_load_im2col_4d(dst, &map_a, fb + fsel, cx + ((X3 && term == 1) ? lo_off : 0), w0, h0, n0, (uint16_t)s, (uint16_t)r);
+                    fsel ^= FLIP;
                     if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = smem_a; }
-                    else { fb += 8; eb += 8; dst += A_STAGE_BYTES; }
+                    else { fb += 16; eb += 8; dst += A_STAGE_BYTES; }
                     if (!X3 || ++term == terms) {
                         term = 0;
                         cx += BKC;
@@ -189,9 +192,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 uint32_t dst = smem_b;
                 for (int i = 0; i < my_iters; ++i) {
                     if (!mbar_wait(eb, par, &s_abort, p.status, 6)) break;
-                    tma_load_3d(dst, &map_b, fb, cx + ((X3 && term == 2) ? lo_off : 0), k0, tap);
+                    tma_load_3d(dst, &map_b, fb + fsel, cx + ((X3 && term == 2) ? lo_off : 0), k0, tap);
+                    fsel ^= FLIP;
                     if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; dst = smem_b; }
-                    else { fb += 8; eb += 8; dst += Cfg::B_STAGE_BYTES; }
+                    else { fb += 16; eb += 8; dst += Cfg::B_STAGE_BYTES; }
                     if (!X3 || ++term == terms) {
                         term = 0;
                         cx += BKC;
@@ -203,36 +207,35 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 uint32_t bytes = Cfg::STAGE_BYTES + ((blockIdx.x | blockIdx.y | blockIdx.z) == 0 ? (uint32_t)p.tx_extra : 0u);
                 for (int i = 0; i < my_iters; ++i) {
                     if (!mbar_wait(eb, par, &s_abort, p.status, 11)) break;
-                    mbar_expect_tx(fb, bytes);
+                    mbar_expect_tx(fb + fsel, bytes);
                     bytes = Cfg::STAGE_BYTES;
+                    fsel ^= FLIP;
                     if (++stage == (uint32_t)STAGES) { stage = 0; par ^= 1u; fb = full_bar; eb = empty_bar; }
-                    else { fb += 8; eb += 8; }
+                    else { fb += 16; eb += 8; }
                 }
             }
         }
     } else if (warp == 1 || warp == 6) {
         if (lane == 0 && (warp == 1 || Cfg::ISSUERS == 2)) {
             const int me = warp == 1 ? 0 : 1;
-            // ---------------- MMA issuers: warp 1 owns ring stages [0, SPLIT), warp 6 the rest.  One thread needs
-            // about 530 clocks per stage (barrier hand-shake plus four MMA issues); two threads share that, so the
-            // tensor pipe itself becomes the limit for BN >= 128.  Each issuer accumulates into its own TMEM
-            // accumulator (columns [0, BN) and [BN, 2*BN)); the epilogue adds the two, so the summation order - and
-            // with it every output bit - is the same in every run.
+            // ---------------- MMA issuers: warp 1 takes the even reduction steps, warp 6 the odd ones.  One thread
+            // needs about 430 clocks per stage (barrier test, four MMA issues, commit) - more than the MMAs take for
+            // BN <= 192 - so with two issuers one issues while the other's MMAs run.  Each issuer accumulates into its
+            // own TMEM accumulator (columns [0, BN) and [BN, 2*BN)); the epilogue adds the two, so the summation
+            // order - and with it every output bit - is the same in every run.
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
-            const int lo = me == 0 ? 0 : Cfg::SPLIT, hi = me == 0 ? Cfg::SPLIT : STAGES;
+            constexpr int STEP = Cfg::ISSUERS;                          // stages between two steps of one issuer
+            // an issuer returns to a barrier after CYCLE of its own steps: then the barrier's phase has advanced
+            constexpr int CYCLE = (STEP == 2 && STAGES % 2 == 0) ? STAGES / 2 : STAGES;
             bool ok = true;
             uint32_t par = 0;
-            int stage = lo;
+            int stage = me, visited = 0;
             const uint32_t my_acc = tmem_acc + (uint32_t)(me * BN);
-            // barrier addresses and operand descriptors of the owned stages advance incrementally, like the producers'
-            const uint64_t da_lo = smem_desc_k_sw128(smem_a) + (uint64_t)lo * (A_STAGE_BYTES >> 4);
-            const uint64_t db_lo = smem_desc_k_sw128(smem_b) + (uint64_t)lo * (Cfg::B_STAGE_BYTES >> 4);
-            const uint32_t fb_lo = full_bar + 8 * lo, eb_lo = empty_bar + 8 * lo;
-            const int skip = STAGES - (hi - lo);         // iterations that belong to the other issuer per ring turn
-            uint64_t da = da_lo, db = db_lo;
-            uint32_t fb = fb_lo, eb = eb_lo;
+            const uint64_t da0 = smem_desc_k_sw128(smem_a), db0 = smem_desc_k_sw128(smem_b);
+            uint64_t da = da0 + (uint64_t)me * (A_STAGE_BYTES >> 4), db = db0 + (uint64_t)me * (Cfg::B_STAGE_BYTES >> 4);
+            uint32_t fb = full_bar + 16 * me + 8 * me, eb = empty_bar + 8 * me;
             uint32_t accumulate = 0;
-            for (int i = lo; i < my_iters;) {
+            for (int i = me; i < my_iters; i += STEP) {
                 ok = mbar_wait(fb, par, &s_abort, p.status, 2);
                 if (!ok) break;
                 tc_fence_after();
@@ -241,9 +244,16 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
                 accumulate = 1u;
                 tc_commit(eb);                          // frees the stage once these MMAs have read it
-                ++i;
-                if (++stage == hi) { stage = lo; i += skip; par ^= 1u; da = da_lo; db = db_lo; fb = fb_lo; eb = eb_lo; }
-                else { da += A_STAGE_BYTES >> 4; db += Cfg::B_STAGE_BYTES >> 4; fb += 8; eb += 8; }
+                stage += STEP;
+                if (stage >= STAGES) {
+                    stage -= STAGES;
+                    da -= (uint64_t)(STAGES - STEP) * (A_STAGE_BYTES >> 4); db -= (uint64_t)(STAGES - STEP) * (Cfg::B_STAGE_BYTES >> 4);
+                    fb -= 16 * (STAGES - STEP); eb -= 8 * (STAGES - STEP);
+                } else {
+                    da += (uint64_t)STEP * (A_STAGE_BYTES >> 4); db += (uint64_t)STEP * (Cfg::B_STAGE_BYTES >> 4);
+                    fb += 16 * STEP; eb += 8 * STEP;
+                }
+                if (++visited == CYCLE) { visited = 0; par ^= 1u; }
             }
             tc_commit(accum_bar);                       // this issuer's MMAs have drained
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
@@ -269,7 +279,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-        const bool two_acc = Cfg::ISSUERS == 2 && my_iters > Cfg::SPLIT;   // a shorter reduction never reaches the second issuer's stages
+        const bool two_acc = Cfg::ISSUERS == 2 && my_iters >= 2;   // a single reduction step never reaches the second issuer
         // 32 accumulator columns of this thread's row (the sum of the two issuers' accumulators)
         auto load32 = [&](int j0, uint32_t (&v)[32]) {
             tmem_ld_32cols(trow + j0, v);
