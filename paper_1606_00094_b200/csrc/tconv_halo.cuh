@@ -26,7 +26,7 @@ namespace halo {
 
 using namespace tc;
 
-constexpr int kThreads = 352;      // warp 0 producer, 1 and 6 MMA issuers, 2..5 and 7..10 epilogue
+constexpr int kThreads = 416;      // warp 0 producer; 1, 6, 11, 12 MMA issuers; 2..5 and 7..10 epilogue
 constexpr int kMaxBStages = 8;
 constexpr int kASlots = 2;
 constexpr int kSmemBudget = 200 * 1024;
@@ -67,9 +67,10 @@ struct HaloCfg {
     static constexpr int ACC_COLS = BN * NACC;
     static constexpr int TMEM_COLS = ACC_COLS <= 32 ? 32 : ACC_COLS <= 64 ? 64 : ACC_COLS <= 128 ? 128 : ACC_COLS <= 256 ? 256 : 512;
     static_assert(ACC_COLS <= 512, "accumulators exceed tensor memory");
-    // One thread can issue an MMA about every 70 clocks; two threads in different warps, each feeding its own
-    // accumulators, reach about 50 (measured).  With two or more accumulators the work is split between two issuers.
-    static constexpr int ISSUERS = NACC >= 2 ? 2 : 1;
+    // One thread can issue an MMA about every 70 clocks; threads in different warps, each feeding its own
+    // accumulators, reach about 50 each (measured).  A reduction step of this kernel is 4 MMAs per accumulator, which
+    // the tensor pipe finishes in 8*BN/4 clocks: with one issuer per accumulator the pipe, not the issue, is the limit.
+    static constexpr int ISSUERS = NACC >= 4 ? 4 : NACC >= 2 ? 2 : 1;
 };
 
 template <int BN, int NACC>
@@ -151,11 +152,12 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (++tap == p.taps) { tap = 0; cx += 32; need_slab = true; }
             }
         }
-    } else if (warp == 1 || warp == 6) {
-        if (lane == 0 && (warp == 1 || Cfg::ISSUERS == 2)) {
-            // ---------------- MMA issuer(s): warp 1 feeds the first half of the accumulators, warp 6 the second half
+    } else if (warp == 1 || warp == 6 || warp >= 11) {
+        const int issuer = warp == 1 ? 0 : warp == 6 ? 1 : warp - 9;          // warps 1, 6, 11, 12
+        if (lane == 0 && issuer < Cfg::ISSUERS) {
+            // ---------------- MMA issuers: each feeds its own share of the accumulators
             constexpr int ACC_PER = NACC / Cfg::ISSUERS;
-            const int acc0 = warp == 1 ? 0 : ACC_PER;
+            const int acc0 = issuer * ACC_PER;
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
             const int chunk0 = it_begin / p.taps;
             int tap = it_begin - chunk0 * p.taps;
@@ -235,13 +237,20 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             constexpr uint32_t TILE_BYTES = 128u * out_tile_row_bytes<BN>();
             const int nbuf = (int)((uint32_t)(kASlots * p.a_slot_bytes + p.b_stages * Cfg::B_STAGE_BYTES) / TILE_BYTES);
             const bool bulk = p.o.packed && nbuf >= (NACC == 1 ? 1 : 2);      // with several accumulators: a buffer per group
-            int turn = 0;
+            // Which accumulator and which tile buffer a group takes on its turn.  One accumulator: both groups share
+            // it (column halves) and buffer 0.  Two: one each.  Four: with three buffers group 0 takes accumulators
+            // 0 and 3 through buffer 0 and group 1 takes 1 and 2 through buffers 1 and 2, so that only one of the four
+            // tiles waits for an earlier copy to leave its buffer; with two buffers each group reuses its own.
+            const bool three = NACC == 4 && nbuf >= 3;
+            constexpr int TURNS = NACC == 1 ? 1 : NACC / 2;
 #pragma unroll 1
-            for (int acc = (NACC == 1 ? 0 : group); acc < NACC; acc += (NACC == 1 ? 1 : 2), ++turn) {
+            for (int turn = 0; turn < TURNS; ++turn) {
+                const int acc = NACC == 1 ? 0 : !three ? group + 2 * turn : group == 0 ? 3 * turn : 1 + turn;
+                const int buf = NACC == 1 ? 0 : !three ? group : group == 0 ? 0 : 1 + turn;
+                const bool reuse = turn > 0 && !(three && group == 1);
                 const RowDst d = halo_row_dst(p, f0 + acc * 128 + row);
-                const uint32_t row_addr = smem_base + (NACC == 1 ? 0u : (uint32_t)group * TILE_BYTES)
-                                        + (uint32_t)row * out_tile_row_bytes<BN>();
-                if (bulk && turn > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+                const uint32_t row_addr = smem_base + (uint32_t)buf * TILE_BYTES + (uint32_t)row * out_tile_row_bytes<BN>();
+                if (bulk && reuse) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
 #pragma unroll 1
                 for (int c = c_begin; c < c_end; ++c) {
                     uint32_t v[32];
