@@ -127,6 +127,20 @@ def time_oracle(batch: int, reps: int):
     return wl.stack_flops(batch) / best / 1e9, best, orc.num_threads()
 
 
+def time_oracle_one_thread(batch: int = 2):
+    """The same oracle on ONE host thread (a fresh interpreter with OMP_NUM_THREADS=1), on `batch` images."""
+    import subprocess
+    env = dict(os.environ, OMP_NUM_THREADS="1")
+    code = "import bench; v, t, n = bench.time_oracle(%d, 1); print(v, t, n)" % batch
+    try:
+        res = subprocess.run([sys.executable, "-c", code], env=env, cwd=os.path.dirname(os.path.abspath(__file__)),
+                             capture_output=True, text=True, timeout=300)
+        v, t, n = res.stdout.split()[-3:]
+        return float(v), float(t), int(n)
+    except Exception:
+        return None, None, 0
+
+
 def max_over_ranks(values, world: int, device: str):
     """Each rank passes its own device-measured times; every rank gets the maximum over all ranks."""
     import torch
@@ -421,6 +435,7 @@ def run_ours(args):
         per_config = [] if args.stack_only else single_layer_configs(B, wl, torch, peaks, flush)
         sgemm_rows = [] if args.stack_only else sgemm_table1(B, torch, peaks)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
+        cpu1_v, cpu1_t, _ = time_oracle_one_thread(2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
             "metric": METRIC, "value": round(value, 1), "unit": UNIT, "n_gpus": world, "steps": args.steps,
             "warmup": max(args.warmup, 3), "ms_per_step": round(ms_per_step, 5), "higher_is_better": True,
@@ -434,7 +449,9 @@ def run_ours(args):
             "clocks": clocks,
             "roofline": roofline,
             "cpu_baseline": {"value": round(cpu_v, 2) if cpu_v else None, "unit": UNIT, "cores": cpu_threads,
-                             "kind": "oracle", "sample": f"the whole batch-{BATCH} stack, best of 2 ({cpu_t:.2f} s)" if cpu_t else "skipped"},
+                             "kind": "oracle", "sample": f"the whole batch-{BATCH} stack, best of 2 ({cpu_t:.2f} s)" if cpu_t else "skipped",
+                             "one_thread": {"value": round(cpu1_v, 2) if cpu1_v else None, "unit": UNIT,
+                                            "sample": f"2 of the {BATCH} images, one run ({cpu1_t:.2f} s)" if cpu1_t else "skipped"}},
             "layers": layers,
             "single_layer_configs": per_config,
             "sgemm_table1": sgemm_rows,
