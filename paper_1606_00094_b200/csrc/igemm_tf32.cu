@@ -966,6 +966,26 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
                   p->splits, p->tiles_m, p->tiles_n, p->splits);
 }
 
+// 1x1 filters with C a multiple of 4 are already [K][C] rows: the staging is a rounding copy, 16 bytes per thread
+__global__ void __launch_bounds__(256)
+pack_filters_1x1_kernel(const float4* __restrict__ filt, float* __restrict__ wp, int K, int C4, int Cp, int split)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int Cs = split ? 2 * Cp : Cp, Cp4 = Cp >> 2;
+    const int total = K * Cp4;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int k = idx / Cp4, c4 = idx - k * Cp4;
+        const float4 x = c4 < C4 ? __ldg(filt + (size_t)k * C4 + c4) : make_float4(0.f, 0.f, 0.f, 0.f);
+        const float4 hi = make_float4(round_tf32(x.x), round_tf32(x.y), round_tf32(x.z), round_tf32(x.w));
+        float* row = wp + (size_t)k * Cs;
+        reinterpret_cast<float4*>(row)[c4] = hi;
+        if (split)
+            reinterpret_cast<float4*>(row + Cp)[c4] = make_float4(round_tf32(x.x - hi.x), round_tf32(x.y - hi.y),
+                                                                  round_tf32(x.z - hi.z), round_tf32(x.w - hi.w));
+    }
+}
+
 static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
 {
     const ConvDims& d = p->d;
@@ -975,6 +995,10 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
         const ConvDims& o = p->orig;
         BODA_CUDA_TRY(launch_kernel(pack_filters_s2d_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, o.K, o.C, o.R,
                                     o.S, o.stride, d.R, d.S, p->Cp));
+    } else if (d.R * d.S == 1 && d.C % 4 == 0 && ((uintptr_t)filt & 15) == 0 && (long long)d.K * p->Cp < (1LL << 31)) {
+        const int blocks4 = (int)std::min<long long>((total / 4 + 255) / 256, 148 * 8);
+        BODA_CUDA_TRY(launch_kernel(pack_filters_1x1_kernel, dim3(blocks4), dim3(256), 0, stream, 1,
+                                    reinterpret_cast<const float4*>(filt), p->d_wp, d.K, d.C / 4, p->Cp, p->terms == 3 ? 1 : 0));
     } else {
         BODA_CUDA_TRY(launch_kernel(pack_filters_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.C, p->Cp,
                                     d.R * d.S, p->terms == 3 ? 1 : 0));
