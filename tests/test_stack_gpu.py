@@ -25,15 +25,18 @@ def _oracle_chain(x, params, ops):
     return outs
 
 
-@pytest.mark.parametrize("batch,math,tol", [(2, 0, TF32_TOL), (1, 1, FP32_TOL), (20, 0, TF32_TOL)])
-def test_stack_every_layer_matches_fp64_chain(batch, math, tol):
+# (20, auto, tuned) is the launch configuration bench.py times; math 3 is the error-compensated TF32 mode, which
+# must hold the FP32 bar through the whole chain (its layers hand over in NCHW)
+@pytest.mark.parametrize("batch,math,tol,tune", [(2, 0, TF32_TOL, 0), (1, 1, FP32_TOL, 0), (20, 0, TF32_TOL, 0),
+                                                 (20, 0, TF32_TOL, 1), (2, 3, FP32_TOL, 0)])
+def test_stack_every_layer_matches_fp64_chain(batch, math, tol, tune):
     import torch
     from paper_1606_00094_b200 import binding as B
     from paper_1606_00094_b200.stack import ConvStack
     ops = wl.alexnet_stack(batch)
     x, params = wl.stack_tensors(batch)
     ref = _oracle_chain(x, params, ops)
-    stack = ConvStack(ops, params, math=math)
+    stack = ConvStack(ops, params, math=math, tune=tune)
     try:
         dx = torch.from_numpy(x).cuda()
         out_graph = stack.forward(dx).clone()            # first call: eager pass + graph capture + launch
@@ -57,6 +60,8 @@ def test_stack_every_layer_matches_fp64_chain(batch, math, tol):
         assert torch.equal(eager, out_graph)
         if math == 0:
             assert any("tconv" in d for d in descs)
+        elif math == 3:
+            assert any("tf32x3" in d for d in descs)
         else:
             assert all("direct" in d or "maxpool" in d for d in descs)
         assert stack.kernels_per_forward() >= len(ops)
