@@ -73,7 +73,10 @@ typedef struct boda_conv_shape {
 
 typedef struct boda_plan_opts {
     int math;                    /* BODA_MATH_* */
-    int tune;                    /* 0: pick variant and tile by rule; 1: time the candidates on the device (synchronises) */
+    int tune;                    /* 0: pick variant and tile by rule; 1: time the candidates on the device (synchronises):
+                                    every tile and split of the rule's variant and, where `variant` and `math` are
+                                    left automatic, of the alternative variant too (FP32 kernel against tensor-core
+                                    kernel, a strided TCONV layer with and without its space-to-depth view) */
     int variant;                 /* BODA_VARIANT_AUTO or a forced variant (used by tests) */
     int tile_id;                 /* -1: automatic; otherwise index into the variant's tile table */
     int split_k;                 /* 0: automatic; otherwise the number of reduction splits of a tensor-core variant */
@@ -98,9 +101,11 @@ void boda_plan_opts_default(boda_plan_opts* opts);
  * Variant selection and blocking for one layer shape: the analogue of the paper's flow
  * "operation -> variant -> blocking constants" (Section 4, Figure "codegen", and the variant rules
  * of Section 5: k1conv for kernel size 1, tconv for kernel sizes 2..11, conv otherwise).  With
- * opts->tune != 0 the legal candidates are timed on scratch buffers and the fastest is kept (the
- * automated tuning the paper names as future work); this synchronises the device.  If the environment variable
- * BODA_TUNE_CACHE names a file, tuned choices are read from and appended to it (one text line per shape).
+ * opts->tune != 0 the legal candidates are timed on scratch buffers (ten calls captured in a CUDA graph,
+ * best of three replays) and the fastest is kept (the automated tuning the paper names as future work);
+ * this allocates, launches and synchronises, so it must not run while a stream is being captured.  If the
+ * environment variable BODA_TUNE_CACHE names a file, tuned choices are read from and appended to it (one
+ * text line "shape-and-options tile split variant s2d" per tuned shape).
  * `opts` may be NULL (defaults).  On success *plan owns device memory (index tables, packed filter
  * storage, workspace); destroy it with boda_conv_plan_destroy.
  * Errors: INVALID_ARG (bad shape), UNSUPPORTED (forced variant illegal, device not sm_100), CUDA, NOMEM.
