@@ -10,10 +10,12 @@
 //            the tap offset (s, r) and fills out-of-image pixels with zeros (= the padding);
 //   B tile  [BN channels][32 channels] <- TMA tiled load from tap-major filters [R*S][K][C].
 // k1conv (kernel size 1) is the same kernel with a single tap: a plain GEMM over C.
-// Roles inside the CTA (192 threads): warp 0 = TMA producer (one elected lane), warp 1 = TMEM owner and
-// MMA issuer (one elected lane issues tcgen05.mma, tcgen05.commit releases shared-memory stages),
-// warps 2..5 = epilogue (tcgen05.ld of the accumulator, bias, ReLU, store).  This is Listing 1's
-// "load block / fma block / store block" loop with hardware pipelines in place of barriers.
+// Roles inside the CTA (416 threads, 13 warps): warps 0, 11, 12 = producers (one elected lane each: input tile
+// TMA, filter tile TMA, byte counts), warps 1 and 6 = MMA issuers (one elected lane each issues tcgen05.mma on
+// alternate reduction steps into its own accumulator; tcgen05.commit releases shared-memory stages; warp 1 also
+// owns the tensor-memory allocation), warps 2..5 and 7..10 = epilogue (tcgen05.ld of the accumulators, bias,
+// ReLU, store or split reduction).  This is Listing 1's "load block / fma block / store block" loop with
+// hardware pipelines in place of barriers.
 // Every wait is bounded (4e9 SM cycles, about two seconds): on expiry the kernel records BODA_ERR_DEVICE_TIMEOUT in the
 // status word, all roles leave their loops, tensor memory is released and the CTA returns.
 #include <cuda.h>
@@ -308,7 +310,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     float y[32];
                     bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
                     if (p.o.packed) out_tile_put32(row_addr, 32 * c, y);
-                    else store_row32(p.o, d, k0 + 32 * c, y, 0u);
+                    else store_row32(p.o, d, k0 + 32 * c, y);
                 }
                 if (p.o.packed) {
                     fence_proxy_async_smem();
@@ -369,7 +371,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
                     bias_relu32(v, s_bias + rank * per + c0, p.o.relu != 0, y);
-                    store_row32(p.o, d, k0 + rank * per + c0, y, 0u);
+                    store_row32(p.o, d, k0 + rank * per + c0, y);
                 }
             }
         } else if (ok) {
@@ -396,7 +398,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             cluster_sync_all();
             if (warp >= 2 && warp <= 5 && s_abort == 0) {
                 const int row = (warp & 3) * 32 + lane;
-                cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias, 0u);
+                cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, igemm_row_dst(p, m0 + row), p.o, k0, s_bias);
             }
         }
         cluster_sync_all();          // nobody leaves while a peer may still read or write its shared memory

@@ -284,8 +284,8 @@ __device__ __forceinline__ RowDst row_dst(const OutSpec& o, bool valid, int n, i
 
 // 32 consecutive output channels kc .. kc+31 of one output row (one row per lane; bias and ReLU already applied).
 // NCHW: lane = pixel, so each of the 32 stores of a lane joins its neighbours' into one 128-byte line.
-// Staged layout: see below.  (`tile` is a per-warp shared-memory scratch address, currently unused.)
-__device__ __forceinline__ void store_row32(const OutSpec& o, const RowDst& d, int kc, const float (&y)[32], uint32_t tile)
+// Staged layout: see below.
+__device__ __forceinline__ void store_row32(const OutSpec& o, const RowDst& d, int kc, const float (&y)[32])
 {
     if (o.packed) {
         // channels are innermost: the lane's 32 values are 128 contiguous bytes; four 32-byte stores, each a whole sector
@@ -299,7 +299,6 @@ __device__ __forceinline__ void store_row32(const OutSpec& o, const RowDst& d, i
                                 "f"(round_to_tf32(y[8 * g + 5])), "f"(round_to_tf32(y[8 * g + 6])), "f"(round_to_tf32(y[8 * g + 7]))
                              : "memory");
         }
-        (void)tile;
     } else if (d.valid) {
         float* oj = o.out + d.base + (size_t)kc * o.PQ;
         if (kc + 32 <= o.K) {
@@ -330,7 +329,7 @@ __device__ __forceinline__ void stash_row32(uint32_t stash, int row, int j0, con
 // keeps 32 loads per peer in flight.
 template <int BN>
 __device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int row, uint32_t rank, int splits, const RowDst& d,
-                                                     const OutSpec& o, int k0, const float* s_bias, uint32_t tile)
+                                                     const OutSpec& o, int k0, const float* s_bias)
 {
     const int per = ((((BN + splits - 1) / splits) + 31) / 32) * 32;
     const int c_begin = (int)rank * per;
@@ -359,7 +358,7 @@ __device__ __forceinline__ void cluster_reduce_store(uint32_t stash, int row, ui
             for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
             bias_relu32(v, s_bias + c0, o.relu != 0, y);
         }
-        store_row32(o, d, k0 + c0, y, tile);
+        store_row32(o, d, k0 + c0, y);
     }
 }
 

@@ -14,9 +14,10 @@
 //   for every tap, issues the MMAs with the A descriptor advanced by (r*Wp + s) rows of 128 bytes.
 //   Positions with p >= P or q >= Q are computed and dropped (for the AlexNet shapes: 7..16 % of the rows).
 //
-// NACC = 2 keeps two 128-row accumulators in tensor memory so that every filter tile fetched from L2 feeds
-// 256 output rows: operand traffic per MMA cycle halves again.
-// Roles, pipeline and bounded waits are those of the im2col kernel (igemm_tf32.cu).
+// NACC = 2 or 4 keeps that many 128-row accumulators in tensor memory so that every filter tile fetched from L2
+// feeds 256 or 512 output rows: operand traffic per MMA cycle halves again, and again.
+// Roles (416 threads): warp 0 = TMA producer, warps 1, 6, 11, 12 = MMA issuers (as many as the tile uses),
+// warps 2..5 and 7..10 = epilogue.  Pipeline and bounded waits are those of the im2col kernel (igemm_tf32.cu).
 #pragma once
 
 #include "tc_ptx.cuh"
@@ -259,7 +260,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     float y[32];
                     bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
                     if (bulk) out_tile_put32(row_addr, 32 * c, y);
-                    else store_row32(p.o, d, k0 + 32 * c, y, 0u);
+                    else store_row32(p.o, d, k0 + 32 * c, y);
                 }
                 if (bulk) {
                     fence_proxy_async_smem();
@@ -296,7 +297,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
             cluster_sync_all();
             if (warp >= 2 && warp <= 5 && ok)
-                cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row), p.o, k0, s_bias, smem_base + (uint32_t)(BN * 512) + (uint32_t)(warp & 3) * 4224u);
+                cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row), p.o, k0, s_bias);
             cluster_sync_all();      // peers are done with this CTA's shared memory
         }
     }
