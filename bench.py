@@ -238,8 +238,10 @@ def single_layer_configs(B, wl, torch, peaks, flush):
 def sgemm_table1(B, torch, peaks):
     """boda_sgemm on the square sizes of the paper's Table 1 (context, not the headline): device time per call
     from a captured graph of 20 calls, operands L2-warm."""
+    # the paper's own column of Table 1 (Boda-RTC on a Titan X, 2016, fp32 SIMT): context, not a target
+    paper_gflops = {128: 114, 256: 619, 384: 1410, 512: 2240, 768: 3550, 1024: 3570, 1536: 4440, 2048: 4210}
     out = []
-    for n in (128, 256, 512, 1024, 2048):
+    for n in (128, 256, 384, 512, 768, 1024, 1536, 2048):
         a = torch.randn((n, n), dtype=torch.float32, device="cuda")
         b = torch.randn((n, n), dtype=torch.float32, device="cuda")
         c = torch.empty((n, n), dtype=torch.float32, device="cuda")
@@ -250,7 +252,8 @@ def sgemm_table1(B, torch, peaks):
         tf = 2.0 * n * n * n / us / 1e6
         out.append({"n": n, "us_per_call": round(us, 2), "gflops": round(tf * 1e3, 1),
                     "flops_per_byte": round(2.0 * n * n * n / (12.0 * n * n), 1),
-                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4)})
+                    "frac_of_tf32_peak": round(tf / (0.5 * peaks["bf16_tflops"]), 4),
+                    "paper_table1_boda_titanx_gflops": paper_gflops[n]})
     return out
 
 

@@ -28,7 +28,7 @@ def _run(A, Bm):
 
 
 # Table 1 of the paper lists square problems 128 ... 2048 (the largest two are checked on sampled rows below)
-@pytest.mark.parametrize("n", [128, 256, 512, 1024])
+@pytest.mark.parametrize("n", [128, 256, 384, 512, 768, 1024])
 def test_table1_square_sizes(n):
     A = wl.normal(0x5601 + n, (n, n))
     Bm = wl.normal(0x5602 + n, (n, n))
