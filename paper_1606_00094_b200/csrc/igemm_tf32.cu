@@ -30,6 +30,7 @@
 #include "igemm_tf32.h"
 #include "tc_ptx.cuh"
 #include "tconv_halo.cuh"
+#include "gconv_tf32.cuh"
 
 namespace boda {
 namespace {
@@ -593,8 +594,10 @@ int load_driver_entry_points()
 
 // Tile table.  Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
 // with NACC accumulators of 128 rows each (ids 5..8: 1, 9..12: 2, 13..15: 4).
-constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128};
-constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4};
+// accumulators per tile: 0 = im2col kernel, 1 / 2 / 4 = halo kernel, -1 = gather kernel (gconv_tf32.cuh)
+constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1};
+constexpr int kFirstGatherTile = 16;
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
 constexpr int kFirstHaloTile = 5;
 constexpr int kSplitCandidates[] = {1, 2, 3, 4, 6, 8};
@@ -625,8 +628,12 @@ struct IgemmPlan {
     int tx_extra = 0;                // test hook (BODA_TEST_TX_MISMATCH): makes one bounded wait of one CTA expire
     bool in_packed = false;          // the input already is this plan's staged layout: skip the staging kernel
     int out_packed = 0, oHp = 0, oWp = 0, oCp = 0;
+    // gather kernel only
+    int2* d_tab = nullptr;           // per reduction index: element offset and tap
+    int gather_chunks = 0;           // ceil(C*R*S / 32)
+    int sm_count = 148;
     // halo kernel only
-    int nacc = 0;                    // 0: im2col kernel; 1 or 2: halo kernel with that many accumulators
+    int nacc = 0;                    // 0: im2col kernel; 1, 2 or 4: halo kernel with that many accumulators; -1: gather kernel
     int Hp = 0, Wp = 0, lead = 0, slab_rows = 0, nbox = 0, box_rows = 0, a_slot_bytes = 0, b_stages = 0;
 };
 
@@ -699,7 +706,10 @@ bool igemm_variant_profitable(const ConvDims& d)
     // layers stay on the FP32 kernel.
     if (d.K < 16 || (long long)d.M * d.K < 128 * 64) return false;
     const int Cp = ((d.C + BKC - 1) / BKC) * BKC;
-    return std::max((double)d.C / Cp, s2d_efficiency(d)) >= 0.2;     // measured: C = 8 of 32 wins, C = 3 of 32 loses
+    // measured: staged input with C = 8 of 32 channels wins, C = 3 of 32 loses; the gather kernel needs no staged input
+    // (tiny layers stay on the FP32 kernel: one 3 us launch beats the tensor-core kernel's fixed costs)
+    return std::max((double)d.C / Cp, s2d_efficiency(d)) >= 0.2 ||
+           (d.R * d.S >= 2 && ((d.Kred + 31) / 32) * 32 <= gconv::kMaxKred && (long long)d.M * d.K >= 128 * 256);
 }
 
 int igemm_num_tiles() { return kNumIgemmTiles; }
@@ -760,6 +770,55 @@ double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
     const long long tm = (mflat + 128 * nacc - 1) / (128 * nacc), tn = (d.K + BN - 1) / BN;
     const double per_iter = std::max(2.2 * BN * nacc, 290.0 * nacc + 390.0);
     return wave_count((double)tm * tn, se) * (ips * per_iter + 5000.0 + nacc * epilogue_cost(BN, se, false));
+}
+
+// Gather kernel: persistent over ceil(M/128) * ceil(K/BN) tiles.  Measured: a 32-index reduction step costs about
+// 1250 clocks of gather work (1500 with padding, whose bounds tests ride along): neighbouring output points read
+// addresses `stride` floats apart, so every load instruction of a producer warp costs L1 four wavefronts.  That is
+// six to eight times the MMAs' 2*BN clocks - and still the fastest path for small-C layers with up to 7x7 windows,
+// because nothing is staged (the other tensor-core paths pay about 6000 clocks for their staging kernel).
+bool gather_legal(const ConvDims& d, int variant, bool x3)
+{
+    if (variant != BODA_VARIANT_TCONV || x3) return false;
+    const int Kp = ((d.Kred + 31) / 32) * 32;
+    return Kp <= gconv::kMaxKred && d.K >= 8 && (long long)d.N * d.C * d.H * d.W < (1LL << 31);
+}
+
+double model_cost_gather(const ConvDims& d, int BN, int sm_count)
+{
+    const long long tiles = (long long)((d.M + BM - 1) / BM) * ((d.K + BN - 1) / BN);
+    const double per_cta = (double)((tiles + sm_count - 1) / sm_count);
+    const int chunks = (d.Kred + 31) / 32;
+    return per_cta * chunks * std::max(2.0 * BN, d.pad ? 1500.0 : 1250.0) + 4500.0 + 32.0 * BN;
+}
+
+// filters [K][C*R*S] -> [K][Kp] rounded to TF32, zeros past C*R*S: the K-major B operand of the gather kernel
+__global__ void __launch_bounds__(256)
+pack_filters_flat_kernel(const float* __restrict__ filt, float* __restrict__ wp, int K, int Kred, int Kp)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const int total = K * Kp;
+    for (int idx = blockIdx.x * blockDim.x + threadIdx.x; idx < total; idx += gridDim.x * blockDim.x) {
+        const int k = idx / Kp, j = idx - k * Kp;
+        wp[idx] = j < Kred ? round_tf32(__ldg(filt + (size_t)k * Kred + j)) : 0.f;
+    }
+}
+
+template <int BN>
+int launch_gather(IgemmPlan* p, const gconv::GconvParams& prm, cudaStream_t stream)
+{
+    using C = gconv::Cfg<BN>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        BODA_CUDA_TRY(cudaFuncSetAttribute(gconv::gconv_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        attr_set = true;
+    }
+    const int grid = std::min(prm.tiles_total, p->sm_count);
+    BODA_CUDA_TRY(launch_kernel(gconv::gconv_tf32_kernel<BN>, dim3(grid), dim3(gconv::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
+                                p->map_b, prm));
+    count_launch();
+    return BODA_OK;
 }
 
 template <int BN, int NACC>
@@ -842,6 +901,22 @@ int encode_map_a(IgemmPlan* p, const void* xp)
 int encode_map_b(IgemmPlan* p)
 {
     const ConvDims& d = p->d;
+    if (p->nacc < 0) {
+        const cuuint64_t Kp = (cuuint64_t)p->gather_chunks * 32;
+        const cuuint64_t gdims[2] = {Kp, (cuuint64_t)d.K};
+        const cuuint64_t gstrides[1] = {Kp * 4};
+        const cuuint32_t gbox[2] = {BKC, (cuuint32_t)p->BN};
+        const cuuint32_t gestr[2] = {1, 1};
+        CUresult gr = g_encode_tiled(&p->map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, p->d_wp, gdims, gstrides, gbox, gestr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (gr != CUDA_SUCCESS) {
+            char msg[96];
+            std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (gather B) failed with CUresult %d", (int)gr);
+            return record_cuda_error(cudaErrorInvalidValue, msg);
+        }
+        return BODA_OK;
+    }
     const cuuint64_t Cs = (cuuint64_t)p->Cs();
     const cuuint64_t dims[3] = {Cs, (cuuint64_t)d.K, (cuuint64_t)(d.R * d.S)};
     const cuuint64_t strides[2] = {Cs * 4, (cuuint64_t)d.K * Cs * 4};
@@ -867,7 +942,9 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     ConvDims d = d_in;
     bool use_s2d = false;
     if (x3 && s2d > 0) return BODA_ERR_UNSUPPORTED;      // the error-compensated mode runs on the im2col kernel only
-    if (variant == BODA_VARIANT_TCONV && s2d != 0 && !x3) {
+    const bool force_gather = tile_id >= kFirstGatherTile;
+    if (force_gather && (s2d > 0 || !gather_legal(d_in, variant, x3))) return BODA_ERR_UNSUPPORTED;
+    if (variant == BODA_VARIANT_TCONV && s2d != 0 && !x3 && !force_gather) {
         ConvDims e;
         const bool can = s2d_view(d_in, &e);
         if (s2d > 0 && !can) return BODA_ERR_UNSUPPORTED;
@@ -904,14 +981,28 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     // tile and split: forced, or the minimum of the cost model
     double best = 1e300;
     int best_t = 2, best_s = 1;
+    (void)cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, 0);
+    {
+        int dev = 0;
+        if (cudaGetDevice(&dev) == cudaSuccess) (void)cudaDeviceGetAttribute(&p->sm_count, cudaDevAttrMultiProcessorCount, dev);
+        if (p->sm_count <= 0) p->sm_count = 148;
+    }
     for (int t = 0; t < kNumIgemmTiles; ++t) {
         if (tile_id >= 0 && t != tile_id) continue;
         const int nacc = kTileNacc[t];
+        if (nacc < 0) {
+            // the gather kernel works on the layer as given (never on a space-to-depth view) and has no split
+            if (!gather_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) continue;
+            const double c = model_cost_gather(d_in, kTileBN[t], p->sm_count);
+            if (c < best) { best = c; best_t = t; best_s = 1; }
+            continue;
+        }
         if (nacc > 0 && (x3 || variant != BODA_VARIANT_TCONV || !halo_geometry(d, kTileBN[t], nacc, nullptr))) continue;
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
             if (s > p->iters_total) continue;
-            const double c = nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms, kTileBN[t], s);
+            const double staging = 6000.0;         // the input staging kernel these tiles need and the gather tiles do not
+            const double c = staging + (nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms, kTileBN[t], s));
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
     }
@@ -920,6 +1011,39 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->tile_id = best_t;
     p->BN = kTileBN[best_t];
     p->nacc = kTileNacc[best_t];
+    if (p->nacc < 0) {
+        // ---- gather kernel: no staged input, filters flat [K][Kp], offset table on the device
+        if (!gather_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) { delete p; return BODA_ERR_UNSUPPORTED; }
+        p->d = d_in;
+        p->s2d = false;
+        const ConvDims& g = p->d;
+        p->gather_chunks = (g.Kred + 31) / 32;
+        const int Kp = p->gather_chunks * 32;
+        p->Cp = ((g.C + BKC - 1) / BKC) * BKC;
+        p->splits = 1;
+        p->iters_total = p->iters_per_split = p->gather_chunks;
+        p->tiles_m = (g.M + BM - 1) / BM;
+        p->tiles_n = (g.K + p->BN - 1) / p->BN;
+        p->xp_bytes = 0;
+        p->partial_bytes = 0;
+        std::vector<int2> tab((size_t)Kp);
+        for (int k = 0; k < Kp; ++k) {
+            if (k < g.Kred) {
+                const int c = k / (g.R * g.S), rs = k - c * g.R * g.S, r = rs / g.S, sx = rs - r * g.S;
+                tab[k] = make_int2(c * g.H * g.W + r * g.W + sx, (r << 16) | sx);
+            } else {
+                tab[k] = make_int2(0, 0x4000 << 16);
+            }
+        }
+        cudaError_t ge = cudaMalloc(&p->d_tab, (size_t)Kp * sizeof(int2));
+        if (ge == cudaSuccess) ge = cudaMemcpy(p->d_tab, tab.data(), (size_t)Kp * sizeof(int2), cudaMemcpyHostToDevice);
+        if (ge == cudaSuccess) ge = cudaMalloc(&p->d_wp, (size_t)g.K * Kp * 4);
+        if (ge != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(ge, "gather plan allocation"); }
+        rc = encode_map_b(p);
+        if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
+        *out = p;
+        return BODA_OK;
+    }
     if (p->nacc > 0 && (x3 || variant != BODA_VARIANT_TCONV || !halo_geometry(d, p->BN, p->nacc, p))) { delete p; return BODA_ERR_UNSUPPORTED; }
     p->iters_per_split = (p->iters_total + best_s - 1) / best_s;
     p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;   // no empty split
@@ -947,6 +1071,7 @@ void igemm_plan_destroy(IgemmPlan* p)
 {
     if (!p) return;
     if (p->d_wp) cudaFree(p->d_wp);
+    if (p->d_tab) cudaFree(p->d_tab);
     delete p;
 }
 
@@ -957,6 +1082,12 @@ size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
     const char* view = p->s2d ? "s2d " : "";
+    if (p->nacc < 0) {
+        const int tiles = p->tiles_m * p->tiles_n;
+        std::snprintf(buf, n, "tile=gconv_128x%d(id %d) stages=%d split_k=1 grid=%dx1x1 tiles=%d", p->BN, p->tile_id,
+                      p->BN <= 96 ? 5 : 4, std::min(tiles, p->sm_count), tiles);
+        return;
+    }
     if (p->nacc > 0) {
         std::snprintf(buf, n, "%stile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d", view, 128 * p->nacc, p->BN,
                       p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits);
@@ -993,7 +1124,11 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const ConvDims& d = p->d;
     const long long total = (long long)d.R * d.S * d.K * p->Cp;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
-    if (p->s2d) {
+    if (p->nacc < 0) {
+        const int Kp = p->gather_chunks * 32;
+        const int gblocks = (int)std::min<long long>(((long long)d.K * Kp + 255) / 256, 148 * 8);
+        BODA_CUDA_TRY(launch_kernel(pack_filters_flat_kernel, dim3(gblocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.Kred, Kp));
+    } else if (p->s2d) {
         const ConvDims& o = p->orig;
         BODA_CUDA_TRY(launch_kernel(pack_filters_s2d_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, p->d_wp, o.K, o.C, o.R,
                                     o.S, o.stride, d.R, d.S, p->Cp));
@@ -1032,7 +1167,7 @@ static OutSpec make_out_spec(const IgemmPlan* p, float* out)
 
 bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 {
-    if (p->s2d || p->terms == 3) return false;      // space-to-depth staging and the hi/lo operand split read NCHW only
+    if (p->s2d || p->terms == 3 || p->nacc < 0) return false;   // space-to-depth staging, the hi/lo operand split and the gather kernel read NCHW only
     if (p->nacc > 0) { *Hp = p->Hp; *Wp = p->Wp; } else { *Hp = p->d.H; *Wp = p->d.W; }
     *Cp = p->Cp;
     return true;
@@ -1040,7 +1175,7 @@ bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 
 int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
-    if (in_packed && p->s2d) return BODA_ERR_UNSUPPORTED;
+    if (in_packed && (p->s2d || p->nacc < 0)) return BODA_ERR_UNSUPPORTED;
     if ((in_packed || out_packed) && p->terms == 3) return BODA_ERR_UNSUPPORTED;
     if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < p->d.P || oWp < p->d.Q)) return BODA_ERR_INVALID_ARG;
     p->in_packed = in_packed != 0;
@@ -1053,13 +1188,31 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
                  cudaStream_t stream, cudaEvent_t after_staging)
 {
     const ConvDims& d = p->d;
-    if (!p->in_packed && !workspace) return BODA_ERR_NOMEM;
-    if (!p->in_packed && ((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
+    const bool needs_staging = !p->in_packed && p->nacc >= 0;
+    if (needs_staging && !workspace) return BODA_ERR_NOMEM;
+    if (needs_staging && ((uintptr_t)workspace & 255) != 0) return BODA_ERR_INVALID_ARG;
     float* xp = p->in_packed ? const_cast<float*>(in) : (float*)workspace;
     if (filt != p->bound_filt || !filt) {
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
+    }
+    if (p->nacc < 0) {
+        if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
+        gconv::GconvParams gp;
+        gp.in = in; gp.tab = p->d_tab; gp.bias = bias;
+        gp.CHW = d.C * d.H * d.W; gp.H = d.H; gp.W = d.W; gp.stride = d.stride; gp.pad = d.pad;
+        gp.M = d.M; gp.Kred = d.Kred; gp.nchunks = p->gather_chunks;
+        gp.tiles_n = p->tiles_n; gp.tiles_total = p->tiles_m * p->tiles_n;
+        gp.o = make_out_spec(p, out);
+        gp.status = p->d_status;
+        gp.tx_extra = p->tx_extra;
+        switch (p->BN) {
+            case 64: return launch_gather<64>(p, gp, stream);
+            case 96: return launch_gather<96>(p, gp, stream);
+            case 128: return launch_gather<128>(p, gp, stream);
+            default: return BODA_ERR_UNSUPPORTED;
+        }
     }
     if (p->s2d && !p->in_packed) {
         // both kernels read the same [N][H'][W'][Cp] layout here (the view has no padding)

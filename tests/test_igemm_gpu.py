@@ -173,7 +173,7 @@ def test_space_to_depth_off_and_auto_agree_with_oracle():
     ref = oracle_out(shape, x, w, b)
     a, da = run_planned(shape, x, w, b, variant=TC, s2d=0)
     c, dc = run_planned(shape, x, w, b)                      # automatic: tconv through the space-to-depth view
-    assert "s2d" not in da and "s2d" in dc and "tconv" in dc
+    assert "s2d" not in da and "tconv" in dc and ("s2d" in dc or "gconv" in dc)     # automatic: the view or the gather kernel
     assert_parity(a, ref, TF32_TOL, da)
     assert_parity(c, ref, TF32_TOL, dc)
 
@@ -183,3 +183,52 @@ def test_space_to_depth_refused_for_stride_one():
     with pytest.raises(B.BodaError) as e:
         B.ConvPlan((1, 32, 8, 8, 16, 3, 3, 1, 1, 0), variant=TC, s2d=1)
     assert e.value.status == B.BODA_ERR_UNSUPPORTED
+
+
+# ---- gather kernel (tiles 16..18): the input tile is built by producer warps straight from NCHW
+GATHER_CASES = [
+    (2, 3, 23, 23, 40, 11, 11, 4, 0, 1),       # conv1-like: no padding, 363 reduction indices (ragged last chunk)
+    (1, 3, 32, 32, 16, 3, 3, 1, 1, 1),         # configuration 1: one ragged chunk, padding on all sides
+    (3, 8, 15, 17, 24, 3, 5, 2, 1, 0),         # stride 2, R != S
+    (2, 16, 9, 9, 130, 5, 5, 1, 2, 1),         # several channel tiles per pixel tile, 400 indices
+    (1, 4, 6, 6, 16, 3, 3, 1, 3, 0),           # pad >= window: border outputs are pure bias
+    (7, 3, 40, 40, 96, 7, 7, 2, 3, 1),         # more tiles than one wave of CTAs would need at batch 7? (2800 points)
+    (1, 32, 8, 8, 16, 2, 2, 1, 0, 1),          # exactly four full chunks, no tail
+]
+
+
+@pytest.mark.parametrize("shape", GATHER_CASES)
+@pytest.mark.parametrize("tile", [16, 17, 18])
+def test_gather_tiles_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 2100)
+    got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile)
+    assert "gconv" in desc and f"id {tile}" in desc
+    ref = oracle_out(shape, x, w, b)
+    assert np.abs(ref).max() < 2 ** 24
+    np.testing.assert_array_equal(got.astype(np.float64), ref, err_msg=desc)
+
+
+def test_gather_conv1_shape_real_values_and_persistence():
+    # 60 500 output points at batch 20 = 473 tiles on 148 persistent CTAs: several tiles per CTA, ragged last tile
+    shape = (20, 3, 227, 227, 96, 11, 11, 4, 0, 1)
+    x = wl.uniform(2200, (20, 3, 227, 227), 0.0, 1.0)
+    w = wl.normal(2201, (96, 3, 11, 11), 0, (2.0 / 363) ** 0.5)
+    b = wl.normal(2202, (96,), 0, 0.01)
+    ref = oracle_out(shape, x, w, b)
+    for tile, bind in ((17, False), (17, True), (16, True), (18, True)):
+        got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile, bind=bind)
+        assert "gconv" in desc
+        assert_parity(got, ref, TF32_TOL, desc)
+    a, _ = run_planned(shape, x, w, b, variant=TC, tile_id=17, bind=True)
+    a2, _ = run_planned(shape, x, w, b, variant=TC, tile_id=17, bind=True)
+    assert np.array_equal(a, a2)                # the same plan twice: bit for bit
+
+
+def test_gather_refused_where_it_does_not_apply():
+    from paper_1606_00094_b200 import binding as B
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((1, 256, 13, 13, 64, 3, 3, 1, 1, 1), variant=TC, tile_id=17)        # 2304 reduction indices: table too small
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((1, 3, 32, 32, 16, 3, 3, 1, 1, 1), variant=TC, tile_id=17, split_k=2)
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((1, 3, 33, 33, 16, 3, 3, 2, 1, 1), variant=TC, tile_id=17, s2d=1)
