@@ -16,7 +16,7 @@ from helpers import TF32_TOL, assert_parity, oracle_out
 pytestmark = pytest.mark.gpu
 
 
-@pytest.mark.parametrize("tile,split", [(2, 1), (6, 1), (3, 2), (10, 2)])   # im2col and halo kernels, with and without a cluster
+@pytest.mark.parametrize("tile,split", [(2, 1), (6, 1), (3, 2), (10, 2), (17, 1)])   # im2col and halo kernels, with and without a cluster; gather kernel
 def test_expired_wait_sets_status_and_context_survives(tile, split):
     import torch
     from paper_1606_00094_b200 import binding as B
