@@ -37,7 +37,7 @@ struct GconvParams {
     const int2* tab;             // per reduction index k (padded to nchunks*32): {element offset c*H*W + r*W + s, (r << 16) | s};
                                  // indices past C*R*S carry r = 0x4000 so that the bounds test fails
     const float* bias;
-    int CHW, H, W, stride, pad;
+    int CHW, H, W, R, S, stride, pad;
     int M;                       // N * P * Q output points
     int Kred, nchunks;           // C*R*S and ceil(C*R*S / 32)
     int tiles_n, tiles_total;    // tiles are numbered m_tile * tiles_n + n_tile
@@ -218,11 +218,10 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
         const int group = pw >> 2, row = (pw & 3) * 32 + lane;
         const uint32_t sw = (uint32_t)(row & 7);
         const int total_chunks = my_tiles * nchunks;
-        const bool check_all = p.pad != 0;
         int cur_t = -1;
         long long base = 0;
         int y0 = 0, x0 = 0;
-        bool valid = false;
+        bool valid = false, check_all = false;
         for (int gc = group; gc < total_chunks; gc += kGroups) {
             const int t = gc / nchunks, j = gc - t * nchunks;
             const uint32_t stage = (uint32_t)gc % (uint32_t)kStages, par = (((uint32_t)gc / (uint32_t)kStages) & 1u) ^ 1u;
@@ -239,8 +238,10 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
                     x0 = qq * p.stride - p.pad;
                     base = (long long)n * p.CHW + (long long)y0 * p.W + x0;
                 }
+                // bounds tests are needed only where a window of this warp's 32 output points leaves the image
+                const bool inside = !valid || (y0 >= 0 && y0 + p.R <= p.H && x0 >= 0 && x0 + p.S <= p.W);
+                check_all = !__all_sync(0xffffffffu, inside);
             }
-            if (!mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 25)) break;
             const float* src = p.in + base;
             const int kk0 = 32 * j;
             float v[32];
@@ -265,6 +266,8 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
                     v[i] = (valid && (unsigned)y < (unsigned)p.H && (unsigned)x < (unsigned)p.W) ? __ldg(src + s_off[kk0 + i]) : 0.f;
                 }
             }
+            // the loads above are in flight while this waits for the stage to be free
+            if (!mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 25)) break;
             // 128-byte swizzle: 16-byte piece c of row `row` lives at piece c ^ (row & 7)
             const uint32_t a_row = smem_a + stage * A_STAGE_BYTES + (uint32_t)row * 128u;
 #pragma unroll

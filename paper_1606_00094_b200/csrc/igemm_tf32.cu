@@ -1201,7 +1201,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
         gconv::GconvParams gp;
         gp.in = in; gp.tab = p->d_tab; gp.bias = bias;
-        gp.CHW = d.C * d.H * d.W; gp.H = d.H; gp.W = d.W; gp.stride = d.stride; gp.pad = d.pad;
+        gp.CHW = d.C * d.H * d.W; gp.H = d.H; gp.W = d.W; gp.R = d.R; gp.S = d.S; gp.stride = d.stride; gp.pad = d.pad;
         gp.M = d.M; gp.Kred = d.Kred; gp.nchunks = p->gather_chunks;
         gp.tiles_n = p->tiles_n; gp.tiles_total = p->tiles_m * p->tiles_n;
         gp.o = make_out_spec(p, out);
