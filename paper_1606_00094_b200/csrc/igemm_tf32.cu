@@ -510,30 +510,46 @@ pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int 
     for (int row = warp; row < C * t; row += nwarps) {
         const int c = row / t, dy = row - c * t;
         const int y = yb * t + dy - pad;
-        const bool inside = y >= 0 && y < H;
-        const float* src = in + (((size_t)n * C + c) * H + (inside ? y : 0)) * W;
-        for (int x0 = lane; x0 < W; x0 += 256) {                 // eight loads in flight per lane
-            float v[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j) v[j] = (inside && x0 + 32 * j < W) ? __ldg(src + x0 + 32 * j) : 0.f;
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                if (x0 + 32 * j < W) sm_rows[row * W + x0 + 32 * j] = v[j];
+        float* dstrow = sm_rows + row * W;
+        if (y >= 0 && y < H) {
+            const float* src = in + (((size_t)n * C + c) * H + y) * W;
+#pragma unroll 4
+            for (int x = lane; x < W; x += 32) dstrow[x] = __ldg(src + x);
+        } else {
+            for (int x = lane; x < W; x += 32) dstrow[x] = 0.f;
         }
     }
     __syncthreads();
-    // write the row of blocks: one warp per block xb, lanes along the packed channels (contiguous 128-byte stores)
+    // write the row of blocks: a thread takes four consecutive packed channels of a block (one 16-byte store; the
+    // sixteen-byte stores of a warp cover whole 128-byte lines) and keeps them for every block it writes, so the
+    // table look-ups leave the loop.  The kernel is bound by instruction issue, not by memory: the loop body is four
+    // bounds tests, four shared-memory loads, four roundings and one store.
     float* dst = xs + ((size_t)n * Hb + yb) * Wb * Cp;
-    for (int xb = warp; xb < Wb; xb += nwarps) {
-        const int xoff = xb * t;
-        for (int cp = lane; cp < Cp; cp += 32) {
-            const int rowbase = sm_src[cp];
-            float v = 0.f;
-            if (rowbase >= 0) {
-                const int x = xoff + sm_dx[cp];                  // column in the input image
-                if (x >= 0 && x < W) v = sm_rows[rowbase + x];
-            }
-            dst[(size_t)xb * Cp + cp] = round_tf32(v);
+    const int quads = Cp >> 2;                                       // Cp is a multiple of 32
+    auto emit = [&](int cq, int xb, const int (&rb)[4], const int (&dxp)[4]) {
+        const int xo = xb * t;
+        float v[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int x = xo + dxp[i];
+            v[i] = (rb[i] >= 0 && x >= 0 && x < W) ? round_tf32(sm_rows[rb[i] + x]) : 0.f;
+        }
+        *reinterpret_cast<float4*>(dst + (size_t)xb * Cp + 4 * cq) = make_float4(v[0], v[1], v[2], v[3]);
+    };
+    if ((int)blockDim.x % quads == 0) {
+        // the usual case: a thread's channel quad is the same for all its blocks
+        const int cq = threadIdx.x % quads, xstep = blockDim.x / quads;
+        int rb[4], dxp[4];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) { rb[i] = sm_src[4 * cq + i]; dxp[i] = sm_dx[4 * cq + i]; }
+        for (int xb = threadIdx.x / quads; xb < Wb; xb += xstep) emit(cq, xb, rb, dxp);
+    } else {
+        for (int item = threadIdx.x; item < quads * Wb; item += blockDim.x) {
+            const int cq = item % quads, xb = item / quads;
+            int rb[4], dxp[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { rb[i] = sm_src[4 * cq + i]; dxp[i] = sm_dx[4 * cq + i]; }
+            emit(cq, xb, rb, dxp);
         }
     }
 }
