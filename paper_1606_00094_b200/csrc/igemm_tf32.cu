@@ -109,7 +109,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const uint32_t full_bar = bars;                    // STAGES x 2 x 8 bytes: [stage][issuer]
     const uint32_t empty_bar = bars + 16 * STAGES;
     const uint32_t accum_bar = bars + 24 * STAGES;
-    const uint32_t recv_bar = accum_bar + 8;           // split reduction: bytes pushed by the cluster peers
+    const uint32_t recv_bar = accum_bar + 8;           // split reduction: bytes pushed by the cluster peers, [chunk] (4)
     __shared__ uint32_t s_tmem_base;
     __shared__ volatile int s_abort;
     __shared__ __align__(16) float s_bias[BN];
@@ -128,7 +128,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 16 * s, 1); mbar_init(full_bar + 16 * s + 8, 1); mbar_init(empty_bar + 8 * s, 1); }
         mbar_init(accum_bar, Cfg::ISSUERS);           // one arrival per MMA issuer
-        mbar_init(recv_bar, 1);
+        for (int c = 0; c < 4; ++c) mbar_init(recv_bar + 8 * c, 1);      // one per 32-channel chunk of this CTA's share
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
@@ -278,8 +278,12 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         __syncwarp();
         // All epilogue threads meet here whatever their wait returned, then take one common decision:
         // a failed wait has raised the abort flag before returning.
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        const bool ok = (s_abort == 0);
+        // (a barrier with an OR reduction: the decision is the same in all 256 threads even if the flag is raised
+        // while they read it, so that the group barriers below are reached by everyone or by no one)
+        uint32_t stop;
+        asm volatile("{\n\t.reg .pred q, r;\n\tsetp.ne.u32 q, %1, 0;\n\tbar.red.or.pred r, 1, 256, q;\n\tselp.u32 %0, 1, 0, r;\n\t}"
+                     : "=r"(stop) : "r"((uint32_t)s_abort) : "memory");
+        const bool ok = stop == 0;
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         const bool two_acc = Cfg::ISSUERS == 2 && my_iters >= 2;   // a single reduction step never reaches the second issuer
@@ -322,57 +326,64 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
         } else if (exchange) {
             // split reduction by exchange, see split_share(): partial sums of the channels other CTAs own go into
-            // send blocks while the cluster barrier (every CTA's main loop has ended, its stage buffers are free)
-            // completes; then one bulk copy per peer, and the owner adds what it received to its own accumulator.
+            // send blocks, 32 channels (16 KB) at a time; as soon as a chunk is complete one thread pushes it to its
+            // owner with a bulk copy, counted on the owner's barrier for that chunk, and the owner adds each chunk
+            // to its own accumulator as it arrives - so writing, transfer (about 16 bytes per clock) and finishing
+            // overlap.  The first push waits for the cluster barrier: every CTA's main loop has ended and its stage
+            // buffers, which the blocks reuse, are free.
             cluster_arrive();
             const int rank = (int)cluster_cta_rank();
             const int per = split_share(BN, p.splits);
             const int my_w = split_width(BN, per, rank);
             const uint32_t recv_base = smem_base + 512u * (uint32_t)(per * (p.splits - 1));
+            // warp 2 / warp 7 push for their group.  The whole warp takes the cluster barrier's second half together:
+            // lanes of one warp waiting at different places would wait for different phases of the barrier.
+            const bool push_warp = quarter == (group ? 3 : 2);
+            bool waited = false;
             if (ok) {
-                if (threadIdx.x == 64 && my_w > 0) mbar_expect_tx(recv_bar, 512u * (uint32_t)(my_w * (p.splits - 1)));
+                if (threadIdx.x == 64)
+                    for (int c = 0; 32 * c < my_w; ++c) mbar_expect_tx(recv_bar + 8 * c, 16384u * (uint32_t)(p.splits - 1));
                 int turn = 0;
 #pragma unroll 1
                 for (int dst = 0; dst < p.splits; ++dst) {
                     const int wd = split_width(BN, per, dst);
                     if (dst == rank || wd == 0) continue;
                     const uint32_t block = smem_base + 512u * (uint32_t)(per * (dst < rank ? dst : dst - 1));
+                    const uint32_t slot = recv_base + 512u * (uint32_t)(wd * (rank < dst ? rank : rank - 1));
 #pragma unroll 1
-                    for (int c0 = 0; c0 < wd; c0 += 32, ++turn) {
+                    for (int c = 0; 32 * c < wd; ++c, ++turn) {
                         if ((turn & 1) != group) continue;
                         uint32_t v[32];
-                        load32(dst * per + c0, v);
-                        xchg_put32(block, wd, row, c0, v);
+                        load32(dst * per + 32 * c, v);
+                        xchg_put32(block + 16384u * (uint32_t)c, 32, row, 0, v);
+                        fence_proxy_async_smem();
+                        if (group) asm volatile("bar.sync 3, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
+                        if (push_warp) {
+                            if (!waited) { cluster_wait(); waited = true; }
+                            if (lane == 0)
+                                bulk_push_cluster(map_to_cta(slot + 16384u * (uint32_t)c, (uint32_t)dst), block + 16384u * (uint32_t)c, 16384u,
+                                              map_to_cta(recv_bar + 8 * c, (uint32_t)dst));
+                        }
                     }
                 }
-                fence_proxy_async_smem();
             }
-            asm volatile("bar.sync 1, 256;" ::: "memory");
-            cluster_wait();
-            if (threadIdx.x == 64 && s_abort == 0) {
-                for (int dst = 0; dst < p.splits; ++dst) {
-                    const int wd = split_width(BN, per, dst);
-                    if (dst == rank || wd == 0) continue;
-                    const uint32_t block = smem_base + 512u * (uint32_t)(per * (dst < rank ? dst : dst - 1));
-                    const uint32_t slot = smem_base + 512u * (uint32_t)(per * (p.splits - 1))
-                                        + 512u * (uint32_t)(wd * (rank < dst ? rank : rank - 1));
-                    bulk_push_cluster(map_to_cta(slot, (uint32_t)dst), block, 512u * (uint32_t)wd, map_to_cta(recv_bar, (uint32_t)dst));
-                }
-            }
-            if (s_abort == 0 && my_w > 0 && mbar_wait(recv_bar, 0, &s_abort, p.status, 5)) {
+            if (!waited) cluster_wait();           // every thread takes the second half of the barrier exactly once
+            if (ok && my_w > 0) {
                 const RowDst d = igemm_row_dst(p, m);
 #pragma unroll 1
-                for (int c0 = 32 * group; c0 < my_w; c0 += 64) {
+                for (int c = group; 32 * c < my_w; c += 2) {
+                    if (!mbar_wait(recv_bar + 8 * c, 0, &s_abort, p.status, 5)) break;
                     uint32_t v[32];
-                    load32(rank * per + c0, v);
+                    load32(rank * per + 32 * c, v);
                     float y[32];
 #pragma unroll
                     for (int j = 0; j < 32; ++j) y[j] = __uint_as_float(v[j]);
-                    for (int sl = 0; sl < p.splits - 1; ++sl) xchg_add32(recv_base + 512u * (uint32_t)(my_w * sl), my_w, row, c0, y);
+                    for (int sl = 0; sl < p.splits - 1; ++sl)
+                        xchg_add32(recv_base + 512u * (uint32_t)(my_w * sl) + 16384u * (uint32_t)c, 32, row, 0, y);
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
-                    bias_relu32(v, s_bias + rank * per + c0, p.o.relu != 0, y);
-                    store_row32(p.o, d, k0 + rank * per + c0, y);
+                    bias_relu32(v, s_bias + rank * per + 32 * c, p.o.relu != 0, y);
+                    store_row32(p.o, d, k0 + rank * per + 32 * c, y);
                 }
             }
         } else if (ok) {
