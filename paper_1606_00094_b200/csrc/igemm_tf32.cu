@@ -491,76 +491,55 @@ pack_filters_kernel(const float* __restrict__ filt, float* __restrict__ wp, int 
 // is pixel (yb*t + dy, xb*t + dx) of the zero-padded input and the filter taps past R or S are zeros.  It turns
 // a first layer such as 11x11 stride 4 on 3 channels into a 3x3 stride-1 layer on 48 channels, which the
 // tensor-core kernels can run; the paper's tconv likewise needs "an input transformation" (Section 5).
+// Packed channel order: cp = (dy*C + c)*t + dx, so that the t values dx = 0..t-1 of a (dy, c) pair - which are t
+// consecutive floats of one input row - stay together: for t = 4 the transform is a copy of 16-byte pieces.
 // One CTA builds one block-row: it stages the t input rows of all channels in shared memory with coalesced
-// reads, then writes the [W'][Cp] row of blocks contiguously.
+// reads (row pitch rounded up to 4 floats and shifted so that block 0 starts 16-byte aligned), then writes the
+// [W'][Cp] row of blocks.
 __global__ void __launch_bounds__(256)
 pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int C, int H, int W, int t, int pad,
                       int Hb, int Wb, int Cp)
 {
-    extern __shared__ float sm_rows[];            // [C*t rows][W], then two int tables [Cp]
-    int* sm_src = reinterpret_cast<int*>(sm_rows + C * t * W);
-    int* sm_dx = sm_src + Cp;
+    extern __shared__ __align__(16) float sm_rows[];     // [C*t rows][pitch]: element x of a row at [row*pitch + pad + x]
     pdl_launch_dependents();
     const int yb = blockIdx.x, n = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
-    // tables: packed channel cp = (dy*t + dx)*C + c  ->  start of staged row (c, dy) in sm_rows, and dx - pad
-    const int Cs = C * t * t;
-    for (int cp = threadIdx.x; cp < Cp; cp += blockDim.x) {
-        int v = -1, dxp = 0;
-        if (cp < Cs) {
-            const int g = cp / C, c = cp - g * C;
-            const int dy = g / t, dx = g - dy * t;
-            v = (c * t + dy) * W;
-            dxp = dx - pad;
-        }
-        sm_src[cp] = v;
-        sm_dx[cp] = dxp;
-    }
+    const int span = Wb * t;                               // columns -pad .. span-pad-1 of the image feed this block-row
+    const int pitch = (span + 3) & ~3;
+    const int rows = C * t;                                // row index = dy*C + c
     pdl_wait();
-    // stage the t input rows of every channel: one warp per (c, dy) row, lanes along x (coalesced)
-    for (int row = warp; row < C * t; row += nwarps) {
-        const int c = row / t, dy = row - c * t;
+    // stage: one warp per (dy, c) row, lanes along x (coalesced); zeros outside the image
+    for (int row = warp; row < rows; row += nwarps) {
+        const int dy = row / C, c = row - dy * C;
         const int y = yb * t + dy - pad;
-        float* dstrow = sm_rows + row * W;
-        if (y >= 0 && y < H) {
-            const float* src = in + (((size_t)n * C + c) * H + y) * W;
+        float* dstrow = sm_rows + row * pitch;
+        const bool inside = y >= 0 && y < H;
+        const float* src = in + (((size_t)n * C + c) * H + (inside ? y : 0)) * W - pad;
 #pragma unroll 4
-            for (int x = lane; x < W; x += 32) dstrow[x] = __ldg(src + x);
-        } else {
-            for (int x = lane; x < W; x += 32) dstrow[x] = 0.f;
+        for (int i = lane; i < pitch; i += 32) {
+            const int x = i - pad;
+            dstrow[i] = (inside && x >= 0 && x < W) ? __ldg(src + i) : 0.f;
         }
     }
     __syncthreads();
-    // write the row of blocks: a thread takes four consecutive packed channels of a block (one 16-byte store; the
-    // sixteen-byte stores of a warp cover whole 128-byte lines) and keeps them for every block it writes, so the
-    // table look-ups leave the loop.  The kernel is bound by instruction issue, not by memory: the loop body is four
-    // bounds tests, four shared-memory loads, four roundings and one store.
     float* dst = xs + ((size_t)n * Hb + yb) * Wb * Cp;
-    const int quads = Cp >> 2;                                       // Cp is a multiple of 32
-    auto emit = [&](int cq, int xb, const int (&rb)[4], const int (&dxp)[4]) {
-        const int xo = xb * t;
-        float v[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int x = xo + dxp[i];
-            v[i] = (rb[i] >= 0 && x >= 0 && x < W) ? round_tf32(sm_rows[rb[i] + x]) : 0.f;
-        }
-        *reinterpret_cast<float4*>(dst + (size_t)xb * Cp + 4 * cq) = make_float4(v[0], v[1], v[2], v[3]);
-    };
-    if ((int)blockDim.x % quads == 0) {
-        // the usual case: a thread's channel quad is the same for all its blocks
-        const int cq = threadIdx.x % quads, xstep = blockDim.x / quads;
-        int rb[4], dxp[4];
-#pragma unroll
-        for (int i = 0; i < 4; ++i) { rb[i] = sm_src[4 * cq + i]; dxp[i] = sm_dx[4 * cq + i]; }
-        for (int xb = threadIdx.x / quads; xb < Wb; xb += xstep) emit(cq, xb, rb, dxp);
-    } else {
+    if (t == 4) {
+        // 16 lanes cover the 64-byte-aligned channel quads of one block: quad j < rows is (dy, c) = row j, the rest padding
+        const int quads = Cp >> 2;
         for (int item = threadIdx.x; item < quads * Wb; item += blockDim.x) {
-            const int cq = item % quads, xb = item / quads;
-            int rb[4], dxp[4];
-#pragma unroll
-            for (int i = 0; i < 4; ++i) { rb[i] = sm_src[4 * cq + i]; dxp[i] = sm_dx[4 * cq + i]; }
-            emit(cq, xb, rb, dxp);
+            const int j = item % quads, xb = item / quads;
+            float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
+            if (j < rows) {
+                const float4 r = *reinterpret_cast<const float4*>(sm_rows + j * pitch + 4 * xb);
+                v = make_float4(round_tf32(r.x), round_tf32(r.y), round_tf32(r.z), round_tf32(r.w));
+            }
+            *reinterpret_cast<float4*>(dst + (size_t)xb * Cp + 4 * j) = v;
+        }
+    } else {
+        for (int item = threadIdx.x; item < Cp * Wb; item += blockDim.x) {
+            const int cp = item % Cp, xb = item / Cp;
+            const int row = cp / t, dx = cp - row * t;
+            dst[(size_t)xb * Cp + cp] = row < rows ? round_tf32(sm_rows[row * pitch + xb * t + dx]) : 0.f;
         }
     }
 }
@@ -583,9 +562,8 @@ pack_filters_s2d_kernel(const float* __restrict__ filt, float* __restrict__ wp, 
         const int rb = tapb / Sb, sb = tapb - rb * Sb;
         float v = 0.f;
         if (cp < Cs) {
-            const int g = cp / C;
-            const int c = cp - g * C;
-            const int dy = g / t, dx = g - dy * t;
+            const int g = cp / t, dx = cp - g * t;            // packed channel order (dy, c, dx), as in pack_input_s2d_kernel
+            const int dy = g / C, c = g - dy * C;
             const int r = rb * t + dy, sx = sb * t + dx;
             if (r < R && sx < S) v = __ldg(filt + (((size_t)k * C + c) * R + r) * S + sx);
         }
@@ -692,7 +670,7 @@ static bool s2d_view(const ConvDims& d, ConvDims* e)
 {
     const int t = d.stride;
     if (t < 2 || t > 4 || d.R * d.S < 2) return false;
-    if ((size_t)d.C * t * d.W * 4 > 40 * 1024) return false;       // shared-memory staging of the pack kernel
+    if ((size_t)d.C * t * (d.W + 2 * d.pad + t + 4) * 4 > 44 * 1024) return false;   // shared-memory staging of the pack kernel
     if ((long long)d.C * t * t > 1024) return false;
     ConvDims v = d;
     v.C = d.C * t * t;
@@ -1245,7 +1223,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         // both kernels read the same [N][H'][W'][Cp] layout here (the view has no padding)
         const ConvDims& o = p->orig;
         dim3 grid(d.H, d.N);
-        const size_t smem = (size_t)o.C * o.stride * o.W * 4 + (size_t)p->Cp * 8;
+        const size_t smem = (size_t)o.C * o.stride * (((size_t)d.W * o.stride + 3) & ~(size_t)3) * 4;
         BODA_CUDA_TRY(launch_kernel(pack_input_s2d_kernel, grid, dim3(256), smem, stream, 1, in, xp, o.C, o.H, o.W, o.stride,
                                     o.pad, d.H, d.W, p->Cp));
         count_launch();
