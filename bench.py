@@ -235,6 +235,44 @@ def single_layer_configs(B, wl, torch, peaks, flush):
     return out
 
 
+def large_batch_rows(B, wl, torch, peaks, flush):
+    """EXTRA, not a BASELINE configuration: the shapes of configurations 1-3 at batch 256, where a launch moves enough
+    bytes to leave the latency regime; shows the bandwidth fraction these layers approach (L2-cold, median of 5)."""
+    out = []
+    for cid in (1, 2, 3):
+        s0 = wl.CONFIGS[cid].shape
+        shape = (256, s0.C, s0.H, s0.W, s0.K, s0.R, s0.S, s0.stride, s0.pad, 1)
+        N, C, H, W, K, R, S, st, pad, _ = shape
+        P, Q = (H + 2 * pad - R) // st + 1, (W + 2 * pad - S) // st + 1
+        x = torch.rand((N, C, H, W), dtype=torch.float32, device="cuda")
+        w = torch.randn((K, C, R, S), dtype=torch.float32, device="cuda") * 0.05
+        b = torch.zeros((K,), dtype=torch.float32, device="cuda")
+        plan = B.ConvPlan(shape, tune=1)
+        y = torch.empty(plan.out_shape, dtype=torch.float32, device="cuda")
+        plan.bind_filters(w)
+        for _ in range(3):
+            plan(x, w, b, out=y)
+        torch.cuda.synchronize()
+        cold = []
+        for _ in range(5):
+            flush.zero_()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record()
+            plan(x, w, b, out=y)
+            e1.record()
+            torch.cuda.synchronize()
+            cold.append(e0.elapsed_time(e1) * 1e3)
+        us = sorted(cold)[len(cold) // 2]
+        flops = 2.0 * N * K * P * Q * C * R * S
+        nbytes = 4.0 * (N * C * H * W + K * C * R * S + K + N * K * P * Q)
+        out.append({"shape_of_config": cid, "batch": 256, "us_l2_cold": round(us, 1), "gflops": round(flops / us / 1e3, 1),
+                    "algorithmic_gbs": round(nbytes / us / 1e3, 1),
+                    "frac_of_hbm_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4),
+                    "frac_of_tf32_peak": round(flops / us / 1e6 / (0.5 * peaks["bf16_tflops"]), 4), "plan": plan.describe()})
+        plan.close()
+    return out
+
+
 def sgemm_table1(B, torch, peaks):
     """boda_sgemm on the square sizes of the paper's Table 1 (context, not the headline): device time per call
     from a captured graph of 20 calls, operands L2-warm."""
@@ -437,6 +475,7 @@ def run_ours(args):
                     "timing": f"{dom_reps} launches of that layer in place, back to back in one captured graph, per event pair; L2-warm as inside the step"}
         per_config = [] if args.stack_only else single_layer_configs(B, wl, torch, peaks, flush)
         sgemm_rows = [] if args.stack_only else sgemm_table1(B, torch, peaks)
+        extra_rows = [] if args.stack_only else large_batch_rows(B, wl, torch, peaks, flush)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
         cpu1_v, cpu1_t, _ = time_oracle_one_thread(2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
@@ -458,6 +497,7 @@ def run_ours(args):
             "layers": layers,
             "single_layer_configs": per_config,
             "sgemm_table1": sgemm_rows,
+            "extra_not_baseline_batch256": extra_rows,
             "frac_of_tf32_peak_whole_step": round(value / 1e3 / (0.5 * peaks["bf16_tflops"]) / world, 4),
         }
         print(json.dumps(line))

@@ -232,7 +232,7 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
     int rc = BODA_OK;
     if (variant == BODA_VARIANT_DIRECT) {
         p->math = BODA_MATH_FP32;
-        if (tile_id >= direct_num_tiles()) { delete p; return BODA_ERR_UNSUPPORTED; }
+        if (tile_id >= direct_num_tiles() || (tile_id >= 0 && !direct_tile_legal(p->d, tile_id))) { delete p; return BODA_ERR_UNSUPPORTED; }
         p->tile_id = tile_id >= 0 ? tile_id : direct_pick_tile(p->d);
         const int len = direct_table_len(p->d);
         std::vector<DirectTapEntry> tab(len);

@@ -91,6 +91,8 @@ struct DirectTapEntry { int offset; int rs; };
 int direct_num_tiles();
 const char* direct_tile_name(int tile_id);
 int direct_pick_tile(const ConvDims& d);
+// false for a tile that cannot run the shape (the pixel-per-thread tiles need the input patch to fit shared memory)
+bool direct_tile_legal(const ConvDims& d, int tile_id);
 // Length (entries) of the table the tile needs; build it on the host into `host_tab`.
 int direct_table_len(const ConvDims& d);
 void direct_build_table(const ConvDims& d, DirectTapEntry* host_tab);

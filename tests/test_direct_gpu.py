@@ -36,7 +36,7 @@ def test_direct_matches_oracle(shape):
     assert_parity(got, oracle_out(shape, x, w, b), FP32_TOL, desc)
 
 
-@pytest.mark.parametrize("tile", range(9))
+@pytest.mark.parametrize("tile", range(12))        # 0..8: GEMM-blocked tiles; 9..11: pixel-per-thread tiles
 def test_every_direct_tile(tile):
     shape = (2, 5, 19, 17, 37, 3, 3, 2, 1, 1)
     x, w, b = _tensors(shape, 2000)
@@ -115,3 +115,43 @@ def _opts(B, **kw):
     for k, v in kw.items():
         setattr(o, k, v)
     return o
+
+
+# ---- pixel-per-thread tiles (small input-channel count): exact on integers, every shape quirk
+PIXEL_CASES = [
+    (1, 3, 32, 32, 16, 3, 3, 1, 1, 1),          # configuration 1
+    (3, 3, 45, 70, 20, 5, 5, 2, 2, 1),          # patch edges on both sides, stride 2, ragged channel group
+    (2, 3, 59, 59, 40, 11, 11, 4, 0, 1),        # conv1-like window and stride
+    (2, 1, 9, 40, 5, 3, 3, 1, 1, 0),            # one input channel, fewer outputs than a group
+    (1, 4, 7, 7, 70, 7, 7, 1, 3, 1),            # window as large as the image, three channel groups
+    (5, 2, 33, 65, 9, 2, 4, 3, 0, 0),           # R != S, stride 3, floor in the output extent
+]
+
+
+@pytest.mark.parametrize("shape", PIXEL_CASES)
+@pytest.mark.parametrize("tile", [9, 10, 11])
+def test_pixel_tiles_exact(shape, tile):
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x, w, b = wl.integers(4100, (N, C, H, W)), wl.integers(4101, (K, C, R, S)), wl.integers(4102, (K,))
+    got, desc = run_planned(shape, x, w, b, variant=0, math=1, tile_id=tile)
+    assert "direct_pixel" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_pixel_tile_is_the_automatic_choice_for_large_batches_of_configuration_1_and_meets_the_fp32_bar():
+    shape = (40, 3, 32, 32, 16, 3, 3, 1, 1, 1)          # configuration 1's layer at batch 40: 40 960 output pixels
+    x, w, b = _tensors(shape, 4200)
+    got, desc = run_planned(shape, x, w, b, math=1)
+    assert "direct_pixel_k16" in desc
+    assert_parity(got, oracle_out(shape, x, w, b), FP32_TOL, desc)
+    c = wl.CONFIGS[1]                                    # at batch 1 the blocked tiles stay the choice
+    x, w, b = c.tensors()
+    got, desc = run_planned(c.shape.as_tuple(), x, w, b, math=1)
+    assert "direct_pixel" not in desc
+    assert_parity(got, oracle_out(c.shape.as_tuple(), x, w, b), FP32_TOL, desc)
+
+
+def test_pixel_tile_refused_when_the_patch_does_not_fit():
+    from paper_1606_00094_b200 import binding as B
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((1, 64, 56, 56, 32, 11, 11, 4, 0, 1), variant=0, math=1, tile_id=11)
