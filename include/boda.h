@@ -176,6 +176,23 @@ int boda_conv_fwd_host(const float* in_host, const float* filt_host, const float
 int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, void* stream);
 
 /*
+ * Run-time compilation (Section 4 of the paper: kernels are generated and compiled for the exact problem once its
+ * sizes are known, so that every extent is a literal).  The DIRECT tiles named direct_rtc_k4 / k8 / k16 / k32
+ * (tile ids 12..15 of BODA_VARIANT_DIRECT; also what automatic selection uses in place of the pixel-per-thread
+ * tiles) are compiled by NVRTC when their plan is created: one thread per output pixel and `kt` output channels,
+ * all of N, C, H, W, K, R, S, stride, pad, ReLU and the blocking as compile-time constants.  They need the NVRTC
+ * shared library at run time (looked up with dlopen; without it those tiles return BODA_ERR_UNSUPPORTED and
+ * automatic selection keeps the precompiled kernels) and an input patch plus filters of at most 48 KB.
+ *
+ * boda_direct_rtc_compile compiles the kernel for `shape` without loading or running it - it needs no GPU - and
+ * reports the blocking chosen and the size of the device image.  Any of the four output pointers may be NULL.
+ * Returns BODA_OK, BODA_ERR_INVALID_ARG (bad shape, kt not 4, 8, 16 or 32), BODA_ERR_UNSUPPORTED (no NVRTC, or
+ * the shape does not fit), BODA_ERR_CUDA (the compiler refused the source; boda_last_error_string has its log).
+ */
+int boda_direct_rtc_compile(const boda_conv_shape* shape, int kt, int* block_x, int* block_y, size_t* smem_bytes,
+                            size_t* image_bytes);
+
+/*
  * The forward pass for callers that must not allocate device memory.  (The paper has no counterpart: this
  * is a property of the library, not of the method.)
  *

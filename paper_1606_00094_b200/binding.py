@@ -69,6 +69,9 @@ _lib.boda_conv_fwd.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd.restype = _i
 _lib.boda_sgemm.argtypes = [_vp] * 3 + [_i] * 3 + [_vp]
 _lib.boda_sgemm.restype = _i
+_lib.boda_direct_rtc_compile.argtypes = [ctypes.POINTER(boda_conv_shape), _i, ctypes.POINTER(_i), ctypes.POINTER(_i),
+                                         ctypes.POINTER(ctypes.c_size_t), ctypes.POINTER(ctypes.c_size_t)]
+_lib.boda_direct_rtc_compile.restype = _i
 _lib.boda_conv_fwd_host.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd_host.restype = _i
 _lib.boda_conv_fwd_noalloc.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
@@ -225,6 +228,17 @@ def boda_conv_fwd_noalloc(inp, filt, bias, out, N, C, H, W, K, R, S, stride, pad
     BODA_ERR_TOO_LARGE when the shape's scratch exceeds BODA_NOALLOC_SCRATCH_BYTES."""
     _check(_lib.boda_conv_fwd_noalloc(_addr(inp), _addr(filt), _addr(bias), _addr(out), N, C, H, W, K, R, S, stride,
                                       pad, int(bool(relu)), _stream(stream)), "boda_conv_fwd_noalloc")
+
+
+def boda_direct_rtc_compile(shape, kt):
+    """Compiles the run-time specialised DIRECT kernel for `shape` (N,C,H,W,K,R,S,stride,pad,relu) without loading it
+    (no GPU needed).  Returns (block_x, block_y, smem_bytes, image_bytes)."""
+    s = boda_conv_shape(*shape)
+    bx, by = _i(0), _i(0)
+    sm, im = ctypes.c_size_t(0), ctypes.c_size_t(0)
+    _check(_lib.boda_direct_rtc_compile(ctypes.byref(s), kt, ctypes.byref(bx), ctypes.byref(by), ctypes.byref(sm),
+                                        ctypes.byref(im)), "boda_direct_rtc_compile")
+    return bx.value, by.value, sm.value, im.value
 
 
 def boda_sgemm(A, Bm, C, M, N, K, stream=None) -> None:

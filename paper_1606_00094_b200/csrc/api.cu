@@ -140,6 +140,7 @@ struct boda_conv_plan {
     int math = BODA_MATH_FP32;
     int* d_status = nullptr;
     DirectTapEntry* d_tab = nullptr;     // DIRECT
+    DirectRtc* rtc = nullptr;            // DIRECT, tiles compiled at run time
     IgemmPlan* ig = nullptr;             // K1CONV / TCONV
     size_t ws_bytes = 0;
     bool in_packed = false;              // chained layers: the input arrives in the staged layout
@@ -154,6 +155,7 @@ int conv_fwd_planned_ex(boda_conv_plan* p, const float* in, const float* filt, c
     if (p->variant == BODA_VARIANT_DIRECT) {
         if (!filt) return BODA_ERR_INVALID_ARG;
         if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
+        if (p->rtc) return direct_rtc_launch(p->rtc, in, filt, bias, out, stream);
         return direct_launch(p->d, p->tile_id, in, filt, bias, out, p->d_tab, stream);
     }
     if (p->ws_bytes && !workspace && !p->in_packed) return BODA_ERR_NOMEM;
@@ -211,6 +213,7 @@ int boda_conv_plan_destroy(boda_conv_plan* plan)
     (void)cudaGetDevice(&prev);
     (void)cudaSetDevice(plan->device);
     if (plan->d_tab) (void)cudaFree(plan->d_tab);
+    if (plan->rtc) direct_rtc_destroy(plan->rtc);
     if (plan->ig) igemm_plan_destroy(plan->ig);
     (void)cudaSetDevice(prev);
     delete plan;
@@ -241,6 +244,13 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
         if (e == cudaSuccess)
             e = cudaMemcpy(p->d_tab, tab.data(), len * sizeof(DirectTapEntry), cudaMemcpyHostToDevice);
         if (e != cudaSuccess) rc = record_cuda_error(e, "tap table upload");
+        if (rc == BODA_OK && tile_id < 0) {
+            // short reductions with few output channels run in their run-time compiled form where NVRTC is there
+            const int rt = direct_rtc_pick(p->d);
+            if (rt >= 0 && direct_rtc_create(p->d, direct_tile_rtc_kt(rt), &p->rtc) == BODA_OK) p->tile_id = rt;
+        } else if (rc == BODA_OK && direct_tile_rtc_kt(p->tile_id) > 0) {
+            rc = direct_rtc_create(p->d, direct_tile_rtc_kt(p->tile_id), &p->rtc);
+        }
         p->ws_bytes = 0;
     } else {
         p->math = o.math == BODA_MATH_TF32X3 ? BODA_MATH_TF32X3 : BODA_MATH_TF32;
@@ -365,8 +375,10 @@ int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
     if (!p || !buf || n == 0) return BODA_ERR_INVALID_ARG;
     static const char* vn[] = {"direct", "k1conv", "tconv"};
     if (p->variant == BODA_VARIANT_DIRECT) {
-        std::snprintf(buf, n, "variant=%s tile=%s(id %d) math=fp32 split_k=1 workspace=%zu", vn[p->variant],
-                      direct_tile_name(p->tile_id), p->tile_id, p->ws_bytes);
+        char extra[96] = "";
+        if (p->rtc) { extra[0] = ' '; direct_rtc_describe(p->rtc, extra + 1, sizeof(extra) - 1); }
+        std::snprintf(buf, n, "variant=%s tile=%s(id %d)%s math=fp32 split_k=1 workspace=%zu", vn[p->variant],
+                      direct_tile_name(p->tile_id), p->tile_id, extra, p->ws_bytes);
     } else {
         char tmp[160];
         igemm_plan_describe(p->ig, tmp, sizeof(tmp));
@@ -530,6 +542,23 @@ int boda_conv_fwd(const float* in, const float* filt, const float* bias, float* 
     int rc = cache_lookup(s, false, &e);
     if (rc != BODA_OK) return rc;
     return boda_conv_fwd_planned(e->plan, in, filt, bias, out, e->workspace, stream);
+}
+
+int boda_direct_rtc_compile(const boda_conv_shape* shape, int kt, int* block_x, int* block_y, size_t* smem_bytes,
+                            size_t* image_bytes)
+{
+    if (!shape || !shape_ok(*shape) || (kt != 4 && kt != 8 && kt != 16 && kt != 32)) return BODA_ERR_INVALID_ARG;
+    const ConvDims d = make_dims(*shape);
+    int bx = 0, by = 0;
+    size_t smem = 0;
+    std::vector<char> image;
+    const int rc = direct_rtc_compile(d, kt, &bx, &by, &smem, &image);
+    if (rc != BODA_OK) return rc;
+    if (block_x) *block_x = bx;
+    if (block_y) *block_y = by;
+    if (smem_bytes) *smem_bytes = smem;
+    if (image_bytes) *image_bytes = image.size();
+    return BODA_OK;
 }
 
 int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, void* stream)

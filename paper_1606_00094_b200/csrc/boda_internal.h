@@ -1,5 +1,6 @@
 // Internal declarations shared by the translation units of the library (not part of the ABI).
 #pragma once
+#include <vector>
 
 #include <cuda_runtime.h>
 #include <stddef.h>
@@ -98,6 +99,20 @@ int direct_table_len(const ConvDims& d);
 void direct_build_table(const ConvDims& d, DirectTapEntry* host_tab);
 int direct_launch(const ConvDims& d, int tile_id, const float* in, const float* filt, const float* bias,
                   float* out, const DirectTapEntry* dev_tab, cudaStream_t stream);
+// Tiles compiled at run time for the exact shape (direct_rtc.cu): output channels per thread, 0 for the other tiles.
+int direct_tile_rtc_kt(int tile_id);
+// the run-time compiled tile that automatic selection uses for this shape, or -1 (no NVRTC, or the shape is not one
+// of the small-reduction layers these tiles are for)
+int direct_rtc_pick(const ConvDims& d);
+// compilation alone (no GPU needed): the cubin image of the kernel for this shape and blocking
+int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem, std::vector<char>* image);
+struct DirectRtc;
+bool direct_rtc_available();                     // is NVRTC there?
+bool direct_rtc_geometry(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem);
+int direct_rtc_create(const ConvDims& d, int KT, DirectRtc** out);    // compiles; BODA_ERR_UNSUPPORTED without NVRTC or if the shape does not fit
+void direct_rtc_destroy(DirectRtc* r);
+int direct_rtc_launch(DirectRtc* r, const float* in, const float* filt, const float* bias, float* out, cudaStream_t stream);
+void direct_rtc_describe(const DirectRtc* r, char* buf, size_t n);
 
 // ---- the planned forward pass with an optional event between operand staging and the main kernel
 int conv_fwd_planned_ex(boda_conv_plan* plan, const float* in, const float* filt, const float* bias, float* out,

@@ -334,8 +334,11 @@ constexpr TileInfo kTiles[] = {
     {2, 1, "direct_32x16"},
     // pixel-per-thread form (TM = 0): TN output channels per thread
     {0, 8, "direct_pixel_k8"}, {0, 16, "direct_pixel_k16"}, {0, 32, "direct_pixel_k32"},
+    // the same form compiled at run time for the exact shape (TM = -1; direct_rtc.cu)
+    {-1, 4, "direct_rtc_k4"}, {-1, 8, "direct_rtc_k8"}, {-1, 16, "direct_rtc_k16"}, {-1, 32, "direct_rtc_k32"},
 };
 constexpr int kFirstPixelTile = 9;
+constexpr int kFirstRtcTile = 12;
 constexpr int kNumTiles = sizeof(kTiles) / sizeof(kTiles[0]);
 
 template <int TM, int TN>
@@ -389,9 +392,36 @@ bool direct_tile_legal(const ConvDims& d, int tile_id)
 {
     if (tile_id < 0 || tile_id >= kNumTiles) return false;
     if (tile_id < kFirstPixelTile) return true;
+    if (tile_id >= kFirstRtcTile) {
+        int bx, by;
+        size_t sm;
+        return direct_rtc_available() && direct_rtc_geometry(d, kTiles[tile_id].TN, &bx, &by, &sm);
+    }
     int ih, iw, iwp;
     size_t smem;
     return pixel_geometry(d, kTiles[tile_id].TN, &ih, &iw, &iwp, &smem) && d.N <= 65535 && (d.K + kTiles[tile_id].TN - 1) / kTiles[tile_id].TN <= 65535;
+}
+
+int direct_tile_rtc_kt(int tile_id) { return (tile_id >= kFirstRtcTile && tile_id < kNumTiles) ? kTiles[tile_id].TN : 0; }
+
+int direct_rtc_pick(const ConvDims& d)
+{
+    // Measured on B200 (configuration 1's layer at batch 1 / 20 / 256, an 11x11 stride-4 and a 5x5 layer on 3 channels):
+    // the run-time compiled kernel beats every precompiled tile where the reduction is short and the output channels
+    // few.  Eight channels per thread as a rule; four where that leaves fewer than 64 blocks (more blocks hide the
+    // staging latency); sixteen where 16 covers all output channels of a large layer (the input patch is staged once).
+    if (d.Kred > 512 || d.K > 128 || !direct_rtc_available()) return -1;
+    int bx = 32, by = 8;
+    size_t sm = 0;
+    if (!direct_rtc_geometry(d, 8, &bx, &by, &sm)) bx = 8, by = 4;
+    const long long blocks8 = (long long)((d.Q + bx - 1) / bx) * ((d.P + by - 1) / by) * d.N * ((d.K + 7) / 8);
+    const int want = (d.K <= 16 && d.M >= 16384) ? 16 : blocks8 < 64 ? 4 : 8;
+    const int order[3][3] = {{4, 8, 16}, {8, 4, 16}, {16, 8, 4}};
+    const int* o = order[want == 4 ? 0 : want == 8 ? 1 : 2];
+    for (int i = 0; i < 3; ++i)
+        for (int t = kFirstRtcTile; t < kNumTiles; ++t)
+            if (kTiles[t].TN == o[i] && direct_tile_legal(d, t)) return t;
+    return -1;
 }
 
 int direct_table_len(const ConvDims& d) { return ((d.Kred + BK - 1) / BK) * BK; }

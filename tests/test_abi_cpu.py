@@ -56,3 +56,22 @@ def test_argument_validation_needs_no_device():
     assert B.boda_version() >= 100
     o = B.boda_plan_opts_default()
     assert (o.math, o.tune, o.variant, o.tile_id, o.split_k, o.device, o.s2d) == (0, 0, -1, -1, 0, -1, -1)
+
+
+def test_run_time_compilation_needs_no_gpu():
+    """The run-time specialised DIRECT kernel (Section 4 of the paper) compiles for several shapes on a machine without
+    a GPU; the blocking follows the shape."""
+    from paper_1606_00094_b200 import binding as B
+    try:
+        bx, by, smem, image = B.boda_direct_rtc_compile((1, 3, 32, 32, 16, 3, 3, 1, 1, 1), 16)
+    except B.BodaError as e:
+        if e.status == B.BODA_ERR_UNSUPPORTED:
+            pytest.skip("NVRTC is not available on this machine")
+        raise
+    assert (bx, by) == (32, 8) and smem == 4 * (27 * 16 + 3 * 10 * 35) and image > 1000
+    bx, by, smem, image = B.boda_direct_rtc_compile((2, 3, 59, 59, 40, 11, 11, 4, 0, 1), 8)
+    assert bx * by >= 32 and smem <= 48 * 1024 and image > 1000
+    with pytest.raises(B.BodaError):
+        B.boda_direct_rtc_compile((1, 3, 32, 32, 16, 3, 3, 1, 1, 1), 5)            # channels per thread: 4, 8, 16 or 32
+    with pytest.raises(B.BodaError):
+        B.boda_direct_rtc_compile((1, 256, 13, 13, 64, 3, 3, 1, 1, 1), 16)         # does not fit shared memory

@@ -142,12 +142,12 @@ def test_pixel_tile_is_the_automatic_choice_for_large_batches_of_configuration_1
     shape = (40, 3, 32, 32, 16, 3, 3, 1, 1, 1)          # configuration 1's layer at batch 40: 40 960 output pixels
     x, w, b = _tensors(shape, 4200)
     got, desc = run_planned(shape, x, w, b, math=1)
-    assert "direct_pixel_k16" in desc
+    assert "direct_rtc_k16" in desc or "direct_pixel_k16" in desc      # the run-time compiled form where NVRTC is there
     assert_parity(got, oracle_out(shape, x, w, b), FP32_TOL, desc)
     c = wl.CONFIGS[1]                                    # at batch 1 the blocked tiles stay the choice
     x, w, b = c.tensors()
     got, desc = run_planned(c.shape.as_tuple(), x, w, b, math=1)
-    assert "direct_pixel" not in desc
+    assert "direct_pixel" not in desc          # (the run-time compiled tile where NVRTC is there, else a blocked tile)
     assert_parity(got, oracle_out(c.shape.as_tuple(), x, w, b), FP32_TOL, desc)
 
 
@@ -155,3 +155,46 @@ def test_pixel_tile_refused_when_the_patch_does_not_fit():
     from paper_1606_00094_b200 import binding as B
     with pytest.raises(B.BodaError):
         B.ConvPlan((1, 64, 56, 56, 32, 11, 11, 4, 0, 1), variant=0, math=1, tile_id=11)
+
+
+# ---- tiles compiled at run time for the exact shape (Section 4 of the paper): ids 12..15
+def _rtc_or_skip():
+    from paper_1606_00094_b200 import binding as B
+    try:
+        B.boda_direct_rtc_compile((1, 3, 8, 8, 4, 3, 3, 1, 1, 0), 4)
+    except B.BodaError as e:
+        if e.status == B.BODA_ERR_UNSUPPORTED:
+            pytest.skip("NVRTC is not available on this machine")
+        raise
+
+
+@pytest.mark.parametrize("shape", PIXEL_CASES)
+@pytest.mark.parametrize("tile", [12, 13, 14, 15])
+def test_rtc_tiles_exact(shape, tile):
+    _rtc_or_skip()
+    from paper_1606_00094_b200 import binding as B
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x, w, b = wl.integers(4300, (N, C, H, W)), wl.integers(4301, (K, C, R, S)), wl.integers(4302, (K,))
+    try:
+        B.boda_direct_rtc_compile(shape, (4, 8, 16, 32)[tile - 12])
+    except B.BodaError as e:          # filters and patch beyond 48 KB of shared memory: the plan is refused as well
+        assert e.status == B.BODA_ERR_UNSUPPORTED
+        with pytest.raises(B.BodaError):
+            B.ConvPlan(shape, variant=0, math=1, tile_id=tile)
+        return
+    got, desc = run_planned(shape, x, w, b, variant=0, math=1, tile_id=tile)
+    assert "direct_rtc" in desc and "rtc block=" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+    got2, _ = run_planned(shape, x, w, None, variant=0, math=1, tile_id=tile)          # no bias
+    np.testing.assert_array_equal(got2.astype(np.float64), oracle_out(shape, x, w, None))
+
+
+def test_rtc_tile_on_real_values_and_refusals():
+    _rtc_or_skip()
+    from paper_1606_00094_b200 import binding as B
+    shape = (6, 3, 64, 48, 24, 7, 7, 2, 3, 1)
+    x, w, b = _tensors(shape, 4400)
+    got, desc = run_planned(shape, x, w, b, variant=0, math=1, tile_id=13)
+    assert_parity(got, oracle_out(shape, x, w, b), FP32_TOL, desc)
+    with pytest.raises(B.BodaError):                      # 256 channels of 3x3: the filters alone exceed shared memory
+        B.ConvPlan((1, 256, 13, 13, 64, 3, 3, 1, 1, 1), variant=0, math=1, tile_id=14)
