@@ -178,8 +178,8 @@ int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, vo
 /*
  * Run-time compilation (Section 4 of the paper: kernels are generated and compiled for the exact problem once its
  * sizes are known, so that every extent is a literal).  The DIRECT tiles named direct_rtc_k4 / k8 / k16 / k32
- * (tile ids 12..15 of BODA_VARIANT_DIRECT; also what automatic selection uses in place of the pixel-per-thread
- * tiles) are compiled by NVRTC when their plan is created: one thread per output pixel and `kt` output channels,
+ * (tile ids 12..15 of BODA_VARIANT_DIRECT; also what automatic selection uses for layers with C*R*S <= 512 and
+ * K <= 128 that stay on the FP32 kernel) are compiled by NVRTC when their plan is created: one thread per output pixel and `kt` output channels,
  * all of N, C, H, W, K, R, S, stride, pad, ReLU and the blocking as compile-time constants.  They need the NVRTC
  * shared library at run time (looked up with dlopen; without it those tiles return BODA_ERR_UNSUPPORTED and
  * automatic selection keeps the precompiled kernels) and an input patch plus filters of at most 48 KB.

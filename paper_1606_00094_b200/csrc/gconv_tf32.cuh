@@ -51,7 +51,8 @@ template <int BN> struct Cfg {
     static constexpr int B_STAGE_BYTES = BN * 128;
     static constexpr int STAGE_BYTES = A_STAGE_BYTES + B_STAGE_BYTES;
     static constexpr int TMEM_COLS = 2 * BN <= 128 ? 128 : 2 * BN <= 256 ? 256 : 512;
-    static constexpr uint32_t OUT_TILE_BYTES = 128u * out_tile_row_bytes<BN>();
+    // the staged-layout output tile; the widest tile has no room for one and stores from registers instead
+    static constexpr uint32_t OUT_TILE_BYTES = BN <= 128 ? 128u * out_tile_row_bytes<BN>() : 0u;
     static constexpr int SMEM_BYTES = STAGES * STAGE_BYTES + (int)OUT_TILE_BYTES + 1024 /*alignment slack*/ + 256 /*barriers*/;
 };
 
@@ -190,7 +191,8 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
                 }
                 d = row_dst(p.o, valid, n, pp, qq);
             }
-            if (p.o.packed && t > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // this row's slot is free again
+            const bool via_tile = C::OUT_TILE_BYTES != 0 && p.o.packed;     // staged rows leave through shared memory as bulk copies
+            if (via_tile && t > 0) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");   // this row's slot is free again
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -198,20 +200,20 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
                 tmem_ld_wait();
                 float y[32];
                 bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
-                if (p.o.packed) out_tile_put32(row_addr, 32 * c, y);
+                if (via_tile) out_tile_put32(row_addr, 32 * c, y);
                 else store_row32(p.o, d, k0 + 32 * c, y);
             }
             // the accumulator has been read: hand the slot back to the issuer
             tc_fence_before();
             __syncwarp();
             if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(acc_empty + 8 * slot) : "memory");
-            if (p.o.packed) {
+            if (via_tile) {
                 fence_proxy_async_smem();
                 out_tile_store_row(p.o, d, k0, BN, row_addr);
                 bulk_commit();
             }
         }
-        if (p.o.packed) bulk_wait_all();
+        if (C::OUT_TILE_BYTES != 0 && p.o.packed) bulk_wait_all();
     } else {
         // ---------------- gather producers: group g builds the stages of chunks g, g + 3, ... of the CTA's chunk sequence
         const int pw = warp - kFirstProducerWarp;

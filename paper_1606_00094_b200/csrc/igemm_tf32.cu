@@ -597,11 +597,12 @@ int load_driver_entry_points()
     return BODA_OK;
 }
 
-// Tile table.  Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
+// Tile table.  Ids 16..19: gather kernel (gconv_tf32.cuh; NCHW input, tconv with short reductions and k1conv).
+// Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
 // with NACC accumulators of 128 rows each (ids 5..8: 1, 9..12: 2, 13..15: 4).
 // accumulators per tile: 0 = im2col kernel, 1 / 2 / 4 = halo kernel, -1 = gather kernel (gconv_tf32.cuh)
-constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128};
-constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1};
+constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128, 192};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1, -1};
 constexpr int kFirstGatherTile = 16;
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
 constexpr int kFirstHaloTile = 5;
@@ -784,7 +785,7 @@ double model_cost_halo(const ConvDims& d, int Cp, int BN, int nacc, int splits)
 // because nothing is staged (the other tensor-core paths pay about 6000 clocks for their staging kernel).
 bool gather_legal(const ConvDims& d, int variant, bool x3)
 {
-    if (variant != BODA_VARIANT_TCONV || x3) return false;
+    if ((variant != BODA_VARIANT_TCONV && variant != BODA_VARIANT_K1CONV) || x3) return false;
     const int Kp = ((d.Kred + 31) / 32) * 32;
     return Kp <= gconv::kMaxKred && d.K >= 8 && (long long)d.N * d.C * d.H * d.W < (1LL << 31);
 }
@@ -1006,7 +1007,9 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
             if (s > p->iters_total) continue;
-            const double staging = 6000.0;         // the input staging kernel these tiles need and the gather tiles do not
+            // the input staging kernel these tiles need and the gather tiles do not: a launch, or the time to read
+            // the input and write its staged copy (about 3000 bytes per clock measured on staging kernels)
+            const double staging = std::max(6000.0, ((double)d_in.N * d_in.C * d_in.H * d_in.W + (double)d.N * d.H * d.W * p->Cp) * 4.0 / 3000.0);
             const double c = staging + (nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms, kTileBN[t], s));
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
@@ -1216,6 +1219,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
             case 64: return launch_gather<64>(p, gp, stream);
             case 96: return launch_gather<96>(p, gp, stream);
             case 128: return launch_gather<128>(p, gp, stream);
+            case 192: return launch_gather<192>(p, gp, stream);
             default: return BODA_ERR_UNSUPPORTED;
         }
     }

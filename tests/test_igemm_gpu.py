@@ -185,7 +185,7 @@ def test_space_to_depth_refused_for_stride_one():
     assert e.value.status == B.BODA_ERR_UNSUPPORTED
 
 
-# ---- gather kernel (tiles 16..18): the input tile is built by producer warps straight from NCHW
+# ---- gather kernel (tiles 16..19): the input tile is built by producer warps straight from NCHW
 GATHER_CASES = [
     (2, 3, 23, 23, 40, 11, 11, 4, 0, 1),       # conv1-like: no padding, 363 reduction indices (ragged last chunk)
     (1, 3, 32, 32, 16, 3, 3, 1, 1, 1),         # configuration 1: one ragged chunk, padding on all sides
@@ -198,7 +198,7 @@ GATHER_CASES = [
 
 
 @pytest.mark.parametrize("shape", GATHER_CASES)
-@pytest.mark.parametrize("tile", [16, 17, 18])
+@pytest.mark.parametrize("tile", [16, 17, 18, 19])
 def test_gather_tiles_exact(shape, tile):
     x, w, b = _int_tensors(shape, 2100)
     got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile)
@@ -232,3 +232,28 @@ def test_gather_refused_where_it_does_not_apply():
         B.ConvPlan((1, 3, 32, 32, 16, 3, 3, 1, 1, 1), variant=TC, tile_id=17, split_k=2)
     with pytest.raises(B.BodaError):
         B.ConvPlan((1, 3, 33, 33, 16, 3, 3, 2, 1, 1), variant=TC, tile_id=17, s2d=1)
+
+
+# the gather kernel also runs 1x1 layers straight from NCHW (consecutive output points are consecutive addresses):
+# no staged copy of the input, which is what large batches of such layers spend their time on otherwise
+@pytest.mark.parametrize("shape", [
+    (5, 40, 7, 9, 200, 1, 1, 1, 0, 0),            # C not a multiple of 32, K ragged against every tile, tiles straddle images
+    (3, 480, 14, 14, 192, 1, 1, 1, 0, 1),         # configuration 3's layer
+    (2, 64, 9, 9, 24, 1, 1, 2, 0, 1),             # stride 2
+])
+@pytest.mark.parametrize("tile", [16, 19])
+def test_gather_tiles_run_k1conv_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 1700)
+    got, desc = run_planned(shape, x, w, b, variant=K1, tile_id=tile)
+    assert "gconv" in desc and "k1conv" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_large_batch_k1conv_chooses_the_gather_kernel_and_small_batch_does_not():
+    from paper_1606_00094_b200 import binding as B
+    big = B.ConvPlan((256, 480, 14, 14, 192, 1, 1, 1, 0, 1))
+    small = B.ConvPlan((5, 480, 14, 14, 192, 1, 1, 1, 0, 1))
+    try:
+        assert "gconv_128x192" in big.describe() and "gconv" not in small.describe()
+    finally:
+        big.close(); small.close()
