@@ -181,8 +181,9 @@ int boda_sgemm(const float* A, const float* B, float* C, int M, int N, int K, vo
  * (tile ids 12..15 of BODA_VARIANT_DIRECT; also what automatic selection uses for layers with C*R*S <= 512 and
  * K <= 128 that stay on the FP32 kernel) are compiled by NVRTC when their plan is created: one thread per output pixel and `kt` output channels,
  * all of N, C, H, W, K, R, S, stride, pad, ReLU and the blocking as compile-time constants.  They need the NVRTC
- * shared library at run time (looked up with dlopen; without it those tiles return BODA_ERR_UNSUPPORTED and
- * automatic selection keeps the precompiled kernels) and an input patch plus filters of at most 48 KB.
+ * shared library at run time (looked up with dlopen; without it - or with BODA_NO_RTC=1 in the environment - those
+ * tiles return BODA_ERR_UNSUPPORTED and automatic selection keeps the precompiled kernels; the first plan for a
+ * shape pays the compilation, 0.3 to 3 seconds) and an input patch plus filters of at most 48 KB.
  *
  * boda_direct_rtc_compile compiles the kernel for `shape` without loading or running it - it needs no GPU - and
  * reports the blocking chosen and the size of the device image.  Any of the four output pointers may be NULL.

@@ -8,6 +8,7 @@
 #include <nvrtc.h>
 
 #include <cstdio>
+#include <cstdlib>
 #include <map>
 #include <mutex>
 #include <new>
@@ -38,6 +39,8 @@ NvrtcApi* nvrtc_api()
     static NvrtcApi api;
     static std::once_flag once;
     std::call_once(once, [] {
+        const char* off = std::getenv("BODA_NO_RTC");        // "1": behave as if NVRTC were not installed
+        if (off && *off == '1') return;
         const char* names[] = {"libnvrtc.so.12", "libnvrtc.so", "/usr/local/cuda/lib64/libnvrtc.so.12", "/usr/local/cuda/lib64/libnvrtc.so"};
         for (const char* nm : names) {
             api.handle = dlopen(nm, RTLD_NOW | RTLD_LOCAL);
