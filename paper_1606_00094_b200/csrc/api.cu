@@ -549,13 +549,13 @@ int boda_direct_rtc_compile(const boda_conv_shape* shape, int kt, int* block_x, 
 {
     if (!shape || !shape_ok(*shape) || (kt != 4 && kt != 8 && kt != 16 && kt != 32)) return BODA_ERR_INVALID_ARG;
     const ConvDims d = make_dims(*shape);
-    int bx = 0, by = 0;
+    int bx = 0, by = 0, py = 1;
     size_t smem = 0;
     std::vector<char> image;
-    const int rc = direct_rtc_compile(d, kt, &bx, &by, &smem, &image);
+    const int rc = direct_rtc_compile(d, kt, &bx, &by, &py, &smem, &image);
     if (rc != BODA_OK) return rc;
     if (block_x) *block_x = bx;
-    if (block_y) *block_y = by;
+    if (block_y) *block_y = by * py;
     if (smem_bytes) *smem_bytes = smem;
     if (image_bytes) *image_bytes = image.size();
     return BODA_OK;

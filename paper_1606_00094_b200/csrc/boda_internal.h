@@ -105,10 +105,10 @@ int direct_tile_rtc_kt(int tile_id);
 // of the small-reduction layers these tiles are for)
 int direct_rtc_pick(const ConvDims& d);
 // compilation alone (no GPU needed): the cubin image of the kernel for this shape and blocking
-int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem, std::vector<char>* image);
+int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, int* PY, size_t* smem, std::vector<char>* image);
 struct DirectRtc;
 bool direct_rtc_available();                     // is NVRTC there?
-bool direct_rtc_geometry(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem);
+bool direct_rtc_geometry(const ConvDims& d, int KT, int* BX, int* BY, int* PY, size_t* smem);
 int direct_rtc_create(const ConvDims& d, int KT, DirectRtc** out);    // compiles; BODA_ERR_UNSUPPORTED without NVRTC or if the shape does not fit
 void direct_rtc_destroy(DirectRtc* r);
 int direct_rtc_launch(DirectRtc* r, const float* in, const float* filt, const float* bias, float* out, cudaStream_t stream);

@@ -393,9 +393,9 @@ bool direct_tile_legal(const ConvDims& d, int tile_id)
     if (tile_id < 0 || tile_id >= kNumTiles) return false;
     if (tile_id < kFirstPixelTile) return true;
     if (tile_id >= kFirstRtcTile) {
-        int bx, by;
+        int bx, by, py;
         size_t sm;
-        return direct_rtc_available() && direct_rtc_geometry(d, kTiles[tile_id].TN, &bx, &by, &sm);
+        return direct_rtc_available() && direct_rtc_geometry(d, kTiles[tile_id].TN, &bx, &by, &py, &sm);
     }
     int ih, iw, iwp;
     size_t smem;
@@ -411,10 +411,10 @@ int direct_rtc_pick(const ConvDims& d)
     // few.  Eight channels per thread as a rule; four where that leaves fewer than 64 blocks (more blocks hide the
     // staging latency); sixteen where 16 covers all output channels of a large layer (the input patch is staged once).
     if (d.Kred > 512 || d.K > 128 || !direct_rtc_available()) return -1;
-    int bx = 32, by = 8;
+    int bx = 32, by = 8, py = 1;
     size_t sm = 0;
-    if (!direct_rtc_geometry(d, 8, &bx, &by, &sm)) bx = 8, by = 4;
-    const long long blocks8 = (long long)((d.Q + bx - 1) / bx) * ((d.P + by - 1) / by) * d.N * ((d.K + 7) / 8);
+    if (!direct_rtc_geometry(d, 8, &bx, &by, &py, &sm)) bx = 8, by = 4, py = 1;
+    const long long blocks8 = (long long)((d.Q + bx - 1) / bx) * ((d.P + by * py - 1) / (by * py)) * d.N * ((d.K + 7) / 8);
     const int want = (d.K <= 16 && d.M >= 16384) ? 16 : blocks8 < 64 ? 4 : 8;
     const int order[3][3] = {{4, 8, 16}, {8, 4, 16}, {16, 8, 4}};
     const int* o = order[want == 4 ? 0 : want == 8 ? 1 : 2];

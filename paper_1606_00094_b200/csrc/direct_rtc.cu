@@ -71,25 +71,35 @@ std::string def(const char* name, long long v)
 
 struct DirectRtc {
     ConvDims d;
-    int KT = 16, BX = 32, BY = 8;
+    int KT = 16, BX = 32, BY = 8, PY = 1;
     size_t smem = 0, cubin_bytes = 0;
     cudaLibrary_t lib = nullptr;
     cudaKernel_t kernel = nullptr;
 };
 
-// Blocking for a shape: the widest block patch (32 x 8, 16 x 8, 16 x 4, 8 x 4 output pixels) whose input patch and
-// filters fit the 48 KB of static shared memory; false if none does.
-bool direct_rtc_geometry(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem)
+// Blocking for a shape: the widest thread block (32 x 8, 16 x 8, 16 x 4, 8 x 4 threads) and the most output rows per
+// thread (4, 2, 1: the weights of a tap are loaded once for all of a thread's rows) such that the input patch and the
+// filters fit the 48 KB of static shared memory and the grid still has a few blocks per SM; false if nothing fits.
+bool direct_rtc_geometry(const ConvDims& d, int KT, int* BX, int* BY, int* PY, size_t* smem)
 {
     if (KT % 4 != 0 || KT < 4 || KT > 32) return false;
     if (d.N > 65535 || (d.K + KT - 1) / KT > 65535) return false;
+    int force_py = 0;
+    if (const char* e = std::getenv("BODA_RTC_ROWS_PER_THREAD")) force_py = std::atoi(e);     // measurement hook: 1, 2 or 4
     const int cand[4][2] = {{32, 8}, {16, 8}, {16, 4}, {8, 4}};
+    const int pys[3] = {4, 2, 1};
     for (const auto& c : cand) {
         // no wider than the output row needs (a 13-pixel row does not want a 32-pixel patch)
         if (c[0] >= 2 * d.Q && c[0] > 8) continue;
-        const int ih = (c[1] - 1) * d.stride + d.R, iw = (c[0] - 1) * d.stride + d.S, iwp = iw | 1;
-        const size_t bytes = ((size_t)d.Kred * KT + (size_t)d.C * ih * iwp) * sizeof(float);
-        if (bytes <= 48 * 1024 - 64) { *BX = c[0]; *BY = c[1]; *smem = bytes; return true; }
+        for (int py : pys) {
+            if (force_py > 0 && py != force_py) continue;
+            if (py > 1 && KT * py > 64) continue;                                  // accumulators stay in registers
+            const long long blocks = (long long)((d.Q + c[0] - 1) / c[0]) * ((d.P + c[1] * py - 1) / (c[1] * py)) * d.N * ((d.K + KT - 1) / KT);
+            if (force_py == 0 && py > 1 && (blocks < 8 * 148 || c[1] * py > d.P)) continue;
+            const int ih = (c[1] * py - 1) * d.stride + d.R, iw = (c[0] - 1) * d.stride + d.S, iwp = iw | 1;
+            const size_t bytes = ((size_t)d.Kred * KT + (size_t)d.C * ih * iwp) * sizeof(float);
+            if (bytes <= 48 * 1024 - 64) { *BX = c[0]; *BY = c[1]; *PY = py; *smem = bytes; return true; }
+        }
     }
     return false;
 }
@@ -111,14 +121,14 @@ struct ImageCache {
 };
 static ImageCache& image_cache() { static ImageCache c; return c; }
 
-int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem, std::vector<char>* image)
+int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, int* PY, size_t* smem, std::vector<char>* image)
 {
     NvrtcApi* api = nvrtc_api();
     if (!api->ok) return BODA_ERR_UNSUPPORTED;
-    if (!direct_rtc_geometry(d, KT, BX, BY, smem)) return BODA_ERR_UNSUPPORTED;
+    if (!direct_rtc_geometry(d, KT, BX, BY, PY, smem)) return BODA_ERR_UNSUPPORTED;
     char key[160];
-    std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,%d,kt%d,%dx%d", d.N, d.C, d.H, d.W, d.K, d.R, d.S, d.stride, d.pad,
-                  d.relu, KT, *BX, *BY);
+    std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,%d,kt%d,%dx%dx%d", d.N, d.C, d.H, d.W, d.K, d.R, d.S, d.stride, d.pad,
+                  d.relu, KT, *BX, *BY, *PY);
     {
         std::lock_guard<std::mutex> lock(image_cache().mu);
         auto it = image_cache().images.find(key);
@@ -126,14 +136,15 @@ int direct_rtc_compile(const ConvDims& d, int KT, int* BX, int* BY, size_t* smem
     }
     // full unrolling of the reduction while the kernel stays a few thousand instructions long (compilation time
     // grows faster than the body: 0.3 s for 600 instructions, 5 s for 4000); otherwise the window, or its rows, only
-    const long long body = (long long)d.Kred * (KT + KT / 4 + 1);
+    const long long per_tap = (long long)KT * *PY + KT / 4 + *PY;
+    const long long body = (long long)d.Kred * per_tap;
     const int unroll_c = body <= 2500 ? d.C : 1;
-    const int unroll_r = (body <= 2500 || (long long)d.R * d.S * (KT + KT / 4 + 1) <= 2500) ? d.R : 1;
+    const int unroll_r = (body <= 2500 || (long long)d.R * d.S * per_tap <= 2500) ? d.R : 1;
     std::vector<std::string> opts = {
         "--gpu-architecture=sm_100a", "--std=c++17", "-lineinfo",
         def("N", d.N), def("C", d.C), def("H", d.H), def("W", d.W), def("K", d.K), def("R", d.R), def("S", d.S),
         def("STRIDE", d.stride), def("PAD", d.pad), def("RELU", d.relu), def("P", d.P), def("Q", d.Q),
-        def("KT", KT), def("BX", *BX), def("BY", *BY), def("UNROLL_C", unroll_c), def("UNROLL_R", unroll_r),
+        def("KT", KT), def("BX", *BX), def("BY", *BY), def("PY", *PY), def("UNROLL_C", unroll_c), def("UNROLL_R", unroll_r),
     };
     std::vector<const char*> optp;
     for (const auto& o : opts) optp.push_back(o.c_str());
@@ -168,7 +179,7 @@ int direct_rtc_create(const ConvDims& d, int KT, DirectRtc** out)
     r->d = d;
     r->KT = KT;
     std::vector<char> image;
-    const int rc = direct_rtc_compile(d, KT, &r->BX, &r->BY, &r->smem, &image);
+    const int rc = direct_rtc_compile(d, KT, &r->BX, &r->BY, &r->PY, &r->smem, &image);
     if (rc != BODA_OK) { delete r; return rc; }
     r->cubin_bytes = image.size();
     cudaError_t e = cudaLibraryLoadData(&r->lib, image.data(), nullptr, nullptr, 0, nullptr, nullptr, 0);
@@ -182,7 +193,7 @@ int direct_rtc_launch(DirectRtc* r, const float* in, const float* filt, const fl
 {
     const ConvDims& d = r->d;
     cudaLaunchConfig_t cfg = {};
-    cfg.gridDim = dim3(((d.Q + r->BX - 1) / r->BX) * ((d.P + r->BY - 1) / r->BY), d.N, (d.K + r->KT - 1) / r->KT);
+    cfg.gridDim = dim3(((d.Q + r->BX - 1) / r->BX) * ((d.P + r->BY * r->PY - 1) / (r->BY * r->PY)), d.N, (d.K + r->KT - 1) / r->KT);
     cfg.blockDim = dim3(r->BX * r->BY);
     cfg.dynamicSmemBytes = 0;
     cfg.stream = stream;
@@ -203,7 +214,7 @@ int direct_rtc_launch(DirectRtc* r, const float* in, const float* filt, const fl
 
 void direct_rtc_describe(const DirectRtc* r, char* buf, size_t n)
 {
-    std::snprintf(buf, n, "rtc block=%dx%d kt=%d smem=%zu cubin=%zu", r->BX, r->BY, r->KT, r->smem, r->cubin_bytes);
+    std::snprintf(buf, n, "rtc block=%dx%d rows=%d kt=%d smem=%zu cubin=%zu", r->BX, r->BY, r->PY, r->KT, r->smem, r->cubin_bytes);
 }
 
 }  // namespace boda

@@ -198,3 +198,15 @@ def test_rtc_tile_on_real_values_and_refusals():
     assert_parity(got, oracle_out(shape, x, w, b), FP32_TOL, desc)
     with pytest.raises(B.BodaError):                      # 256 channels of 3x3: the filters alone exceed shared memory
         B.ConvPlan((1, 256, 13, 13, 64, 3, 3, 1, 1, 1), variant=0, math=1, tile_id=14)
+
+
+@pytest.mark.parametrize("rows", ["2", "4"])
+def test_rtc_tile_with_several_rows_per_thread(rows, monkeypatch):
+    _rtc_or_skip()
+    monkeypatch.setenv("BODA_RTC_ROWS_PER_THREAD", rows)        # large layers choose this themselves; forced here on a small one
+    shape = (3, 3, 45, 70, 20, 5, 5, 2, 2, 1)
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x, w, b = wl.integers(4500, (N, C, H, W)), wl.integers(4501, (K, C, R, S)), wl.integers(4502, (K,))
+    got, desc = run_planned(shape, x, w, b, variant=0, math=1, tile_id=13)
+    assert f"rows={rows}" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
