@@ -150,6 +150,8 @@ S2D_SHAPES = [
     (2, 8, 16, 16, 40, 2, 2, 2, 0, 1),           # window = stride: the view is a 1x1 convolution
     (1, 5, 20, 23, 33, 7, 7, 3, 3, 0),           # stride 3, window not a multiple of the stride, padding
     (3, 16, 9, 9, 16, 3, 3, 2, 1, 1),
+    (2, 3, 50, 61, 16, 7, 7, 4, 3, 1),           # stride 4 on 3 channels with padding and odd extents (the specialised staging kernel)
+    (1, 3, 300, 251, 16, 9, 9, 4, 2, 0),         # rows longer than 256 staged columns: more than one pass of staging loads
 ]
 
 
