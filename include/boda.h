@@ -287,8 +287,13 @@ int boda_stack_fwd_eager(boda_stack* stack, const float* in, float* out, void* s
 /* Runs op `op_index` alone on the activations that the last forward pass left in the stack (for timing one layer
  * in place).  `in` is read only by op 0 and `out` written only by the last op; pass NULL otherwise. */
 int boda_stack_run_op(boda_stack* stack, int op_index, const float* in, float* out, void* stream);
-/* Forward pass with HOST buffers: copies `in_host` to the device, runs boda_stack_fwd, copies the result into
- * `out_host` and synchronises `stream`.  Pinned host memory makes the copies asynchronous. */
+/* Forward pass with HOST buffers: copies `in_host` to the device, runs the chain, copies the result into
+ * `out_host` and synchronises `stream`.  Pinned host memory makes the copies asynchronous.  Batch items are
+ * independent (Section 2 of the paper), so for even N >= 4 the batch is copied in two slices (BODA_STACK_HOST_CHUNKS=k: k slices) on a second
+ * stream and each slice runs, as soon as it has arrived, through a stack of the same layers planned for the
+ * sub-batch (created on the first call; same filters; BODA_STACK_HOST_CHUNKS=1 in the environment keeps the batch
+ * whole): host-to-device copies and kernels overlap.  Results meet the same error bars as boda_stack_fwd but need
+ * not be bitwise equal to it (the sub-batch plans may sum in another order). */
 int boda_stack_fwd_host(boda_stack* stack, const float* in_host, float* out_host, void* stream);
 
 /*

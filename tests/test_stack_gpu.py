@@ -50,11 +50,21 @@ def test_stack_every_layer_matches_fp64_chain(batch, math, tol, tune):
             assert got.shape == r.shape
             err = orc.rel_l2(got, r)
             assert err <= tol, f"op {i} ({descs[i]}): rel-L2 {err:.3e} > {tol:.0e}"
-        # host-buffer entry point and the eager path give the same numbers
+        # host-buffer entry point: from batch 4 on it runs the batch in slices through plans made for the sub-batch
+        # (copies overlap kernels), so it is held to the oracle like the device path, and to itself bit for bit;
+        # smaller batches take the very same graph
         hx = torch.from_numpy(x).pin_memory()
         ho = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+        ho2 = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
         stack.forward_host(hx, ho)
-        assert torch.equal(ho, out_graph.cpu())
+        stack.forward_host(hx, ho2)
+        assert B.boda_query_status() == 0
+        assert torch.equal(ho, ho2)
+        if batch < 4:
+            assert torch.equal(ho, out_graph.cpu())
+        else:
+            err = orc.rel_l2(ho.numpy(), ref[-1])
+            assert err <= tol, f"host path: rel-L2 {err:.3e} > {tol:.0e}"
         eager = stack.forward_eager(dx).clone()
         torch.cuda.synchronize()
         assert torch.equal(eager, out_graph)
