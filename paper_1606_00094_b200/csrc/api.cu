@@ -172,7 +172,7 @@ bool conv_plan_input_geometry(const boda_conv_plan* p, int* Hp, int* Wp, int* Cp
     return p->ig ? igemm_plan_input_geometry(p->ig, Hp, Wp, Cp) : false;
 }
 
-bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && p->math != BODA_MATH_TF32X3; }
+bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && p->math != BODA_MATH_TF32X3 && igemm_plan_writes_packed(p->ig); }
 
 int conv_plan_set_io(boda_conv_plan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {

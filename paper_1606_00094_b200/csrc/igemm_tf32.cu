@@ -31,6 +31,7 @@
 #include "tc_ptx.cuh"
 #include "tconv_halo.cuh"
 #include "gconv_tf32.cuh"
+#include "k1nchw_tf32.cuh"
 
 namespace boda {
 namespace {
@@ -652,8 +653,11 @@ int load_driver_entry_points()
 // Ids 0..4: im2col kernel (any stride; k1conv and tconv).  Ids 5..12: halo kernel (tconv, stride 1)
 // with NACC accumulators of 128 rows each (ids 5..8: 1, 9..12: 2, 13..15: 4).
 // accumulators per tile: 0 = im2col kernel, 1 / 2 / 4 = halo kernel, -1 = gather kernel (gconv_tf32.cuh)
-constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128, 192};
-constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1, -1};
+// Ids 20..22: 1x1 layers by TMA straight from NCHW (k1nchw_tf32.cuh), accumulator code -2.
+constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128, 192,
+                           /*1x1 from NCHW*/ 64, 128, 192};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1, -1, -2, -2, -2};
+constexpr int kFirstK1nTile = 20;
 constexpr int kFirstGatherTile = 16;
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
 constexpr int kFirstHaloTile = 5;
@@ -690,7 +694,7 @@ struct IgemmPlan {
     int gather_chunks = 0;           // ceil(C*R*S / 32)
     int sm_count = 148;
     // halo kernel only
-    int nacc = 0;                    // 0: im2col kernel; 1, 2 or 4: halo kernel with that many accumulators; -1: gather kernel
+    int nacc = 0;                    // 0: im2col kernel; 1, 2 or 4: halo kernel with that many accumulators; -1: gather kernel; -2: 1x1 from NCHW
     int Hp = 0, Wp = 0, lead = 0, slab_rows = 0, nbox = 0, box_rows = 0, a_slot_bytes = 0, b_stages = 0;
 };
 
@@ -846,7 +850,9 @@ double model_cost_gather(const ConvDims& d, int BN, int sm_count)
     const long long tiles = (long long)((d.M + BM - 1) / BM) * ((d.K + BN - 1) / BN);
     const double per_cta = (double)((tiles + sm_count - 1) / sm_count);
     const int chunks = (d.Kred + 31) / 32;
-    return per_cta * chunks * std::max(2.0 * BN, d.pad ? 1500.0 : 1250.0) + 4500.0 + 32.0 * BN;
+    // 1x1 layers gather whole 128-byte lines (consecutive output points are consecutive addresses): about 1000 clocks
+    const double gather = d.R * d.S == 1 ? 1000.0 : d.pad ? 1500.0 : 1250.0;
+    return per_cta * chunks * std::max(2.0 * BN, gather) + 4500.0 + 32.0 * BN;
 }
 
 // filters [K][C*R*S] -> [K][Kp] rounded to TF32, zeros past C*R*S: the K-major B operand of the gather kernel
@@ -874,6 +880,63 @@ int launch_gather(IgemmPlan* p, const gconv::GconvParams& prm, cudaStream_t stre
     const int grid = std::min(prm.tiles_total, p->sm_count);
     BODA_CUDA_TRY(launch_kernel(gconv::gconv_tf32_kernel<BN>, dim3(grid), dim3(gconv::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
                                 p->map_b, prm));
+    count_launch();
+    return BODA_OK;
+}
+
+// 1x1 from NCHW: stride 1, no padding, rows of HW floats that TMA can address (16-byte multiples), and the staged
+// output layout is not offered (tiles follow images, not the flat output-point index of a consumer's tiles - the
+// stores themselves would work).
+bool k1n_legal(const ConvDims& d, int variant, bool x3)
+{
+    if (variant != BODA_VARIANT_K1CONV || x3) return false;
+    if (d.R != 1 || d.S != 1 || d.stride != 1 || d.pad != 0) return false;
+    return (d.H * d.W) % 4 == 0 && (long long)d.N * ((d.H * d.W + BM - 1) / BM) <= 0x7fffffffLL;
+}
+
+// One kernel, no staging: about 380 clocks per 32-channel step (or the MMAs' 2*BN), 3500 of prologue and tail,
+// 32 per output channel of epilogue; tiles follow images, so an image of HW points costs ceil(HW/128) tiles.
+double model_cost_k1n(const ConvDims& d, int BN, int sm_count)
+{
+    const long long tiles = (long long)d.N * ((d.H * d.W + BM - 1) / BM) * ((d.K + BN - 1) / BN);
+    const double waves = (double)((tiles + sm_count - 1) / sm_count);
+    const int steps = (d.C + BKC - 1) / BKC;
+    return waves * (steps * std::max(2.0 * BN, 380.0) + 3500.0 + 32.0 * BN);
+}
+
+int encode_map_a_k1n(IgemmPlan* p, const void* in)
+{
+    const ConvDims& d = p->d;
+    const cuuint64_t HW = (cuuint64_t)d.H * d.W;
+    const cuuint64_t dims[3] = {HW, (cuuint64_t)d.C, (cuuint64_t)d.N};
+    const cuuint64_t strides[2] = {HW * 4, HW * d.C * 4};
+    const cuuint32_t box[3] = {32, BKC, 1};
+    const cuuint32_t estr[3] = {1, 1, 1};
+    // MN-major TF32 operands take the 128-byte swizzle in 32-byte pieces (the only layout the tensor core accepts for them)
+    CUresult r = g_encode_tiled(&p->map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, const_cast<void*>(in), dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B_ATOM_32B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (NCHW input) failed with CUresult %d", (int)r);
+        return record_cuda_error(cudaErrorInvalidValue, msg);
+    }
+    p->map_a_base = in;
+    return BODA_OK;
+}
+
+template <int BN>
+int launch_k1n(IgemmPlan* p, const k1n::K1nParams& prm, cudaStream_t stream)
+{
+    using C = k1n::Cfg<BN>;
+    static bool attr_set = false;
+    if (!attr_set) {
+        BODA_CUDA_TRY(cudaFuncSetAttribute(k1n::k1nchw_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
+        attr_set = true;
+    }
+    dim3 grid(p->tiles_m, p->tiles_n);
+    BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
+                                p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
 }
@@ -958,7 +1021,7 @@ int encode_map_a(IgemmPlan* p, const void* xp)
 int encode_map_b(IgemmPlan* p)
 {
     const ConvDims& d = p->d;
-    if (p->nacc < 0) {
+    if (p->nacc == -1) {
         const cuuint64_t Kp = (cuuint64_t)p->gather_chunks * 32;
         const cuuint64_t gdims[2] = {Kp, (cuuint64_t)d.K};
         const cuuint64_t gstrides[1] = {Kp * 4};
@@ -999,7 +1062,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     ConvDims d = d_in;
     bool use_s2d = false;
     if (x3 && s2d > 0) return BODA_ERR_UNSUPPORTED;      // the error-compensated mode runs on the im2col kernel only
-    const bool force_gather = tile_id >= kFirstGatherTile;
+    const bool force_gather = tile_id >= kFirstGatherTile && tile_id < kFirstK1nTile;
     if (force_gather && (s2d > 0 || !gather_legal(d_in, variant, x3))) return BODA_ERR_UNSUPPORTED;
     if (variant == BODA_VARIANT_TCONV && s2d != 0 && !x3 && !force_gather) {
         ConvDims e;
@@ -1047,6 +1110,12 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     for (int t = 0; t < kNumIgemmTiles; ++t) {
         if (tile_id >= 0 && t != tile_id) continue;
         const int nacc = kTileNacc[t];
+        if (nacc == -2) {
+            if (!k1n_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) continue;
+            const double c = model_cost_k1n(d_in, kTileBN[t], p->sm_count);
+            if (c < best) { best = c; best_t = t; best_s = 1; }
+            continue;
+        }
         if (nacc < 0) {
             // the gather kernel works on the layer as given (never on a space-to-depth view) and has no split
             if (!gather_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) continue;
@@ -1070,6 +1139,25 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->tile_id = best_t;
     p->BN = kTileBN[best_t];
     p->nacc = kTileNacc[best_t];
+    if (p->nacc == -2) {
+        // ---- 1x1 from NCHW: no staged input; filters [K][Cp] as for the im2col kernel
+        if (!k1n_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) { delete p; return BODA_ERR_UNSUPPORTED; }
+        p->d = d_in;
+        p->s2d = false;
+        p->Cp = ((d_in.C + BKC - 1) / BKC) * BKC;
+        p->splits = 1;
+        p->iters_total = p->iters_per_split = p->Cp / BKC;
+        p->tiles_m = d_in.N * ((d_in.H * d_in.W + BM - 1) / BM);
+        p->tiles_n = (d_in.K + p->BN - 1) / p->BN;
+        p->xp_bytes = 0;
+        p->partial_bytes = 0;
+        cudaError_t ke = cudaMalloc(&p->d_wp, (size_t)d_in.K * p->Cp * 4);
+        if (ke != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(ke, "plan allocation"); }
+        rc = encode_map_b(p);
+        if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
+        *out = p;
+        return BODA_OK;
+    }
     if (p->nacc < 0) {
         // ---- gather kernel: no staged input, filters flat [K][Kp], offset table on the device
         if (!gather_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) { delete p; return BODA_ERR_UNSUPPORTED; }
@@ -1135,12 +1223,18 @@ void igemm_plan_destroy(IgemmPlan* p)
 }
 
 int igemm_plan_tile(const IgemmPlan* p) { return p->tile_id; }
+bool igemm_plan_writes_packed(const IgemmPlan* p) { return p->nacc != -2 && p->terms != 3; }
 int igemm_plan_splits(const IgemmPlan* p) { return p->splits; }
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->partial_bytes; }
 
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
     const char* view = p->s2d ? "s2d " : "";
+    if (p->nacc == -2) {
+        std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=1 grid=%dx%dx1", p->BN, p->tile_id,
+                      p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES, p->tiles_m, p->tiles_n);
+        return;
+    }
     if (p->nacc < 0) {
         const int tiles = p->tiles_m * p->tiles_n;
         std::snprintf(buf, n, "tile=gconv_128x%d(id %d) stages=%d split_k=1 grid=%dx1x1 tiles=%d", p->BN, p->tile_id,
@@ -1183,7 +1277,7 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const ConvDims& d = p->d;
     const long long total = (long long)d.R * d.S * d.K * p->Cp;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
-    if (p->nacc < 0) {
+    if (p->nacc == -1) {
         const int Kp = p->gather_chunks * 32;
         const int gblocks = (int)std::min<long long>(((long long)d.K * Kp + 255) / 256, 148 * 8);
         BODA_CUDA_TRY(launch_kernel(pack_filters_flat_kernel, dim3(gblocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.Kred, Kp));
@@ -1236,6 +1330,7 @@ int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int 
 {
     if (in_packed && (p->s2d || p->nacc < 0)) return BODA_ERR_UNSUPPORTED;
     if ((in_packed || out_packed) && p->terms == 3) return BODA_ERR_UNSUPPORTED;
+    if (out_packed && p->nacc == -2) return BODA_ERR_UNSUPPORTED;        // that kernel's tiles follow images: NCHW output only
     if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < p->d.P || oWp < p->d.Q)) return BODA_ERR_INVALID_ARG;
     p->in_packed = in_packed != 0;
     p->out_packed = out_packed ? 1 : 0;
@@ -1255,6 +1350,26 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
+    }
+    if (p->nacc == -2) {
+        if (p->map_a_base != in) {
+            const int rc = encode_map_a_k1n(p, in);
+            if (rc != BODA_OK) return rc;
+        }
+        if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
+        k1n::K1nParams kp;
+        kp.HW = d.H * d.W; kp.tiles_per_image = (kp.HW + BM - 1) / BM;
+        kp.cchunks = p->Cp / BKC;
+        kp.bias = bias;
+        kp.o = make_out_spec(p, out);
+        kp.status = p->d_status;
+        kp.tx_extra = p->tx_extra;
+        switch (p->BN) {
+            case 64: return launch_k1n<64>(p, kp, stream);
+            case 128: return launch_k1n<128>(p, kp, stream);
+            case 192: return launch_k1n<192>(p, kp, stream);
+            default: return BODA_ERR_UNSUPPORTED;
+        }
     }
     if (p->nacc < 0) {
         if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));

@@ -259,3 +259,40 @@ def test_large_batch_k1conv_chooses_the_gather_kernel_and_small_batch_does_not()
         assert "gconv_128x192" in big.describe() and "gconv" not in small.describe()
     finally:
         big.close(); small.close()
+
+
+# ---- 1x1 layers by TMA straight from NCHW (tiles 20..22): the input tile is an MN-major tensor-core operand
+K1N_SHAPES = [
+    (2, 64, 14, 14, 48, 1, 1, 1, 0, 1),           # two tiles per image, the second ragged (196 = 128 + 68)
+    (5, 40, 6, 6, 200, 1, 1, 1, 0, 0),            # image smaller than a tile, C not a multiple of 32, K ragged against every tile
+    (3, 480, 14, 14, 192, 1, 1, 1, 0, 1),         # configuration 3's layer
+    (1, 32, 16, 24, 16, 1, 1, 1, 0, 1),           # exactly three tiles, one reduction step
+]
+
+
+@pytest.mark.parametrize("shape", K1N_SHAPES)
+@pytest.mark.parametrize("tile", [20, 21, 22])
+def test_k1conv_from_nchw_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 1800)
+    got, desc = run_planned(shape, x, w, b, variant=K1, tile_id=tile)
+    assert "k1nchw_128x" in desc and f"id {tile}" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_k1conv_from_nchw_on_real_values_is_the_choice_for_configuration_3_and_refuses_what_it_cannot_address():
+    from paper_1606_00094_b200 import binding as B
+    c = wl.CONFIGS[3]
+    x, w, b = c.tensors()
+    got, desc = run_planned(c.shape.as_tuple(), x, w, b)
+    assert "k1nchw" in desc           # one kernel, no staging: faster than staging + the tiled kernel at this size
+    # the input is used as it lies in memory: the tensor core truncates it to TF32 (no rounding pass), still inside the bar
+    assert_parity(got, oracle_out(c.shape.as_tuple(), x, w, b), TF32_TOL, desc)
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((2, 64, 7, 9, 32, 1, 1, 1, 0, 1), variant=K1, tile_id=20)          # rows of 63 floats: not a multiple of 16 bytes
+    with pytest.raises(B.BodaError):
+        B.ConvPlan((2, 64, 8, 8, 32, 1, 1, 2, 0, 1), variant=K1, tile_id=20)          # stride 2
+    auto = B.ConvPlan((2, 64, 7, 9, 32, 1, 1, 1, 0, 1), variant=K1)                   # automatic selection falls back to the staged path
+    try:
+        assert "k1nchw" not in auto.describe()
+    finally:
+        auto.close()
