@@ -46,3 +46,33 @@ def test_expired_wait_sets_status_and_context_survives(tile, split):
     assert B.boda_query_status() == 0
     plan.close()
     assert_parity(got, oracle_out(shape, x, w, b), TF32_TOL)
+
+
+def test_expired_wait_in_the_nchw_1x1_kernel():
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    shape = (3, 64, 12, 12, 200, 1, 1, 1, 0, 1)
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x = wl.half_normal(4, (N, C, H, W))
+    w = wl.normal(5, (K, C, R, S), 0, (2.0 / C) ** 0.5)
+    b = wl.normal(6, (K,), 0, 0.01)
+    dx, dw, db = (torch.from_numpy(t).cuda() for t in (x, w, b))
+    assert B.boda_query_status() == 0
+    os.environ["BODA_TEST_TX_MISMATCH"] = "1"
+    os.environ["BODA_WAIT_LIMIT_CYCLES"] = "100000000"
+    try:
+        plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20)
+    finally:
+        del os.environ["BODA_TEST_TX_MISMATCH"]
+        del os.environ["BODA_WAIT_LIMIT_CYCLES"]
+    plan(dx, dw, db)
+    torch.cuda.synchronize()
+    assert B.boda_query_status() == B.BODA_ERR_DEVICE_TIMEOUT
+    assert B.boda_query_status() == 0
+    plan.close()
+    plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20)
+    got = plan(dx, dw, db).cpu().numpy()
+    torch.cuda.synchronize()
+    assert B.boda_query_status() == 0
+    plan.close()
+    assert_parity(got, oracle_out(shape, x, w, b), TF32_TOL)
