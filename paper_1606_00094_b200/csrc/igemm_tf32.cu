@@ -547,52 +547,54 @@ pack_input_s2d_kernel(const float* __restrict__ in, float* __restrict__ xs, int 
 
 // The same for stride 4 with the channel count a compile-time constant (first layers: C = 3).  The general kernel above
 // spends most of its instructions on divisions by run-time extents and was bound by instruction issue (measured: 780
-// instructions per warp for 14.6 KB of output per CTA); here every index computation is a shift, a literal or a
-// multiplication by a constant, and each warp issues all of its staging loads - twelve coalesced 128-byte pieces - before
-// it stores the first one.
+// instructions per warp for 14.6 KB of output per CTA); here a warp stages one 32-column piece of all C*4 rows at a
+// time, so that the row index is a literal and the C*4 coalesced 128-byte loads of a piece are in flight together.
 template <int C>
 __global__ void __launch_bounds__(256)
 pack_input_s2d_t4_kernel(const float* __restrict__ in, float* __restrict__ xs, int H, int W, int pad, int Hb, int Wb)
 {
-    constexpr int T = 4, ROWS = C * T, CP = ((C * T * T + 31) / 32) * 32, QUADS = CP / 4, PER_PASS = 12;
+    constexpr int T = 4, ROWS = C * T, CP = ((C * T * T + 31) / 32) * 32, QUADS = CP / 4;
     static_assert(256 % QUADS == 0, "a block-row's 16-byte pieces are dealt to the threads without a remainder");
     extern __shared__ __align__(16) float sm_rows[];     // [ROWS][pitch]: element x of a row at [row*pitch + pad + x]
     pdl_launch_dependents();
     const int yb = blockIdx.x, n = blockIdx.y;
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int pitch = (Wb * T + 3) & ~3;
-    const int tasks = ROWS * ((pitch + 31) >> 5);          // task = piece * ROWS + row: one 32-column piece of one row
+    const int pieces = (pitch + 31) >> 5;                  // 32-column pieces of a staged row
     const float* img = in + (size_t)n * C * H * W;
     pdl_wait();
-    for (int t0 = warp; t0 < tasks; t0 += 8 * PER_PASS) {
-        float v[PER_PASS];
+    // A warp takes 32-column pieces warp, warp + 8, ... of ALL the rows: the row index is a literal, so (dy, c) and the
+    // row's offset cost nothing, and the ROWS loads of a piece are in flight together.
+    const int y_first = yb * T - pad;
+    for (int piece = warp; piece < pieces; piece += 8) {
+        const int i = piece * 32 + lane, x = i - pad;
+        const bool xin = i < pitch && (unsigned)x < (unsigned)W;
+        const float* src = img + (ptrdiff_t)y_first * W + x;
+        float v[ROWS];
 #pragma unroll
-        for (int u = 0; u < PER_PASS; ++u) {
-            const int task = t0 + 8 * u;
-            const int piece = task / ROWS, row = task - piece * ROWS;
-            const int dy = row / C, c = row - dy * C;
-            const int y = yb * T + dy - pad, x = piece * 32 + lane - pad;
-            v[u] = (task < tasks && (unsigned)y < (unsigned)H && (unsigned)x < (unsigned)W) ? __ldg(img + ((size_t)c * H + y) * W + x) : 0.f;
+        for (int row = 0; row < ROWS; ++row) {
+            const int dy = row / C, c = row - dy * C;      // literals after unrolling
+            const bool yin = (unsigned)(y_first + dy) < (unsigned)H;
+            v[row] = (xin && yin) ? __ldg(src + (c * H + dy) * W) : 0.f;      // one image's offsets fit 32 bits
         }
+        if (i < pitch) {
 #pragma unroll
-        for (int u = 0; u < PER_PASS; ++u) {
-            const int task = t0 + 8 * u;
-            const int piece = task / ROWS, row = task - piece * ROWS;
-            const int i = piece * 32 + lane;
-            if (task < tasks && i < pitch) sm_rows[row * pitch + i] = v[u];
+            for (int row = 0; row < ROWS; ++row) sm_rows[row * pitch + i] = v[row];
         }
     }
     __syncthreads();
     // 16-byte piece j of a block is row j = (dy, c) of the staged rows, four consecutive floats; pieces past ROWS are padding
     float* dst = xs + ((size_t)n * Hb + yb) * Wb * CP;
-    const int j = threadIdx.x % QUADS;
-    for (int xb = threadIdx.x / QUADS; xb < Wb; xb += 256 / QUADS) {
+    const int j = threadIdx.x % QUADS, xb0 = threadIdx.x / QUADS;
+    const float* srow = sm_rows + (j < ROWS ? j : 0) * pitch + 4 * xb0;
+    float* d4 = dst + xb0 * CP + 4 * j;
+    for (int xb = xb0; xb < Wb; xb += 256 / QUADS, srow += 4 * (256 / QUADS), d4 += (256 / QUADS) * CP) {
         float4 v = make_float4(0.f, 0.f, 0.f, 0.f);
         if (j < ROWS) {
-            const float4 r = *reinterpret_cast<const float4*>(sm_rows + j * pitch + 4 * xb);
+            const float4 r = *reinterpret_cast<const float4*>(srow);
             v = make_float4(round_tf32(r.x), round_tf32(r.y), round_tf32(r.z), round_tf32(r.w));
         }
-        *reinterpret_cast<float4*>(dst + (size_t)xb * CP + 4 * j) = v;
+        *reinterpret_cast<float4*>(d4) = v;
     }
 }
 
