@@ -78,6 +78,25 @@ cudaError_t launch_kernel(Kernel kernel, dim3 grid, dim3 block, size_t smem, cud
     return cudaLaunchKernelEx(&cfg, kernel, args...);
 }
 
+// cudaFuncSetAttribute applies to the current device only: a kernel's dynamic shared-memory limit is raised once per
+// device and kernel (one static DeviceSmemLimit per kernel instantiation), not once per process.
+struct DeviceSmemLimit {
+    int granted[64];
+    explicit DeviceSmemLimit(int initial = 0) { for (int& v : granted) v = initial; }
+    template <typename Kernel>
+    cudaError_t ensure(Kernel kernel, size_t bytes)
+    {
+        int dev = 0;
+        cudaError_t e = cudaGetDevice(&dev);
+        if (e != cudaSuccess) return e;
+        const bool tracked = dev >= 0 && dev < 64;
+        if (tracked && (int)bytes <= granted[dev]) return cudaSuccess;
+        e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)bytes);
+        if (e == cudaSuccess && tracked) granted[dev] = (int)bytes;
+        return e;
+    }
+};
+
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -302,11 +302,8 @@ int launch_pixel_sw(const ConvDims& d, const float* in, const float* filt, const
     int ih, iw, iwp;
     size_t smem;
     if (!pixel_geometry(d, KT, &ih, &iw, &iwp, &smem)) return BODA_ERR_UNSUPPORTED;
-    static size_t attr_smem = 48 * 1024;
-    if (smem > attr_smem) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(direct_pixel_kernel<KT, SW>, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-        attr_smem = smem;
-    }
+    static DeviceSmemLimit limit(48 * 1024);
+    BODA_CUDA_TRY(limit.ensure(direct_pixel_kernel<KT, SW>, smem));
     const int tiles_x = (d.Q + 31) / 32, tiles_y = (d.P + 7) / 8;
     dim3 grid(tiles_x * tiles_y, d.N, (d.K + KT - 1) / KT);
     if (grid.y > 65535 || grid.z > 65535) return BODA_ERR_UNSUPPORTED;

@@ -874,11 +874,8 @@ template <int BN>
 int launch_gather(IgemmPlan* p, const gconv::GconvParams& prm, cudaStream_t stream)
 {
     using C = gconv::Cfg<BN>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(gconv::gconv_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-        attr_set = true;
-    }
+    static DeviceSmemLimit limit;
+    BODA_CUDA_TRY(limit.ensure(gconv::gconv_tf32_kernel<BN>, C::SMEM_BYTES));
     const int grid = std::min(prm.tiles_total, p->sm_count);
     BODA_CUDA_TRY(launch_kernel(gconv::gconv_tf32_kernel<BN>, dim3(grid), dim3(gconv::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
                                 p->map_b, prm));
@@ -931,11 +928,8 @@ template <int BN>
 int launch_k1n(IgemmPlan* p, const k1n::K1nParams& prm, cudaStream_t stream)
 {
     using C = k1n::Cfg<BN>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(k1n::k1nchw_tf32_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize, C::SMEM_BYTES));
-        attr_set = true;
-    }
+    static DeviceSmemLimit limit;
+    BODA_CUDA_TRY(limit.ensure(k1n::k1nchw_tf32_kernel<BN>, C::SMEM_BYTES));
     dim3 grid(p->tiles_m, p->tiles_n);
     BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
                                 p->map_a, p->map_b, prm));
@@ -947,11 +941,8 @@ template <int BN, int NACC>
 int launch_halo(IgemmPlan* p, const halo::HaloParams& prm, cudaStream_t stream)
 {
     const int smem = halo::kASlots * p->a_slot_bytes + p->b_stages * BN * 128 + 1024 + 256;
-    static int attr_smem = 0;
-    if (smem > attr_smem) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(halo::tconv_halo_kernel<BN, NACC>, cudaFuncAttributeMaxDynamicSharedMemorySize, smem));
-        attr_smem = smem;
-    }
+    static DeviceSmemLimit limit;
+    BODA_CUDA_TRY(limit.ensure(halo::tconv_halo_kernel<BN, NACC>, (size_t)smem));
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
     BODA_CUDA_TRY(launch_kernel(halo::tconv_halo_kernel<BN, NACC>, grid, dim3(halo::kThreads), (size_t)smem, stream, p->splits,
                                 p->map_a, p->map_b, prm));
@@ -982,11 +973,8 @@ template <int BN, bool X3>
 int launch_bn_mode(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 {
     using Cfg = TileCfg<BN>;
-    static bool attr_set = false;
-    if (!attr_set) {
-        BODA_CUDA_TRY(cudaFuncSetAttribute(igemm_tf32_kernel<BN, X3>, cudaFuncAttributeMaxDynamicSharedMemorySize, Cfg::SMEM_BYTES));
-        attr_set = true;
-    }
+    static DeviceSmemLimit limit;
+    BODA_CUDA_TRY(limit.ensure(igemm_tf32_kernel<BN, X3>, Cfg::SMEM_BYTES));
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
     BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN, X3>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
                                 p->map_a, p->map_b, prm));

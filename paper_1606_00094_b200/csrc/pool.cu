@@ -213,11 +213,8 @@ int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int 
     if (G < 1) G = 1;
     const size_t smem = (size_t)G * H * W * sizeof(float);
     if (smem <= 96 * 1024) {
-        static size_t attr_smem = 48 * 1024;
-        if (smem > attr_smem) {
-            BODA_CUDA_TRY(cudaFuncSetAttribute(maxpool_plane_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, (int)smem));
-            attr_smem = smem;
-        }
+        static DeviceSmemLimit limit(48 * 1024);
+        BODA_CUDA_TRY(limit.ensure(maxpool_plane_kernel, smem));
         const int blocks = (NC + G - 1) / G;
         BODA_CUDA_TRY(launch_kernel(maxpool_plane_kernel, dim3(blocks), dim3(256), smem, stream, 1, in, out, NC, H, W, P, Q, ksz, stride, G));
     } else {
