@@ -898,9 +898,9 @@ bool k1n_legal(const ConvDims& d, int variant, bool x3)
 double model_cost_k1n(const ConvDims& d, int BN, int sm_count)
 {
     const long long tiles = (long long)d.N * ((d.H * d.W + BM - 1) / BM) * ((d.K + BN - 1) / BN);
-    const double waves = (double)((tiles + sm_count - 1) / sm_count);
+    const double per_cta = (double)((tiles + sm_count - 1) / sm_count);       // persistent: epilogues hide under the next tile
     const int steps = (d.C + BKC - 1) / BKC;
-    return waves * (steps * std::max(2.0 * BN, 380.0) + 3500.0 + 32.0 * BN);
+    return per_cta * steps * std::max(2.0 * BN, 410.0) + 3500.0 + 32.0 * BN;
 }
 
 int encode_map_a_k1n(IgemmPlan* p, const void* in)
@@ -930,7 +930,7 @@ int launch_k1n(IgemmPlan* p, const k1n::K1nParams& prm, cudaStream_t stream)
     using C = k1n::Cfg<BN>;
     static DeviceSmemLimit limit;
     BODA_CUDA_TRY(limit.ensure(k1n::k1nchw_tf32_kernel<BN>, C::SMEM_BYTES));
-    dim3 grid(p->tiles_m, p->tiles_n);
+    dim3 grid(std::min(prm.tiles_total, p->sm_count));
     BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
                                 p->map_a, p->map_b, prm));
     count_launch();
@@ -1221,8 +1221,9 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
     const char* view = p->s2d ? "s2d " : "";
     if (p->nacc == -2) {
-        std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=1 grid=%dx%dx1", p->BN, p->tile_id,
-                      p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES, p->tiles_m, p->tiles_n);
+        std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=1 grid=%dx1x1 tiles=%d", p->BN, p->tile_id,
+                      p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES,
+                      std::min(p->tiles_m * p->tiles_n, p->sm_count), p->tiles_m * p->tiles_n);
         return;
     }
     if (p->nacc < 0) {
@@ -1350,6 +1351,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         k1n::K1nParams kp;
         kp.HW = d.H * d.W; kp.tiles_per_image = (kp.HW + BM - 1) / BM;
         kp.cchunks = p->Cp / BKC;
+        kp.tiles_n = p->tiles_n; kp.tiles_total = p->tiles_m * p->tiles_n;
         kp.bias = bias;
         kp.o = make_out_spec(p, out);
         kp.status = p->d_status;

@@ -251,14 +251,17 @@ def test_gather_tiles_run_k1conv_exact(shape, tile):
     np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
 
 
-def test_large_batch_k1conv_chooses_the_gather_kernel_and_small_batch_does_not():
+def test_1x1_layers_avoid_the_staged_copy_at_every_batch():
+    # rows TMA can address (H*W a multiple of 4): the NCHW kernel; otherwise the gather kernel once the batch is large
     from paper_1606_00094_b200 import binding as B
     big = B.ConvPlan((256, 480, 14, 14, 192, 1, 1, 1, 0, 1))
     small = B.ConvPlan((5, 480, 14, 14, 192, 1, 1, 1, 0, 1))
+    odd = B.ConvPlan((256, 480, 13, 13, 192, 1, 1, 1, 0, 1))
     try:
-        assert "gconv_128x192" in big.describe() and "gconv" not in small.describe()
+        assert "k1nchw_128x192" in big.describe() and "k1nchw" in small.describe()
+        assert "gconv" in odd.describe()
     finally:
-        big.close(); small.close()
+        big.close(); small.close(); odd.close()
 
 
 # ---- 1x1 layers by TMA straight from NCHW (tiles 20..22): the input tile is an MN-major tensor-core operand
