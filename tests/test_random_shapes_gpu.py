@@ -83,3 +83,35 @@ def test_random_shape_forced_tiles_splits_and_views(idx):
         assert_parity(got, ref, TF32_TOL, f"{shape} {desc}")
         ran += 1
     assert ran >= 1
+
+
+# the degenerate corners, by hand: one element of everything, one-pixel outputs, windows as large as the image, strides
+# larger than the window, rows and columns of one pixel, padding that makes the border outputs pure bias
+DEGENERATE = [
+    (1, 1, 1, 1, 1, 1, 1, 1, 0, 0),
+    (1, 1, 3, 3, 1, 3, 3, 1, 0, 1),
+    (2, 5, 4, 4, 3, 2, 2, 3, 0, 0),
+    (1, 2, 1, 9, 4, 1, 3, 1, 1, 1),
+    (1, 2, 9, 1, 4, 3, 1, 2, 1, 0),
+    (3, 7, 5, 5, 2, 5, 5, 1, 2, 1),
+    (1, 4, 2, 2, 5, 1, 1, 1, 3, 0),
+    (4, 1, 8, 8, 1, 1, 1, 8, 0, 1),
+]
+
+
+@pytest.mark.parametrize("shape", DEGENERATE)
+def test_degenerate_shapes_exact_on_integers(shape):
+    from paper_1606_00094_b200 import binding as B
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x, w, b = wl.integers(8100, (N, C, H, W)), wl.integers(8101, (K, C, R, S)), wl.integers(8102, (K,))
+    ref = oracle_out(shape, x, w, b)
+    ran = 0
+    for variant, math in ((-1, 0), (DIRECT, 1), (K1, 2), (TC, 2), (-1, 3)):
+        try:
+            got, desc = run_planned(shape, x, w, b, variant=variant, math=math)
+        except B.BodaError as e:
+            assert e.status == B.BODA_ERR_UNSUPPORTED, f"{shape} variant {variant} math {math}: {e}"
+            continue
+        np.testing.assert_array_equal(got.astype(np.float64), ref, err_msg=f"{shape} {desc}")
+        ran += 1
+    assert ran >= 2
