@@ -78,7 +78,16 @@ typedef struct boda_plan_opts {
                                     left automatic, of the alternative variant too (FP32 kernel against tensor-core
                                     kernel, a strided TCONV layer with and without its space-to-depth view) */
     int variant;                 /* BODA_VARIANT_AUTO or a forced variant (used by tests) */
-    int tile_id;                 /* -1: automatic; otherwise index into the variant's tile table */
+    int tile_id;                 /* -1: automatic; otherwise index into the variant's tile table (boda_conv_plan_describe
+                                    prints the name).  BODA_VARIANT_DIRECT: 0..8 GEMM-blocked FP32 tiles direct_128x128 ..
+                                    direct_32x16, 9..11 pixel-per-thread direct_pixel_k8/16/32, 12..15 the same compiled
+                                    at run time for the exact shape direct_rtc_k4/8/16/32.  K1CONV / TCONV (pixels x
+                                    channels): 0..4 igemm_128x64/96/128/192/256 (TMA im2col tiles, cluster split),
+                                    5..15 halo_128/256/512xBN (TCONV stride 1 or space-to-depth view: shared-memory
+                                    reuse of the input across taps), 16..19 gconv_128x64/96/128/192 (input gathered
+                                    from NCHW, nothing staged; short reductions and 1x1), 20..22 k1nchw_128x64/128/192
+                                    (K1CONV by TMA straight from NCHW).  A tile that cannot run the shape is refused
+                                    with BODA_ERR_UNSUPPORTED. */
     int split_k;                 /* 0: automatic; otherwise the number of reduction splits of a tensor-core variant */
     int device;                  /* CUDA device ordinal; -1: the current device */
     int s2d;                     /* strided TCONV layers: -1 automatic, 0 never, 1 always run the stride-1
