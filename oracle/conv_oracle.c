@@ -29,6 +29,7 @@
  * paper, hand-computed cases, closed forms, identities, brute-force im2col and library
  * cross-checks).  Nothing here is "parity unpinned".
  */
+#include <math.h>
 #include <stddef.h>
 
 /* Output extent of one spatial dimension (Section 2: out_X = 1 + (in_X - KSZ)/stride, applied to
@@ -149,6 +150,27 @@ int oracle_sgemm_f64(const double* A, const double* B, double* C, int M, int N, 
             for (int k = 0; k < K; ++k) acc += A[(size_t)i * K + k] * B[(size_t)k * N + j];
             C[(size_t)i * N + j] = acc;
         }
+    return 0;
+}
+
+/*
+ * Softmax over the last dimension (Section 2 lists it with convolution and pooling as the operations deployment
+ * needs; the paper does not analyse it): out[r][j] = exp(in[r][j]) / sum over i of exp(in[r][i]).
+ * The definition written out in fp64; the row maximum is subtracted first, which changes no quotient and keeps exp
+ * inside its range.  Returns 0 on success, 1 on invalid arguments.
+ */
+int oracle_softmax_f64(const double* in, double* out, int rows, int cols)
+{
+    if (!in || !out || rows <= 0 || cols <= 0) return 1;
+    for (int r = 0; r < rows; ++r) {
+        const double* x = in + (size_t)r * cols;
+        double* y = out + (size_t)r * cols;
+        double mx = x[0];
+        for (int j = 1; j < cols; ++j) if (x[j] > mx) mx = x[j];
+        double sum = 0.0;
+        for (int j = 0; j < cols; ++j) { y[j] = exp(x[j] - mx); sum += y[j]; }
+        for (int j = 0; j < cols; ++j) y[j] /= sum;
+    }
     return 0;
 }
 

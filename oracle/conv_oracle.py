@@ -29,7 +29,7 @@ def build(force: bool = False) -> str:
         if force or stale:
             tmp = _LIB + f".tmp{os.getpid()}"
             cmd = ["gcc", "-O2", "-fopenmp", "-fPIC", "-shared", "-std=c11", "-Wall", "-Wextra",
-                   "-ffp-contract=off", "-o", tmp, _SRC]
+                   "-ffp-contract=off", "-o", tmp, _SRC, "-lm"]
             subprocess.run(cmd, check=True)
             os.replace(tmp, _LIB)
     return _LIB
@@ -56,6 +56,8 @@ def _load():
         lib.oracle_sgemm_ai.restype = ctypes.c_double
         lib.oracle_sgemm_f64.argtypes = [dp, dp, dp, i, i, i]
         lib.oracle_sgemm_f64.restype = i
+        lib.oracle_softmax_f64.argtypes = [dp, dp, i, i]
+        lib.oracle_softmax_f64.restype = i
         lib.oracle_num_threads.argtypes = []
         lib.oracle_num_threads.restype = i
         _lib = lib
@@ -144,6 +146,18 @@ def sgemm(A, Bm) -> np.ndarray:
     if rc != 0:
         raise ValueError("oracle_sgemm_f64: invalid arguments")
     return c
+
+
+def softmax(x) -> np.ndarray:
+    """Softmax over the last dimension of a 2-D array [rows][cols] by the definition (Section 2 names the operation), fp64."""
+    a = _f64(x)
+    if a.ndim != 2:
+        raise ValueError("softmax: expected [rows][cols]")
+    out = np.empty_like(a)
+    rc = _load().oracle_softmax_f64(_ptr(a), _ptr(out), a.shape[0], a.shape[1])
+    if rc != 0:
+        raise ValueError("oracle_softmax_f64: invalid arguments")
+    return out
 
 
 def num_threads() -> int:

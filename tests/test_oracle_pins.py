@@ -364,3 +364,28 @@ def test_sgemm_against_library_matmul():
     Bm = wl.normal(95, (17, 29))
     ref = A.astype(np.float64) @ Bm.astype(np.float64)
     np.testing.assert_allclose(orc.sgemm(A, Bm), ref, rtol=1e-13, atol=1e-13)
+
+
+# ---- softmax (Section 2 names it among the deployment operations): pins of oracle_softmax_f64
+def test_softmax_closed_forms():
+    # equal logits -> uniform; [0, ln 3] -> [1/4, 3/4]; [ln 1, ln 2, ln 5] -> [1/8, 2/8, 5/8]
+    np.testing.assert_allclose(orc.softmax(np.full((2, 7), 3.25)), np.full((2, 7), 1.0 / 7.0), rtol=1e-15)
+    np.testing.assert_allclose(orc.softmax(np.array([[0.0, np.log(3.0)]])), [[0.25, 0.75]], rtol=1e-15)
+    np.testing.assert_allclose(orc.softmax(np.log(np.array([[1.0, 2.0, 5.0]]))), [[0.125, 0.25, 0.625]], rtol=1e-15)
+    # one column: always 1; rows are independent
+    np.testing.assert_array_equal(orc.softmax(np.array([[-4.0], [900.0]])), [[1.0], [1.0]])
+
+
+def test_softmax_invariants_and_library_cross_check():
+    from scipy.special import softmax as sp_softmax
+    x = wl.normal(9100, (13, 1000), 0.0, 4.0).astype(np.float64)
+    y = orc.softmax(x)
+    np.testing.assert_allclose(y.sum(axis=1), 1.0, rtol=1e-14)
+    assert (y > 0).all() and (np.argmax(y, axis=1) == np.argmax(x, axis=1)).all()
+    np.testing.assert_allclose(orc.softmax(x + 123.5), y, rtol=1e-12)                  # shift invariance
+    np.testing.assert_allclose(y[:, 1:] / y[:, :-1], np.exp(x[:, 1:] - x[:, :-1]), rtol=1e-12)   # ratios are exp of differences
+    np.testing.assert_allclose(y, sp_softmax(x, axis=1), rtol=1e-13)
+    # logits far beyond exp's range in fp64 still give the limit distribution
+    np.testing.assert_allclose(orc.softmax(np.array([[1000.0, 1000.0, -1000.0]])), [[0.5, 0.5, 0.0]], atol=1e-300)
+    with pytest.raises(ValueError):
+        orc.softmax(np.zeros((3,)))
