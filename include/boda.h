@@ -248,6 +248,15 @@ int boda_maxpool_fwd(const float* in, float* out, int N, int C, int H, int W, in
                      void* stream);
 
 /*
+ * Softmax over the last dimension, out[r][j] = exp(in[r][j]) / sum over i of exp(in[r][i]) (the third operation
+ * Section 2 of the paper lists for deployment, beside convolution and pooling; it follows the classifier at the end
+ * of a network).  in, out: [rows][cols] row-major fp32 DEVICE pointers, may be the same buffer; fp32 arithmetic with
+ * the row maximum subtracted before exp.  Enqueues one kernel on `stream`; no allocation, no synchronisation.
+ * Errors: BODA_ERR_INVALID_ARG (NULL pointer, non-positive extent), BODA_ERR_CUDA.
+ */
+int boda_softmax_fwd(const float* in, float* out, int rows, int cols, void* stream);
+
+/*
  * A chain of layers run as one unit: convolutions (each followed by its bias and ReLU) and max-pools, layer
  * i+1 reading layer i's output - the shape of a CNN's convolutional trunk such as the AlexNet-shaped stack the
  * benchmark uses.  (The paper's framework runs a whole compute graph, Section 4 and Figure "Boda flow"; this is

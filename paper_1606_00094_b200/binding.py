@@ -78,6 +78,8 @@ _lib.boda_conv_fwd_noalloc.argtypes = [_vp] * 4 + [_i] * 10 + [_vp]
 _lib.boda_conv_fwd_noalloc.restype = _i
 _lib.boda_maxpool_fwd.argtypes = [_vp, _vp] + [_i] * 6 + [_vp]
 _lib.boda_maxpool_fwd.restype = _i
+_lib.boda_softmax_fwd.argtypes = [_vp, _vp, _i, _i, _vp]
+_lib.boda_softmax_fwd.restype = _i
 _lib.boda_conv_plan_kernels_per_call.argtypes = [_vp]
 _lib.boda_conv_plan_kernels_per_call.restype = _i
 _lib.boda_stack_create.argtypes = [ctypes.POINTER(boda_stack_op), _i, ctypes.POINTER(boda_plan_opts), ctypes.POINTER(_vp)]
@@ -248,6 +250,11 @@ def boda_sgemm(A, Bm, C, M, N, K, stream=None) -> None:
 
 def boda_maxpool_fwd(inp, out, N, C, H, W, ksz=3, stride=2, stream=None) -> None:
     _check(_lib.boda_maxpool_fwd(_addr(inp), _addr(out), N, C, H, W, ksz, stride, _stream(stream)), "boda_maxpool_fwd")
+
+
+def boda_softmax_fwd(inp, out, rows, cols, stream=None) -> None:
+    """out[r][:] = softmax(inp[r][:]) for [rows][cols] fp32 device tensors."""
+    _check(_lib.boda_softmax_fwd(_addr(inp), _addr(out), rows, cols, _stream(stream)), "boda_softmax_fwd")
 
 
 def boda_conv_plan_kernels_per_call(plan: int) -> int:

@@ -598,6 +598,12 @@ int boda_maxpool_fwd(const float* in, float* out, int N, int C, int H, int W, in
     return maxpool_launch(in, out, N, C, H, W, ksz, stride, (cudaStream_t)stream);
 }
 
+int boda_softmax_fwd(const float* in, float* out, int rows, int cols, void* stream)
+{
+    if (!in || !out || rows <= 0 || cols <= 0) return BODA_ERR_INVALID_ARG;
+    return softmax_launch(in, out, rows, cols, (cudaStream_t)stream);
+}
+
 int boda_query_status(void* stream, int* device_status)
 {
     if (!device_status) return BODA_ERR_INVALID_ARG;

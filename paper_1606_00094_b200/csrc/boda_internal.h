@@ -149,6 +149,9 @@ int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int 
 // the same on the staged layout rows [(n*Hp + y)*Wp + x][Cp]; output staged (out_packed) or NCHW
 int maxpool_packed_launch(const float* in, float* out, int N, int C, int H, int W, int iHp, int iWp, int iCp, int ksz, int stride,
                           int out_packed, int oHp, int oWp, int oCp, cudaStream_t stream);
+// ---- softmax over the last dimension of [rows][cols]
+int softmax_launch(const float* in, float* out, int rows, int cols, cudaStream_t stream);
+
 int unpack_to_nchw_launch(const float* in, float* out, int N, int C, int H, int W, int Hp, int Wp, int Cp, cudaStream_t stream);
 
 }  // namespace boda
