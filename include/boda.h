@@ -140,7 +140,9 @@ int boda_conv_plan_kernels_per_call(const boda_conv_plan* plan);
  * tensor-core plan, so that boda_conv_fwd_planned can skip the per-call filter re-layout.  Weights
  * are constants at deployment time (Section 2 speaks of deployment / inference).  After binding,
  * the `filt` argument of boda_conv_fwd_planned is ignored when it equals the bound pointer; passing
- * a different pointer re-packs on that call.  Enqueues on `stream`.
+ * a different pointer re-packs on that call.  Runs the re-layout on `stream` and waits for it (a set-up call,
+ * not for the hot path): later launches may then fetch the packed filters without waiting for their predecessor
+ * in the stream.  `filt` must stay unchanged while bound.
  */
 int boda_conv_plan_bind_filters(boda_conv_plan* plan, const float* filt, void* stream);
 

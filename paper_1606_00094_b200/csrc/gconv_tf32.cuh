@@ -44,6 +44,7 @@ struct GconvParams {
     OutSpec o;
     int* status;
     int tx_extra;                // test hook: bytes added to the expected size of the first filter tile of CTA 0
+    int b_early;                 // bound filters: the filter tiles' loads need not wait for the preceding kernel
 };
 
 template <int BN> struct Cfg {
@@ -105,7 +106,7 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_acc = s_tmem_base;
-    pdl_wait();
+    if (!(p.b_early && warp == 0)) pdl_wait();
 
     if (warp == 0) {
         if (lane == 0) {

@@ -56,6 +56,7 @@ struct IgemmParams {
     OutSpec o;                   // output tensor, layout and activation
     int* status;
     int tx_extra;                // test hook: bytes added to the first stage's expected transfer size of CTA (0,0,0)
+    int b_early;                 // the staged filters were written long before this launch (bound filters): their loads need not wait for the preceding kernel
 };
 
 
@@ -142,7 +143,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_acc = s_tmem_base;
-    pdl_wait();          // everything above overlapped the previous kernel; its results are needed from here on
+    // Everything above overlapped the previous kernel; its results (the input) are needed from here on.  The filter
+    // tiles are not its results: with bound filters their producer and the byte counts start at once, so the first
+    // filter tiles (HBM-cold after a long pause) are on their way while the input is still being written.
+    if (!(p.b_early && (warp == 11 || warp == 12))) pdl_wait();
 
     if (warp == 0 || warp >= 11) {
         if (lane == 0) {
@@ -1291,8 +1295,12 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
 int igemm_bind_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
 {
     int rc = pack_filters(p, filt, stream);
-    if (rc == BODA_OK) p->bound_filt = filt;
-    return rc;
+    if (rc != BODA_OK) return rc;
+    // The kernels fetch bound filters without waiting for the preceding kernel in their stream (they are constants
+    // by then): make sure the packing is not that predecessor.
+    BODA_CUDA_TRY(cudaStreamSynchronize(stream));
+    p->bound_filt = filt;
+    return BODA_OK;
 }
 
 void igemm_unbind_filters(IgemmPlan* p) { p->bound_filt = nullptr; }
@@ -1356,6 +1364,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         kp.o = make_out_spec(p, out);
         kp.status = p->d_status;
         kp.tx_extra = p->tx_extra;
+        kp.b_early = (filt == p->bound_filt) ? 1 : 0;
         switch (p->BN) {
             case 64: return launch_k1n<64>(p, kp, stream);
             case 128: return launch_k1n<128>(p, kp, stream);
@@ -1373,6 +1382,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         gp.o = make_out_spec(p, out);
         gp.status = p->d_status;
         gp.tx_extra = p->tx_extra;
+        gp.b_early = (filt == p->bound_filt) ? 1 : 0;
         switch (p->BN) {
             case 64: return launch_gather<64>(p, gp, stream);
             case 96: return launch_gather<96>(p, gp, stream);
@@ -1449,6 +1459,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     prm.bias = bias;
     prm.o = make_out_spec(p, out);
     prm.tx_extra = p->tx_extra;
+    prm.b_early = (filt == p->bound_filt) ? 1 : 0;
     prm.status = p->d_status;
     switch (p->BN) {
         case 64: return launch_bn<64>(p, prm, stream);
@@ -1544,6 +1555,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     prm.splits = p->splits;
     prm.bias = bias;
     prm.o = make_out_spec(p, out);
+    prm.b_early = 0;
     prm.tx_extra = p->tx_extra;
     prm.status = p->d_status;
     switch (p->BN) {

@@ -39,6 +39,7 @@ struct K1nParams {
     OutSpec o;                   // NCHW only
     int* status;
     int tx_extra;                // test hook: bytes added to the expected size of the first stage of CTA (0, 0)
+    int b_early;                 // bound filters: the filter tiles' loads need not wait for the preceding kernel
 };
 
 template <int BN> struct Cfg {
@@ -116,7 +117,7 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     };
     int n, hw0, k0;
     decode(0, n, hw0, k0);
-    pdl_wait();
+    if (!(p.b_early && warp == 3)) pdl_wait();
 
     if (warp == 0 || warp == 2) {
         if (lane == 0) {
