@@ -309,8 +309,10 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
         // kernel against the tensor-core variant, and a strided tconv layer with and without its space-to-depth
         // view).  The fastest plan is kept and remembered in the file named by BODA_TUNE_CACHE (if set).
         char key[160];
-        std::snprintf(key, sizeof(key), "%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d", shape->N, shape->C, shape->H, shape->W,
-                      shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math);
+        // the leading number names the tile tables: entries written by a build with other tables are not matched
+        constexpr int kTileTableVersion = 3;
+        std::snprintf(key, sizeof(key), "t%d:%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d", kTileTableVersion, shape->N, shape->C,
+                      shape->H, shape->W, shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math);
         int c_tile = -1, c_split = 0, c_variant = variant, c_s2d = o.s2d;
         if (tune_cache_lookup(key, &c_tile, &c_split, &c_variant, &c_s2d)) {
             boda_plan_opts oc = o;
