@@ -270,7 +270,10 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
                 }
             }
             // the loads above are in flight while this waits for the stage to be free
-            if (!mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 25)) break;
+            // one poller per warp and a warp-wide decision: no lane is left behind at the __syncwarp below
+            int free_now = 0;
+            if (lane == 0) free_now = mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 25) ? 1 : 0;
+            if (!__shfl_sync(0xffffffffu, free_now, 0)) break;
             // 128-byte swizzle: 16-byte piece c of row `row` lives at piece c ^ (row & 7)
             const uint32_t a_row = smem_a + stage * A_STAGE_BYTES + (uint32_t)row * 128u;
 #pragma unroll
