@@ -425,13 +425,19 @@ def run_ours(args):
     for _ in range(2):
         stack.forward_host(x_pin, out_pin)
     barrier()
+    # The call is synchronous (it returns when the result has landed in out_host) and ordered on the stream, so the
+    # host clock around it - taken once the L2 flush has drained - must agree with the event pair on the stream.
     e2e_ev = []
+    e2e_host_s = 0.0
     for _ in range(args.steps):
         flush.zero_()
         e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        t0 = time.perf_counter()
         e0.record()
         stack.forward_host(x_pin, out_pin)
         e1.record()
+        e2e_host_s += time.perf_counter() - t0
         e2e_ev.append((e0, e1))
     barrier()
     clocks = sampler.stop()
@@ -486,7 +492,9 @@ def run_ours(args):
                        "parallelism": f"replicas{world}", "l2": "flushed between steps (512 MiB write)",
                        "flops_per_step": flops_step},
             "e2e": {"value": round(e2e_value, 1), "unit": UNIT, "h2d_bytes_per_step": int(x_np.nbytes),
-                    "d2h_bytes_per_step": int(np.prod(stack.out_shape)) * 4},
+                    "d2h_bytes_per_step": int(np.prod(stack.out_shape)) * 4,
+                    "ms_per_step_events": round(e2e_total_ms / args.steps, 5),
+                    "ms_per_step_host_clock_rank0": round(1e3 * e2e_host_s / args.steps, 5)},
             "gpu_launches": int(launches),
             "clocks": clocks,
             "roofline": roofline,

@@ -94,6 +94,10 @@ typedef struct boda_plan_opts {
                                     "space-to-depth" view (stride t on C channels = stride 1 on C*t*t channels
                                     with ceil(R/t) x ceil(S/t) taps); an input transformation in the sense of
                                     Section 5 of the paper */
+    size_t max_workspace;        /* 0: no limit; otherwise the largest boda_conv_plan_workspace_bytes the caller accepts:
+                                    tiles that need more are not considered (a layer may then run on a kernel that
+                                    stages nothing, or on the FP32 kernel); a forced variant or tile that needs more
+                                    is refused with BODA_ERR_NOMEM */
 } boda_plan_opts;
 
 typedef struct boda_conv_plan boda_conv_plan;   /* opaque; created and destroyed by the library */
@@ -277,6 +281,9 @@ typedef struct boda_stack boda_stack;
  * must be a convolution (it fixes the input extent).  Errors as boda_conv_plan_create, INVALID_ARG if shapes do
  * not chain. */
 int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts* opts, boda_stack** stack);
+/* The same with one set of plan options per op: `per_op_opts` points to n_ops entries (those of MAXPOOL ops are
+ * ignored); entry 0 also names the device.  For tests and experiments that force a tile or split per layer. */
+int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_opts* per_op_opts, boda_stack** stack);
 int boda_stack_destroy(boda_stack* stack);
 int boda_stack_num_ops(const boda_stack* stack);
 /* Device pointers to the filters [K][C][R][S] and bias [K] (or NULL) of convolution op `op_index`; the stack keeps
@@ -308,7 +315,9 @@ int boda_stack_fwd_eager(boda_stack* stack, const float* in, float* out, void* s
  * in place).  `in` is read only by op 0 and `out` written only by the last op; pass NULL otherwise. */
 int boda_stack_run_op(boda_stack* stack, int op_index, const float* in, float* out, void* stream);
 /* Forward pass with HOST buffers: copies `in_host` to the device, runs the chain, copies the result into
- * `out_host` and synchronises `stream`.  Pinned host memory makes the copies asynchronous.  Batch items are
+ * `out_host` and synchronises `stream`.  The call is ordered on `stream`: `in_host` is not read before the work
+ * queued on `stream` so far has finished (the copies run on a second stream that first waits for it).  On an
+ * error return no copy is still in flight.  Pinned host memory makes the copies asynchronous.  Batch items are
  * independent (Section 2 of the paper), so for even N >= 4 the batch is copied in two slices (BODA_STACK_HOST_CHUNKS=k: k slices) on a second
  * stream and each slice runs, as soon as it has arrived, through a stack of the same layers planned for the
  * sub-batch (created on the first call; same filters; BODA_STACK_HOST_CHUNKS=1 in the environment keeps the batch

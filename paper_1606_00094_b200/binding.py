@@ -44,7 +44,8 @@ BODA_STACK_CONV, BODA_STACK_MAXPOOL = 0, 1
 
 
 class boda_plan_opts(ctypes.Structure):
-    _fields_ = [(n, ctypes.c_int) for n in ("math", "tune", "variant", "tile_id", "split_k", "device", "s2d")]
+    _fields_ = [(n, ctypes.c_int) for n in ("math", "tune", "variant", "tile_id", "split_k", "device", "s2d")] + \
+               [("max_workspace", ctypes.c_size_t)]
 
 
 _vp = ctypes.c_void_p
@@ -84,6 +85,8 @@ _lib.boda_conv_plan_kernels_per_call.argtypes = [_vp]
 _lib.boda_conv_plan_kernels_per_call.restype = _i
 _lib.boda_stack_create.argtypes = [ctypes.POINTER(boda_stack_op), _i, ctypes.POINTER(boda_plan_opts), ctypes.POINTER(_vp)]
 _lib.boda_stack_create.restype = _i
+_lib.boda_stack_create_ex.argtypes = [ctypes.POINTER(boda_stack_op), _i, ctypes.POINTER(boda_plan_opts), ctypes.POINTER(_vp)]
+_lib.boda_stack_create_ex.restype = _i
 _lib.boda_stack_destroy.argtypes = [_vp]
 _lib.boda_stack_destroy.restype = _i
 _lib.boda_stack_num_ops.argtypes = [_vp]
@@ -270,6 +273,17 @@ def boda_stack_create(ops, opts: Optional[boda_plan_opts] = None) -> int:
     return handle.value
 
 
+def boda_stack_create_ex(ops, per_op_opts) -> int:
+    """ops: list of boda_stack_op; per_op_opts: one boda_plan_opts per op.  Returns the stack handle."""
+    if len(per_op_opts) != len(ops):
+        raise ValueError("one boda_plan_opts per op")
+    arr = (boda_stack_op * len(ops))(*ops)
+    oarr = (boda_plan_opts * len(ops))(*per_op_opts)
+    handle = _vp()
+    _check(_lib.boda_stack_create_ex(arr, len(ops), oarr, ctypes.byref(handle)), "boda_stack_create_ex")
+    return handle.value
+
+
 def boda_stack_destroy(stack: int) -> None:
     _check(_lib.boda_stack_destroy(stack), "boda_stack_destroy")
 
@@ -342,11 +356,13 @@ def boda_clear_caches() -> None:
 class ConvPlan:
     """Owns a plan handle and its workspace; ``plan(x, w, b)`` runs the layer into a new tensor."""
 
-    def __init__(self, shape, math=BODA_MATH_AUTO, variant=BODA_VARIANT_AUTO, tile_id=-1, split_k=0, tune=0, s2d=-1):
+    def __init__(self, shape, math=BODA_MATH_AUTO, variant=BODA_VARIANT_AUTO, tile_id=-1, split_k=0, tune=0, s2d=-1,
+                 max_workspace=0):
         import torch
         self.shape = tuple(int(v) for v in shape)
         o = boda_plan_opts_default()
         o.math, o.variant, o.tile_id, o.split_k, o.tune, o.s2d = math, variant, tile_id, split_k, tune, s2d
+        o.max_workspace = max_workspace
         self.handle = boda_conv_plan_create(self.shape, o)
         nbytes = boda_conv_plan_workspace_bytes(self.handle)
         self.workspace = torch.empty(max(nbytes, 1), dtype=torch.uint8, device="cuda") if nbytes else None

@@ -33,23 +33,51 @@ def is_stale() -> bool:
     if not os.path.exists(LIB_PATH):
         return True
     t = os.path.getmtime(LIB_PATH)
-    deps = sources() + glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) \
-        + glob.glob(os.path.join(_ROOT, "include", "*.h"))
+    deps = sources() + _headers()
     return any(os.path.getmtime(p) > t for p in deps)
 
 
+def _headers():
+    return glob.glob(os.path.join(CSRC, "*.h")) + glob.glob(os.path.join(CSRC, "*.cuh")) \
+        + glob.glob(os.path.join(_ROOT, "include", "*.h"))
+
+
 def build_library(force: bool = False, verbose: bool = False) -> str:
-    """Compile every ``csrc/*.cu`` into one shared library; returns its path."""
+    """Compile every ``csrc/*.cu`` into one shared library; returns its path.
+
+    Each source is compiled to an object under ``csrc/build/`` (in parallel, and only if it or a header changed),
+    then the objects are linked."""
     if not force and not is_stale():
         return LIB_PATH
-    tmp = LIB_PATH + f".tmp{os.getpid()}"
-    cmd = [_nvcc()] + NVCC_FLAGS + (["-Xptxas", "-v"] if verbose else []) + \
-          ["-I", CSRC, "-I", os.path.join(_ROOT, "include"), "-o", tmp] + sources()
-    res = subprocess.run(cmd, capture_output=True, text=True)
-    if res.returncode != 0:
-        raise RuntimeError("nvcc failed:\n" + res.stdout + res.stderr)
+    nvcc = _nvcc()
+    objdir = os.path.join(CSRC, "build")
+    os.makedirs(objdir, exist_ok=True)
+    hdr_time = max(os.path.getmtime(h) for h in _headers())
+    compile_flags = [f for f in NVCC_FLAGS if f != "-shared"]
+    jobs, objs = [], []
+    for src in sources():
+        obj = os.path.join(objdir, os.path.basename(src)[:-3] + ".o")
+        objs.append(obj)
+        if not force and os.path.exists(obj) and os.path.getmtime(obj) > max(os.path.getmtime(src), hdr_time):
+            continue
+        cmd = [nvcc] + compile_flags + (["-Xptxas", "-v"] if verbose else []) + \
+              ["-I", CSRC, "-I", os.path.join(_ROOT, "include"), "-c", "-o", obj, src]
+        jobs.append((src, subprocess.Popen(cmd, stdout=subprocess.PIPE, stderr=subprocess.STDOUT, text=True)))
+    log = []
+    failed = False
+    for src, proc in jobs:
+        out, _ = proc.communicate()
+        log.append(out)
+        if proc.returncode != 0:
+            failed = True
+    if failed:
+        raise RuntimeError("nvcc failed:\n" + "".join(log))
     if verbose:
-        print(res.stdout + res.stderr)
+        print("".join(log))
+    tmp = LIB_PATH + f".tmp{os.getpid()}"
+    res = subprocess.run([nvcc, "-shared", "-o", tmp] + objs, capture_output=True, text=True)
+    if res.returncode != 0:
+        raise RuntimeError("link failed:\n" + res.stdout + res.stderr)
     os.replace(tmp, LIB_PATH)
     return LIB_PATH
 

@@ -204,6 +204,7 @@ void boda_plan_opts_default(boda_plan_opts* o)
     o->split_k = 0;
     o->device = -1;
     o->s2d = -1;
+    o->max_workspace = 0;
 }
 
 int boda_conv_plan_destroy(boda_conv_plan* plan)
@@ -220,7 +221,7 @@ int boda_conv_plan_destroy(boda_conv_plan* plan)
     return BODA_OK;
 }
 
-static int plan_time_ms(boda_conv_plan* plan, float* ms_out);
+static int plan_time_ms(boda_conv_plan* plan, bool chain_in, bool chain_out, float* ms_out);
 
 static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, DeviceCtx* ctx, int variant,
                       int tile_id, int split_k, boda_conv_plan** out)
@@ -254,7 +255,8 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
         p->ws_bytes = 0;
     } else {
         p->math = o.math == BODA_MATH_TF32X3 ? BODA_MATH_TF32X3 : BODA_MATH_TF32;
-        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig, o.math == BODA_MATH_TF32X3);
+        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig, o.math == BODA_MATH_TF32X3,
+                               o.max_workspace);
         if (rc == BODA_OK) { p->tile_id = igemm_plan_tile(p->ig); p->ws_bytes = igemm_plan_workspace_bytes(p->ig); }
     }
     if (rc != BODA_OK) { boda_conv_plan_destroy(p); return rc; }
@@ -263,6 +265,17 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
 }
 
 int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* opts, boda_conv_plan** plan)
+{
+    return boda::conv_plan_create_chained(shape, opts, false, false, plan);
+}
+
+}  // extern "C"
+
+// chain_in / chain_out: the layer will run inside a chain, its input arriving in the plan's own staged layout and its
+// output leaving in a consumer's staged layout.  Only the tuner looks at them: it times every candidate the way it
+// will run (no staging kernel, bulk-copy epilogue) instead of stand-alone with NCHW on both sides.
+int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan_opts* opts, bool chain_in, bool chain_out,
+                                   boda_conv_plan** plan)
 {
     if (!shape || !plan) return BODA_ERR_INVALID_ARG;
     *plan = nullptr;
@@ -303,6 +316,10 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
 
     if (!o.tune || o.tile_id >= 0) {
         rc = plan_build(*shape, o, ctx, variant, o.tile_id, o.split_k, plan);
+        // the workspace limit ruled out every tensor-core tile: the FP32 kernel needs no workspace
+        if (rc == BODA_ERR_NOMEM && o.max_workspace > 0 && o.variant == BODA_VARIANT_AUTO && o.tile_id < 0 &&
+            (o.math == BODA_MATH_AUTO || o.math == BODA_MATH_TF32X3))
+            rc = plan_build(*shape, o, ctx, BODA_VARIANT_DIRECT, -1, 0, plan);
     } else {
         // Automated tuning: the rule above names a variant; timing confirms or overturns it.  Every tile and split
         // of that variant is timed and, when the caller left variant and math open, so is the alternative (the FP32
@@ -310,9 +327,10 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
         // view).  The fastest plan is kept and remembered in the file named by BODA_TUNE_CACHE (if set).
         char key[160];
         // the leading number names the tile tables: entries written by a build with other tables are not matched
-        constexpr int kTileTableVersion = 3;
-        std::snprintf(key, sizeof(key), "t%d:%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d", kTileTableVersion, shape->N, shape->C,
-                      shape->H, shape->W, shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math);
+        constexpr int kTileTableVersion = 4;
+        std::snprintf(key, sizeof(key), "t%d:%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d,io%d%d", kTileTableVersion, shape->N, shape->C,
+                      shape->H, shape->W, shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math,
+                      chain_in ? 1 : 0, chain_out ? 1 : 0);
         int c_tile = -1, c_split = 0, c_variant = variant, c_s2d = o.s2d;
         if (tune_cache_lookup(key, &c_tile, &c_split, &c_variant, &c_s2d)) {
             boda_plan_opts oc = o;
@@ -350,7 +368,7 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
                     boda_conv_plan* cand = nullptr;
                     if (plan_build(*shape, oc, ctx, c.variant, t, split, &cand) != BODA_OK) continue;
                     float ms = 0.f;
-                    if (plan_time_ms(cand, &ms) == BODA_OK && ms < best_ms) {
+                    if (plan_time_ms(cand, chain_in, chain_out, &ms) == BODA_OK && ms < best_ms) {
                         if (best) boda_conv_plan_destroy(best);
                         best = cand;
                         best_ms = ms;
@@ -371,6 +389,8 @@ int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* op
     (void)cudaSetDevice(prev);
     return rc;
 }
+
+extern "C" {
 
 int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
 {
@@ -414,11 +434,27 @@ int boda_conv_fwd_planned(boda_conv_plan* p, const float* in, const float* filt,
 
 }  // extern "C"
 
-// Times one plan on scratch buffers (used by the tuner).  Synchronises.
-static int plan_time_ms(boda_conv_plan* p, float* ms_out)
+// Times one plan on scratch buffers (used by the tuner).  Synchronises.  chain_in / chain_out: time the plan the
+// way a chain runs it - reading its own staged input layout (no staging kernel) and writing a staged output - where
+// the plan's kernel can; operands hold a small non-zero constant (all-zero operands draw less power than real ones).
+static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float* ms_out)
 {
     const ConvDims& d = p->d;
-    const size_t n_in = (size_t)d.N * d.C * d.H * d.W, n_f = (size_t)d.K * d.Kred, n_out = (size_t)d.M * d.K;
+    size_t n_in = (size_t)d.N * d.C * d.H * d.W, n_out = (size_t)d.M * d.K;
+    const size_t n_f = (size_t)d.K * d.Kred;
+    bool in_packed = false, out_packed = false;
+    const int oCp = ((d.K + 31) / 32) * 32;
+    if (p->ig) {
+        int Hp = 0, Wp = 0, Cp = 0;
+        in_packed = chain_in && igemm_plan_input_geometry(p->ig, &Hp, &Wp, &Cp);
+        out_packed = chain_out && igemm_plan_writes_packed(p->ig);
+        if (in_packed) n_in = (size_t)d.N * Hp * Wp * Cp;
+        if (out_packed) n_out = (size_t)d.N * d.P * d.Q * oCp;
+        if (in_packed || out_packed) {
+            const int rc_io = conv_plan_set_io(p, in_packed ? 1 : 0, out_packed ? 1 : 0, d.P, d.Q, oCp);
+            if (rc_io != BODA_OK) return rc_io;
+        }
+    }
     float *in = nullptr, *f = nullptr, *b = nullptr, *out = nullptr;
     void* ws = nullptr;
     int rc = BODA_OK;
@@ -431,12 +467,14 @@ static int plan_time_ms(boda_conv_plan* p, float* ms_out)
         if (stream) { cudaStreamSynchronize(stream); cudaStreamDestroy(stream); }
         if (in) cudaFree(in); if (f) cudaFree(f); if (b) cudaFree(b); if (out) cudaFree(out); if (ws) cudaFree(ws);
         if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1);
+        if (in_packed || out_packed) (void)conv_plan_set_io(p, 0, 0, 0, 0, 0);
     };
 #define TRY_T(x) do { cudaError_t _e = (x); if (_e != cudaSuccess) { rc = record_cuda_error(_e, #x); cleanup(); return rc; } } while (0)
     TRY_T(cudaMalloc(&in, n_in * 4)); TRY_T(cudaMalloc(&f, n_f * 4)); TRY_T(cudaMalloc(&b, d.K * 4));
     TRY_T(cudaMalloc(&out, n_out * 4));
-    if (p->ws_bytes) TRY_T(cudaMalloc(&ws, p->ws_bytes));
-    TRY_T(cudaMemset(in, 0, n_in * 4)); TRY_T(cudaMemset(f, 0, n_f * 4)); TRY_T(cudaMemset(b, 0, d.K * 4));
+    if (p->ws_bytes && !in_packed) TRY_T(cudaMalloc(&ws, p->ws_bytes));
+    // bytes 0x3c -> the float 0.0115 (exact in TF32 after truncation or rounding alike)
+    TRY_T(cudaMemset(in, 0x3c, n_in * 4)); TRY_T(cudaMemset(f, 0x3c, n_f * 4)); TRY_T(cudaMemset(b, 0, d.K * 4));
     TRY_T(cudaEventCreate(&e0)); TRY_T(cudaEventCreate(&e1));
     TRY_T(cudaStreamSynchronize(0));                    // the fills above ran on the default stream
     TRY_T(cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking));

@@ -137,6 +137,10 @@ void direct_rtc_describe(const DirectRtc* r, char* buf, size_t n);
 int conv_fwd_planned_ex(boda_conv_plan* plan, const float* in, const float* filt, const float* bias, float* out,
                         void* workspace, cudaStream_t stream, cudaEvent_t after_staging);
 void conv_plan_out_dims(const boda_conv_plan* plan, int* N, int* K, int* P, int* Q);
+// boda_conv_plan_create for a layer of a chain: with opts->tune the candidates are timed reading a staged input
+// (chain_in) and writing a staged output (chain_out), the way the chain will run them
+int conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan_opts* opts, bool chain_in, bool chain_out,
+                             boda_conv_plan** plan);
 // chained layers: the staged input layout a tensor-core plan reads (false: the plan reads NCHW only), and the
 // switch that makes it read that layout directly / write its output in a consumer's staged layout
 bool conv_plan_input_geometry(const boda_conv_plan* plan, int* Hp, int* Wp, int* Cp);

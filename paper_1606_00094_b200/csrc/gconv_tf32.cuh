@@ -274,6 +274,7 @@ gconv_tf32_kernel(const __grid_constant__ CUtensorMap map_b, const GconvParams p
             int free_now = 0;
             if (lane == 0) free_now = mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 25) ? 1 : 0;
             if (!__shfl_sync(0xffffffffu, free_now, 0)) break;
+            __syncwarp();     // orders the other lanes' stores below after lane 0's acquire of the empty barrier
             // 128-byte swizzle: 16-byte piece c of row `row` lives at piece c ^ (row & 7)
             const uint32_t a_row = smem_a + stage * A_STAGE_BYTES + (uint32_t)row * 128u;
 #pragma unroll

@@ -1049,7 +1049,8 @@ int encode_map_b(IgemmPlan* p)
 
 }  // namespace
 
-int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out, bool x3)
+int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out, bool x3,
+                      size_t max_ws)
 {
     if (!igemm_variant_legal(d_in, variant)) return BODA_ERR_UNSUPPORTED;
     // strided tconv layers may run as their stride-1 space-to-depth view
@@ -1118,6 +1119,11 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
             continue;
         }
         if (nacc > 0 && (x3 || variant != BODA_VARIANT_TCONV || !halo_geometry(d, kTileBN[t], nacc, nullptr))) continue;
+        if (max_ws > 0) {
+            // staged input of this tile's kernel (see xp_bytes below)
+            const size_t rows = nacc > 0 ? (size_t)d.N * (d.H + d.pad) * (d.W + d.pad) : (size_t)d.N * d.H * d.W;
+            if (((rows * p->Cs() * 4 + 1023) & ~(size_t)1023) > max_ws) continue;
+        }
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
             if (s > p->iters_total) continue;
@@ -1128,6 +1134,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
     }
+    if (best >= 1e300 && tile_id < 0) { delete p; return max_ws > 0 ? BODA_ERR_NOMEM : BODA_ERR_UNSUPPORTED; }
     if (split_k > 0) best_s = std::min(split_k, p->iters_total);
     if (tile_id >= 0) best_t = tile_id;
     p->tile_id = best_t;
@@ -1200,6 +1207,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     }
 
+    if (max_ws > 0 && p->xp_bytes > max_ws) { delete p; return BODA_ERR_NOMEM; }
     cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cs() * 4);
     if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
     rc = encode_map_b(p);
@@ -1506,17 +1514,13 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cp * 4) + 1023) & ~(size_t)1023;
     const size_t tiles_max = (size_t)p->tiles_m * (size_t)((d.K + 63) / 64);
     const size_t head_bytes = 256 + ((tiles_max * sizeof(int) + 255) & ~(size_t)255);
-    const size_t fixed = head_bytes + 1024 + wp_bytes + p->xp_bytes;
-    // tile and split by the cost model, among the choices whose partial sums still fit the region
+    if (head_bytes + 1024 + wp_bytes + p->xp_bytes > region_bytes) return BODA_ERR_TOO_LARGE;
+    // tile and split by the cost model (split partial sums stay in shared memory: every choice fits the region)
     double best = 1e300;
     int best_t = -1, best_s = 1;
     for (int t = 0; t < kFirstHaloTile; ++t)
         for (int s : kSplitCandidates) {
             if (s > p->iters_total) continue;
-            const int ips = (p->iters_total + s - 1) / s;
-            const int eff = (p->iters_total + ips - 1) / ips;
-            (void)eff;
-            if (fixed > region_bytes) continue;
             const double c = model_cost(d, p->Cp, kTileBN[t], s);
             if (c < best) { best = c; best_t = t; best_s = s; }
         }

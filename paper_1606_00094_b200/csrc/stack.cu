@@ -1,6 +1,7 @@
 // boda_stack: a chain of convolution and max-pool layers (layer i+1 reads layer i's output) run as one unit.
 // The stack owns the plans, the activations between layers, one workspace shared by all layers and a CUDA graph
 // of the whole chain, so that a forward pass is a single graph launch with no host work between kernels.
+#include <algorithm>
 #include <cstdio>
 #include <cstdlib>
 #include <cstring>
@@ -45,11 +46,11 @@ struct boda_stack {
     // host-buffer path: the batch is copied in `host_chunks` slices on a second stream, and each slice runs through a
     // stack for the sub-batch as soon as it has arrived, so that copies and kernels overlap
     std::vector<boda_stack_op> specs;       // what the stack was created from
-    boda_plan_opts opts{};
-    bool has_opts = false;
+    std::vector<boda_plan_opts> op_opts;    // per-op plan options (empty: defaults)
     boda_stack* sub = nullptr;
     int host_chunks = 0;                    // 0: not decided yet; 1: no slicing
     cudaStream_t copy_stream = nullptr;
+    cudaEvent_t entry_event = nullptr;      // recorded on the caller's stream at entry: the copy stream waits for it
     std::vector<cudaEvent_t> chunk_events;
 };
 
@@ -127,6 +128,7 @@ int boda_stack_destroy(boda_stack* s)
     drop_graph(s);
     if (s->sub) boda_stack_destroy(s->sub);
     for (cudaEvent_t ev : s->chunk_events) cudaEventDestroy(ev);
+    if (s->entry_event) cudaEventDestroy(s->entry_event);
     if (s->copy_stream) cudaStreamDestroy(s->copy_stream);
     if (s->capture_stream) cudaStreamDestroy(s->capture_stream);
     for (auto& op : s->ops) {
@@ -144,15 +146,23 @@ int boda_stack_destroy(boda_stack* s)
 int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts* opts, boda_stack** out)
 {
     if (!ops || n_ops <= 0 || !out) return BODA_ERR_INVALID_ARG;
+    if (!opts) return boda_stack_create_ex(ops, n_ops, nullptr, out);
+    std::vector<boda_plan_opts> per_op((size_t)n_ops, *opts);
+    return boda_stack_create_ex(ops, n_ops, per_op.data(), out);
+}
+
+int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_opts* per_op_opts, boda_stack** out)
+{
+    if (!ops || n_ops <= 0 || !out) return BODA_ERR_INVALID_ARG;
     *out = nullptr;
     if (ops[0].kind != BODA_STACK_CONV) return BODA_ERR_INVALID_ARG;     // the first op fixes the input dims
     boda_stack* s = new (std::nothrow) boda_stack();
     if (!s) return BODA_ERR_NOMEM;
-    int device = opts ? opts->device : -1;
+    int device = per_op_opts ? per_op_opts[0].device : -1;
     if (device < 0) { cudaError_t e = cudaGetDevice(&device); if (e != cudaSuccess) { delete s; return record_cuda_error(e, "cudaGetDevice"); } }
     s->device = device;
     s->specs.assign(ops, ops + n_ops);
-    if (opts) { s->opts = *opts; s->has_opts = true; }
+    if (per_op_opts) s->op_opts.assign(per_op_opts, per_op_opts + n_ops);
     int N = ops[0].conv.N, C = ops[0].conv.C, H = ops[0].conv.H, W = ops[0].conv.W;
     s->in_elems = (size_t)N * C * H * W;
     int rc = BODA_OK;
@@ -163,13 +173,16 @@ int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts*
         if (op.kind == BODA_STACK_CONV) {
             op.conv = ops[i].conv;
             if (op.conv.N != N || op.conv.C != C || op.conv.H != H || op.conv.W != W) { rc = BODA_ERR_INVALID_ARG; break; }
-            rc = boda_conv_plan_create(&op.conv, opts, &op.plan);
+            // first by rule; layers that ask for tuning are re-planned below, once the layouts around them are known
+            boda_plan_opts o;
+            boda_plan_opts_default(&o);
+            if (per_op_opts) o = per_op_opts[i];
+            o.tune = 0;
+            rc = boda_conv_plan_create(&op.conv, &o, &op.plan);
             if (rc != BODA_OK) break;
             int oN, oK, oP, oQ;
             conv_plan_out_dims(op.plan, &oN, &oK, &oP, &oQ);
             op.oC = oK; op.oH = oP; op.oW = oQ;
-            const size_t ws = boda_conv_plan_workspace_bytes(op.plan);
-            if (ws > s->ws_bytes) s->ws_bytes = ws;
         } else if (op.kind == BODA_STACK_MAXPOOL) {
             op.ksz = ops[i].ksz; op.stride = ops[i].stride;
             op.oC = C;
@@ -185,18 +198,40 @@ int boda_stack_create(const boda_stack_op* ops, int n_ops, const boda_plan_opts*
     // (a tensor-core convolution, or a pool whose own input is staged) and the consumer can read it (a tensor-core
     // convolution that is not a space-to-depth view, or a pool); NCHW otherwise.  The chain's input and output are NCHW.
     const bool chain_layouts = !std::getenv("BODA_STACK_NCHW");
-    for (int i = 0; rc == BODA_OK && i + 1 < (int)s->ops.size(); ++i) {
-        boda_stack::Op& prod = s->ops[i];
-        boda_stack::Op& cons = s->ops[i + 1];
-        const bool can_write = prod.kind == BODA_STACK_CONV ? conv_plan_can_write_packed(prod.plan) : prod.in_packed;
-        int Hp = cons.H, Wp = cons.W, Cp = ((cons.C + 31) / 32) * 32;
-        bool can_read = true;
-        if (cons.kind == BODA_STACK_CONV) can_read = conv_plan_input_geometry(cons.plan, &Hp, &Wp, &Cp);
-        if (chain_layouts && can_write && can_read) {
-            prod.out_packed = true; prod.oHp = Hp; prod.oWp = Wp; prod.oCp = Cp;
-            cons.in_packed = true; cons.iHp = Hp; cons.iWp = Wp; cons.iCp = Cp;
+    auto assign_layouts = [&]() {
+        for (auto& op : s->ops) { op.in_packed = op.out_packed = false; op.oHp = op.oWp = op.oCp = op.iHp = op.iWp = op.iCp = 0; }
+        for (int i = 0; i + 1 < (int)s->ops.size(); ++i) {
+            boda_stack::Op& prod = s->ops[i];
+            boda_stack::Op& cons = s->ops[i + 1];
+            const bool can_write = prod.kind == BODA_STACK_CONV ? conv_plan_can_write_packed(prod.plan) : prod.in_packed;
+            int Hp = cons.H, Wp = cons.W, Cp = ((cons.C + 31) / 32) * 32;
+            bool can_read = true;
+            if (cons.kind == BODA_STACK_CONV) can_read = conv_plan_input_geometry(cons.plan, &Hp, &Wp, &Cp);
+            if (chain_layouts && can_write && can_read) {
+                prod.out_packed = true; prod.oHp = Hp; prod.oWp = Wp; prod.oCp = Cp;
+                cons.in_packed = true; cons.iHp = Hp; cons.iWp = Wp; cons.iCp = Cp;
+            }
         }
+    };
+    if (rc == BODA_OK) assign_layouts();
+    // Tuning: every layer that asks for it is planned again, its candidates timed the way the chain will run them
+    // (staged input without a staging kernel, staged output through the bulk-copy epilogue) - not stand-alone with
+    // NCHW on both sides, which would rank the tiles of a different kernel configuration.  A tuned plan may read
+    // another staged layout than the rule's plan did, so the layouts are assigned once more afterwards.
+    bool retuned = false;
+    for (int i = 0; rc == BODA_OK && per_op_opts && i < (int)s->ops.size(); ++i) {
+        boda_stack::Op& op = s->ops[i];
+        if (op.kind != BODA_STACK_CONV || !per_op_opts[i].tune || per_op_opts[i].tile_id >= 0) continue;
+        boda_conv_plan* tuned = nullptr;
+        rc = conv_plan_create_chained(&op.conv, &per_op_opts[i], op.in_packed, op.out_packed, &tuned);
+        if (rc != BODA_OK) break;
+        boda_conv_plan_destroy(op.plan);
+        op.plan = tuned;
+        retuned = true;
     }
+    if (rc == BODA_OK && retuned) assign_layouts();
+    for (const auto& op : s->ops)
+        if (op.kind == BODA_STACK_CONV && op.plan && !op.in_packed) s->ws_bytes = std::max(s->ws_bytes, boda_conv_plan_workspace_bytes(op.plan));
     for (int i = 0; rc == BODA_OK && i < (int)s->ops.size(); ++i) {
         boda_stack::Op& op = s->ops[i];
         if (op.kind == BODA_STACK_CONV) {
@@ -329,9 +364,10 @@ static void prepare_host_slices(boda_stack* s)
     for (auto& op : specs)
         if (op.kind == BODA_STACK_CONV) op.conv.N = N / k;
     boda_stack* sub = nullptr;
-    if (boda_stack_create(specs.data(), (int)specs.size(), s->has_opts ? &s->opts : nullptr, &sub) != BODA_OK) return;
+    if (boda_stack_create_ex(specs.data(), (int)specs.size(), s->op_opts.empty() ? nullptr : s->op_opts.data(), &sub) != BODA_OK) return;
     sub->host_chunks = 1;
     bool ok = cudaStreamCreateWithFlags(&s->copy_stream, cudaStreamNonBlocking) == cudaSuccess;
+    ok = ok && cudaEventCreateWithFlags(&s->entry_event, cudaEventDisableTiming) == cudaSuccess;
     for (int i = 0; ok && i < k; ++i) {
         cudaEvent_t ev = nullptr;
         ok = cudaEventCreateWithFlags(&ev, cudaEventDisableTiming) == cudaSuccess;
@@ -362,18 +398,30 @@ int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, vo
         }
         const int k = s->host_chunks;
         const size_t in_chunk = s->in_elems / k, out_chunk = s->out_elems / k;
-        // the staging buffers are idle: every call of this function ends with a synchronisation of its stream
-        for (int i = 0; i < k; ++i) {
-            BODA_CUDA_TRY(cudaMemcpyAsync(s->staging_in + i * in_chunk, in_host + i * in_chunk, in_chunk * sizeof(float),
-                                          cudaMemcpyHostToDevice, s->copy_stream));
-            BODA_CUDA_TRY(cudaEventRecord(s->chunk_events[i], s->copy_stream));
+        // The call is ordered on `stream`: the slices are copied on a second stream, which first waits for everything
+        // the caller has queued on `stream` so far (a kernel or copy that fills in_host, for instance).
+        BODA_CUDA_TRY(cudaEventRecord(s->entry_event, st));
+        BODA_CUDA_TRY(cudaStreamWaitEvent(s->copy_stream, s->entry_event, 0));
+        // the staging buffers are idle: every return of this function leaves both streams drained
+        int rc = BODA_OK;
+        cudaError_t ce = cudaSuccess;
+        for (int i = 0; i < k && ce == cudaSuccess; ++i) {
+            ce = cudaMemcpyAsync(s->staging_in + i * in_chunk, in_host + i * in_chunk, in_chunk * sizeof(float),
+                                 cudaMemcpyHostToDevice, s->copy_stream);
+            if (ce == cudaSuccess) ce = cudaEventRecord(s->chunk_events[i], s->copy_stream);
         }
-        for (int i = 0; i < k; ++i) {
-            BODA_CUDA_TRY(cudaStreamWaitEvent(st, s->chunk_events[i], 0));
-            const int rc = boda_stack_fwd(s->sub, s->staging_in + i * in_chunk, s->staging_out + i * out_chunk, stream);
-            if (rc != BODA_OK) return rc;
+        for (int i = 0; i < k && ce == cudaSuccess && rc == BODA_OK; ++i) {
+            ce = cudaStreamWaitEvent(st, s->chunk_events[i], 0);
+            if (ce == cudaSuccess) rc = boda_stack_fwd(s->sub, s->staging_in + i * in_chunk, s->staging_out + i * out_chunk, stream);
         }
-        BODA_CUDA_TRY(cudaMemcpyAsync(out_host, s->staging_out, s->out_elems * sizeof(float), cudaMemcpyDeviceToHost, st));
+        if (ce == cudaSuccess && rc == BODA_OK)
+            ce = cudaMemcpyAsync(out_host, s->staging_out, s->out_elems * sizeof(float), cudaMemcpyDeviceToHost, st);
+        if (ce != cudaSuccess || rc != BODA_OK) {
+            // no copy may still be writing the staging buffer when the caller gets the error
+            (void)cudaStreamSynchronize(s->copy_stream);
+            (void)cudaStreamSynchronize(st);
+            return rc != BODA_OK ? rc : record_cuda_error(ce, "boda_stack_fwd_host (sliced copies)");
+        }
         BODA_CUDA_TRY(cudaStreamSynchronize(st));
         return BODA_OK;
     }

@@ -15,8 +15,9 @@ from .workloads import StackOp
 
 class ConvStack:
     def __init__(self, ops: Sequence[StackOp], params: Sequence[Tuple], math: int = B.BODA_MATH_AUTO,
-                 tune: int = 0, device: str = "cuda"):
-        """ops: conv / pool descriptors; params: per conv layer (filters, bias) as numpy fp32 arrays."""
+                 tune: int = 0, device: str = "cuda", per_op: Optional[Sequence[dict]] = None):
+        """ops: conv / pool descriptors; params: per conv layer (filters, bias) as numpy fp32 arrays;
+        per_op: optional plan options per op (dicts with keys of boda_plan_opts, e.g. tile_id, split_k, s2d)."""
         self.ops = list(ops)
         c_ops = []
         for op in self.ops:
@@ -28,9 +29,19 @@ class ConvStack:
                 o.kind = B.BODA_STACK_MAXPOOL
                 o.ksz, o.stride = op.ksz, op.stride
             c_ops.append(o)
-        opts = B.boda_plan_opts_default()
-        opts.math, opts.tune = math, tune
-        self.handle = B.boda_stack_create(c_ops, opts)
+        if per_op is None:
+            opts = B.boda_plan_opts_default()
+            opts.math, opts.tune = math, tune
+            self.handle = B.boda_stack_create(c_ops, opts)
+        else:
+            all_opts = []
+            for d in per_op:
+                o = B.boda_plan_opts_default()
+                o.math, o.tune = math, tune
+                for k, v in (d or {}).items():
+                    setattr(o, k, v)
+                all_opts.append(o)
+            self.handle = B.boda_stack_create_ex(c_ops, all_opts)
         self.filters: List[Optional[torch.Tensor]] = []
         self.biases: List[Optional[torch.Tensor]] = []
         it = iter(params)

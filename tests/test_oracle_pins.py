@@ -51,8 +51,12 @@ def test_worked_example_shapes_and_counts():
 
 
 def test_min_bytes_counts_each_tensor_once():
-    # 205x205x3 input, 96 7x7 filters, stride 2: in + filt + bias + out, 4 bytes each
-    assert orc.conv_min_bytes(1, 3, 205, 205, 96, 7, 7, 2, 0) == 4 * (205 * 205 * 3 + 96 * 147 + 96 + 960000)
+    # The worked example (205x205x3 input, 96 7x7 filters, stride 2).  The paper's AI figure prints 3.84 MB for the
+    # output and 56 448 B for the filters; the input itself is 205*205*3 floats = 504 300 B (counted by hand: the
+    # figure counts the im2col matrix instead) and the bias 96 floats = 384 B.
+    assert orc.conv_min_bytes(1, 3, 205, 205, 96, 7, 7, 2, 0) == 3840000 + 56448 + 504300 + 384
+    # a second hand count: 1x1x1x1 input, one 1x1 filter -> 4 tensors of one float each
+    assert orc.conv_min_bytes(1, 1, 1, 1, 1, 1, 1, 1, 0) == 16
 
 
 def test_sgemm_ai_matches_table1():
@@ -173,7 +177,7 @@ def _im2col_matmul(x, f, b, stride, pad):
             for q in range(Q):
                 inmat[row] = xp[n, :, p * stride:p * stride + R, q * stride:q * stride + S].reshape(-1)
                 row += 1
-    filtsmat = f.reshape(K, -1).T                       # "filtsmat is simply a reshape of filts"
+    filtsmat = f.reshape(K, -1).T                       # Section 3: filtsmat is filts reshaped to (C*R*S) x K
     outmat = inmat @ filtsmat + b[None, :]
     return outmat.reshape(N, P, Q, K).transpose(0, 3, 1, 2)
 

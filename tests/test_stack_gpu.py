@@ -79,6 +79,69 @@ def test_stack_every_layer_matches_fp64_chain(batch, math, tol, tune):
         stack.close()
 
 
+@pytest.mark.parametrize("batch,tune", [(2, 0), (20, 1)])
+def test_stack_layers_in_isolation(batch, tune):
+    """Every GPU layer against the oracle layer applied to the GPU's OWN input of that layer (so an error cannot be
+    blamed on, or hidden by, the layers before it): pooling is compare-and-index work and must be bit-exact in
+    every layout the chain uses; convolutions meet the TF32 bar.  (20, tuned) is what bench.py times."""
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    from paper_1606_00094_b200.stack import ConvStack
+    ops = wl.alexnet_stack(batch)
+    x, params = wl.stack_tensors(batch)
+    stack = ConvStack(ops, params, tune=tune)
+    try:
+        stack.forward(torch.from_numpy(x).cuda())
+        torch.cuda.synchronize()
+        assert B.boda_query_status() == 0
+        descs = stack.describe()
+        prev = x
+        it = iter(params)
+        for i, op in enumerate(ops):
+            got = stack.layer_output(i).cpu().numpy()
+            if op.kind == "conv":
+                w, b = next(it)
+                s = op.shape
+                ref = orc.conv_fwd(prev, w, b, stride=s.stride, pad=s.pad, relu=True)
+                err = orc.rel_l2(got, ref)
+                assert err <= TF32_TOL, f"op {i} ({descs[i]}): rel-L2 {err:.3e}"
+            else:
+                ref = orc.maxpool_fwd(prev, op.ksz, op.stride)
+                np.testing.assert_array_equal(got.astype(np.float64), ref, err_msg=f"op {i} ({descs[i]})")
+            prev = got
+    finally:
+        stack.close()
+
+
+def test_forward_host_is_ordered_behind_earlier_work_on_the_stream():
+    """The host-buffer entry point copies its input on a second stream; that stream must wait for what the caller
+    queued on `stream` before the call.  Here the pinned input buffer is itself filled by a device-to-host copy queued
+    behind a long-running kernel: if the slices were read early, the chain would see the stale zeros."""
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    from paper_1606_00094_b200.stack import ConvStack
+    batch = 4                                           # sliced path (even batch >= 4)
+    ops = wl.alexnet_stack(batch)
+    x, params = wl.stack_tensors(batch)
+    stack = ConvStack(ops, params)
+    try:
+        dx = torch.from_numpy(x).cuda()
+        want = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+        hx_ready = torch.from_numpy(x).pin_memory()
+        stack.forward_host(hx_ready, want)              # reference result (also creates the sub-batch stack)
+        hx = torch.zeros(x.shape, dtype=torch.float32).pin_memory()
+        got = torch.empty(stack.out_shape, dtype=torch.float32).pin_memory()
+        torch.cuda.synchronize()
+        torch.cuda._sleep(200_000_000)                  # about 0.1 s of GPU time on the current stream
+        hx.copy_(dx, non_blocking=True)                 # fills the pinned input once the sleep has ended
+        stack.forward_host(hx, got)
+        assert B.boda_query_status() == 0
+        assert torch.equal(hx, hx_ready)
+        assert torch.equal(got, want), "the input slices were copied before the stream's earlier work had finished"
+    finally:
+        stack.close()
+
+
 def test_stack_rejects_shapes_that_do_not_chain():
     from paper_1606_00094_b200 import binding as B
     a = B.boda_stack_op()
