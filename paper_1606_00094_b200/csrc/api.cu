@@ -174,6 +174,17 @@ bool conv_plan_input_geometry(const boda_conv_plan* p, int* Hp, int* Wp, int* Cp
 
 bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && p->math != BODA_MATH_TF32X3 && igemm_plan_writes_packed(p->ig); }
 
+bool conv_plan_can_fuse_pool(const boda_conv_plan* p, int ksz, int stride)
+{
+    return p->ig != nullptr && p->math != BODA_MATH_TF32X3 && igemm_plan_can_fuse_pool(p->ig, ksz, stride);
+}
+
+int conv_plan_set_pool(boda_conv_plan* p, int ksz, int stride)
+{
+    if (!p->ig) return ksz ? BODA_ERR_UNSUPPORTED : BODA_OK;
+    return igemm_plan_set_pool(p->ig, ksz, stride);
+}
+
 int conv_plan_set_io(boda_conv_plan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
     if (!p->ig) return (in_packed || out_packed) ? BODA_ERR_UNSUPPORTED : BODA_OK;
@@ -221,7 +232,7 @@ int boda_conv_plan_destroy(boda_conv_plan* plan)
     return BODA_OK;
 }
 
-static int plan_time_ms(boda_conv_plan* plan, bool chain_in, bool chain_out, float* ms_out);
+static int plan_time_ms(boda_conv_plan* plan, bool chain_in, bool chain_out, int pool_ksz, int pool_stride, float* ms_out);
 
 static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, DeviceCtx* ctx, int variant,
                       int tile_id, int split_k, boda_conv_plan** out)
@@ -266,16 +277,18 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
 
 int boda_conv_plan_create(const boda_conv_shape* shape, const boda_plan_opts* opts, boda_conv_plan** plan)
 {
-    return boda::conv_plan_create_chained(shape, opts, false, false, plan);
+    return boda::conv_plan_create_chained(shape, opts, false, false, 0, 0, plan);
 }
 
 }  // extern "C"
 
 // chain_in / chain_out: the layer will run inside a chain, its input arriving in the plan's own staged layout and its
 // output leaving in a consumer's staged layout.  Only the tuner looks at them: it times every candidate the way it
-// will run (no staging kernel, bulk-copy epilogue) instead of stand-alone with NCHW on both sides.
+// will run (no staging kernel, bulk-copy epilogue) instead of stand-alone with NCHW on both sides.  pool_ksz > 0: a
+// max-pool follows the layer; candidates that can run it in their epilogue are timed that way, the others together
+// with the separate pooling kernel they would need.
 int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan_opts* opts, bool chain_in, bool chain_out,
-                                   boda_conv_plan** plan)
+                                   int pool_ksz, int pool_stride, boda_conv_plan** plan)
 {
     if (!shape || !plan) return BODA_ERR_INVALID_ARG;
     *plan = nullptr;
@@ -331,6 +344,7 @@ int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan
         std::snprintf(key, sizeof(key), "t%d:%d,%d,%d,%d,%d,%d,%d,%d,%d,v%d,s%d,k%d,m%d,io%d%d", kTileTableVersion, shape->N, shape->C,
                       shape->H, shape->W, shape->K, shape->R, shape->S, shape->stride, shape->pad, o.variant, o.s2d, o.split_k, o.math,
                       chain_in ? 1 : 0, chain_out ? 1 : 0);
+        if (pool_ksz > 0) std::snprintf(key + std::strlen(key), sizeof(key) - std::strlen(key), ",p%dx%d", pool_ksz, pool_stride);
         int c_tile = -1, c_split = 0, c_variant = variant, c_s2d = o.s2d;
         if (tune_cache_lookup(key, &c_tile, &c_split, &c_variant, &c_s2d)) {
             boda_plan_opts oc = o;
@@ -368,7 +382,7 @@ int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan
                     boda_conv_plan* cand = nullptr;
                     if (plan_build(*shape, oc, ctx, c.variant, t, split, &cand) != BODA_OK) continue;
                     float ms = 0.f;
-                    if (plan_time_ms(cand, chain_in, chain_out, &ms) == BODA_OK && ms < best_ms) {
+                    if (plan_time_ms(cand, chain_in, chain_out, pool_ksz, pool_stride, &ms) == BODA_OK && ms < best_ms) {
                         if (best) boda_conv_plan_destroy(best);
                         best = cand;
                         best_ms = ms;
@@ -437,24 +451,43 @@ int boda_conv_fwd_planned(boda_conv_plan* p, const float* in, const float* filt,
 // Times one plan on scratch buffers (used by the tuner).  Synchronises.  chain_in / chain_out: time the plan the
 // way a chain runs it - reading its own staged input layout (no staging kernel) and writing a staged output - where
 // the plan's kernel can; operands hold a small non-zero constant (all-zero operands draw less power than real ones).
-static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float* ms_out)
+static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, int pool_ksz, int pool_stride, float* ms_out)
 {
     const ConvDims& d = p->d;
     size_t n_in = (size_t)d.N * d.C * d.H * d.W, n_out = (size_t)d.M * d.K;
     const size_t n_f = (size_t)d.K * d.Kred;
-    bool in_packed = false, out_packed = false;
+    bool in_packed = false, out_packed = false, fused = false;
     const int oCp = ((d.K + 31) / 32) * 32;
+    int outP = d.P, outQ = d.Q;                  // extent of what the convolution kernel writes
+    const int poolP = pool_ksz > 0 ? boda_conv_out_dim(d.P, pool_ksz, pool_stride, 0) : 0;
+    const int poolQ = pool_ksz > 0 ? boda_conv_out_dim(d.Q, pool_ksz, pool_stride, 0) : 0;
+    const bool pool_after = pool_ksz > 0 && poolP > 0 && poolQ > 0;
     if (p->ig) {
         int Hp = 0, Wp = 0, Cp = 0;
         in_packed = chain_in && igemm_plan_input_geometry(p->ig, &Hp, &Wp, &Cp);
         out_packed = chain_out && igemm_plan_writes_packed(p->ig);
+        if (pool_after && conv_plan_can_fuse_pool(p, pool_ksz, pool_stride) && conv_plan_set_pool(p, pool_ksz, pool_stride) == BODA_OK) {
+            fused = true;
+            outP = poolP; outQ = poolQ;
+        }
         if (in_packed) n_in = (size_t)d.N * Hp * Wp * Cp;
-        if (out_packed) n_out = (size_t)d.N * d.P * d.Q * oCp;
+        if (out_packed) n_out = (size_t)d.N * outP * outQ * oCp;
+        else n_out = (size_t)d.N * d.K * outP * outQ;
         if (in_packed || out_packed) {
-            const int rc_io = conv_plan_set_io(p, in_packed ? 1 : 0, out_packed ? 1 : 0, d.P, d.Q, oCp);
-            if (rc_io != BODA_OK) return rc_io;
+            const int rc_io = conv_plan_set_io(p, in_packed ? 1 : 0, out_packed ? 1 : 0, outP, outQ, oCp);
+            if (rc_io != BODA_OK) { (void)conv_plan_set_pool(p, 0, 0); return rc_io; }
         }
     }
+    const bool separate_pool = pool_after && !fused;
+    float* pool_out = nullptr;
+    // one timed call: the layer, plus the pooling kernel where the layer cannot run it itself
+    auto run_once = [&](float* in_, float* f_, float* b_, float* out_, void* ws_, cudaStream_t st) -> int {
+        int r = boda_conv_fwd_planned(p, in_, f_, b_, out_, ws_, st);
+        if (r != BODA_OK || !separate_pool) return r;
+        if (out_packed)
+            return maxpool_packed_launch(out_, pool_out, d.N, d.K, d.P, d.Q, d.P, d.Q, oCp, pool_ksz, pool_stride, 1, poolP, poolQ, oCp, st);
+        return maxpool_launch(out_, pool_out, d.N, d.K, d.P, d.Q, pool_ksz, pool_stride, st);
+    };
     float *in = nullptr, *f = nullptr, *b = nullptr, *out = nullptr;
     void* ws = nullptr;
     int rc = BODA_OK;
@@ -467,11 +500,14 @@ static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float*
         if (stream) { cudaStreamSynchronize(stream); cudaStreamDestroy(stream); }
         if (in) cudaFree(in); if (f) cudaFree(f); if (b) cudaFree(b); if (out) cudaFree(out); if (ws) cudaFree(ws);
         if (e0) cudaEventDestroy(e0); if (e1) cudaEventDestroy(e1);
+        if (pool_out) cudaFree(pool_out);
         if (in_packed || out_packed) (void)conv_plan_set_io(p, 0, 0, 0, 0, 0);
+        if (fused) (void)conv_plan_set_pool(p, 0, 0);
     };
 #define TRY_T(x) do { cudaError_t _e = (x); if (_e != cudaSuccess) { rc = record_cuda_error(_e, #x); cleanup(); return rc; } } while (0)
     TRY_T(cudaMalloc(&in, n_in * 4)); TRY_T(cudaMalloc(&f, n_f * 4)); TRY_T(cudaMalloc(&b, d.K * 4));
     TRY_T(cudaMalloc(&out, n_out * 4));
+    if (separate_pool) TRY_T(cudaMalloc(&pool_out, (size_t)d.N * oCp * poolP * poolQ * 4));
     if (p->ws_bytes && !in_packed) TRY_T(cudaMalloc(&ws, p->ws_bytes));
     // bytes 0x3c -> the float 0.0115 (exact in TF32 after truncation or rounding alike)
     TRY_T(cudaMemset(in, 0x3c, n_in * 4)); TRY_T(cudaMemset(f, 0x3c, n_f * 4)); TRY_T(cudaMemset(b, 0, d.K * 4));
@@ -479,7 +515,7 @@ static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float*
     TRY_T(cudaStreamSynchronize(0));                    // the fills above ran on the default stream
     TRY_T(cudaStreamCreateWithFlags(&stream, cudaStreamNonBlocking));
     if (p->variant != BODA_VARIANT_DIRECT) { rc = igemm_bind_filters(p->ig, f, stream); if (rc) { cleanup(); return rc; } }
-    for (int i = 0; i < 2; ++i) { rc = boda_conv_fwd_planned(p, in, f, b, out, ws, stream); if (rc) { cleanup(); return rc; } }
+    for (int i = 0; i < 2; ++i) { rc = run_once(in, f, b, out, ws, stream); if (rc) { cleanup(); return rc; } }
     TRY_T(cudaStreamSynchronize(stream));
     // The candidates differ by a few percent, less than the host's launch cost for a small layer: the timed calls are
     // captured in a graph (device time only) and the best of three replays counts.  Without capture: plain launches.
@@ -488,7 +524,7 @@ static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float*
     bool timed = false;
     if (cudaStreamBeginCapture(stream, cudaStreamCaptureModeThreadLocal) == cudaSuccess) {
         int crc = BODA_OK;
-        for (int i = 0; i < iters && crc == BODA_OK; ++i) crc = boda_conv_fwd_planned(p, in, f, b, out, ws, stream);
+        for (int i = 0; i < iters && crc == BODA_OK; ++i) crc = run_once(in, f, b, out, ws, stream);
         const cudaError_t ce = cudaStreamEndCapture(stream, &graph);
         if (crc == BODA_OK && ce == cudaSuccess && graph && cudaGraphInstantiate(&exec, graph, 0) == cudaSuccess) {
             TRY_T(cudaGraphLaunch(exec, stream));
@@ -510,7 +546,7 @@ static int plan_time_ms(boda_conv_plan* p, bool chain_in, bool chain_out, float*
     }
     if (!timed) {
         TRY_T(cudaEventRecord(e0, stream));
-        for (int i = 0; i < iters; ++i) { rc = boda_conv_fwd_planned(p, in, f, b, out, ws, stream); if (rc) { cleanup(); return rc; } }
+        for (int i = 0; i < iters; ++i) { rc = run_once(in, f, b, out, ws, stream); if (rc) { cleanup(); return rc; } }
         TRY_T(cudaEventRecord(e1, stream));
         TRY_T(cudaEventSynchronize(e1));
         TRY_T(cudaEventElapsedTime(&ms, e0, e1));

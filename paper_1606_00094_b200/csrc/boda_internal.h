@@ -140,12 +140,16 @@ void conv_plan_out_dims(const boda_conv_plan* plan, int* N, int* K, int* P, int*
 // boda_conv_plan_create for a layer of a chain: with opts->tune the candidates are timed reading a staged input
 // (chain_in) and writing a staged output (chain_out), the way the chain will run them
 int conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan_opts* opts, bool chain_in, bool chain_out,
-                             boda_conv_plan** plan);
+                             int pool_ksz, int pool_stride, boda_conv_plan** plan);
 // chained layers: the staged input layout a tensor-core plan reads (false: the plan reads NCHW only), and the
 // switch that makes it read that layout directly / write its output in a consumer's staged layout
 bool conv_plan_input_geometry(const boda_conv_plan* plan, int* Hp, int* Wp, int* Cp);
 bool conv_plan_can_write_packed(const boda_conv_plan* plan);
 int conv_plan_set_io(boda_conv_plan* plan, int in_packed, int out_packed, int oHp, int oWp, int oCp);
+// chained layers: a max-pool that follows the convolution, fused into its epilogue (the plan then writes the pooled
+// tensor); set_pool(plan, 0, 0) undoes it; call before conv_plan_set_io
+bool conv_plan_can_fuse_pool(const boda_conv_plan* plan, int ksz, int stride);
+int conv_plan_set_pool(boda_conv_plan* plan, int ksz, int stride);
 
 // ---- pooling -------------------------------------------------------------------------------------
 int maxpool_launch(const float* in, float* out, int N, int C, int H, int W, int ksz, int stride,

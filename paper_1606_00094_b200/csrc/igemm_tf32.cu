@@ -702,6 +702,9 @@ struct IgemmPlan {
     // halo kernel only
     int nacc = 0;                    // 0: im2col kernel; 1, 2 or 4: halo kernel with that many accumulators; -1: gather kernel; -2: 1x1 from NCHW
     int Hp = 0, Wp = 0, lead = 0, slab_rows = 0, nbox = 0, box_rows = 0, a_slot_bytes = 0, b_stages = 0;
+    // fused 3x3 / stride-2 max-pooling of the output (halo kernel with 2 or 4 accumulators, no split)
+    int pool_rows = 0, tiles_per_image = 0, poolP = 0, poolQ = 0;
+    int tiles_m_unpooled = 0;
 };
 
 // Geometry of the halo kernel for a shape and tile; false if the shape does not fit it.
@@ -1245,8 +1248,10 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
         return;
     }
     if (p->nacc > 0) {
-        std::snprintf(buf, n, "%stile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d", view, 128 * p->nacc, p->BN,
-                      p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits);
+        char pool[48] = "";
+        if (p->pool_rows > 0) std::snprintf(pool, sizeof(pool), " +maxpool3x3s2(%d rows/tile)", p->pool_rows);
+        std::snprintf(buf, n, "%stile=halo_%dx%d(id %d) slab=%d stages=%d split_k=%d grid=%dx%dx%d%s", view, 128 * p->nacc, p->BN,
+                      p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits, pool);
         return;
     }
     std::snprintf(buf, n, "%s%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->terms == 3 ? "x3 " : "", p->BN, p->tile_id,
@@ -1320,6 +1325,7 @@ static OutSpec make_out_spec(const IgemmPlan* p, float* out)
     o.out = out;
     o.packed = p->out_packed;
     o.K = d.K; o.P = d.P; o.Q = d.Q; o.PQ = d.P * d.Q;
+    if (p->pool_rows > 0) { o.P = p->poolP; o.Q = p->poolQ; o.PQ = p->poolP * p->poolQ; }   // the pooled tensor
     o.Hp = p->oHp; o.Wp = p->oWp; o.Cp = p->oCp;
     o.relu = d.relu;
     return o;
@@ -1333,12 +1339,54 @@ bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
     return true;
 }
 
+// Pooled rows per tile of the halo kernel when 3x3 / stride-2 pooling is fused into its epilogue; 0 if it cannot be:
+// a tile of 128*nacc flat positions must hold 2*rows + 1 whole output rows, and two blocks of [positions][32 channels]
+// plus the pooled tile must fit in the shared memory the operand buffers leave idle.
+static int halo_pool_rows(const IgemmPlan* p, int ksz, int stride)
+{
+    const ConvDims& d = p->d;
+    if (p->nacc != 2 && p->nacc != 4) return 0;
+    if (p->splits != 1 || ksz != 3 || stride != 2 || d.P < 3 || d.Q < 3) return 0;
+    const int poolP = (d.P - 3) / 2 + 1, poolQ = (d.Q - 3) / 2 + 1;
+    int rows = (128 * p->nacc - d.Q) / (2 * p->Wp);
+    if (rows > poolP) rows = poolP;
+    const long long region = (long long)halo::kASlots * p->a_slot_bytes + (long long)p->b_stages * p->BN * 128;
+    while (rows >= 1 && 2LL * p->nacc * 128 * 128 + (long long)rows * poolQ * p->BN * 4 > region) --rows;
+    return rows < 1 ? 0 : rows;
+}
+
+bool igemm_plan_can_fuse_pool(const IgemmPlan* p, int ksz, int stride) { return halo_pool_rows(p, ksz, stride) > 0; }
+
+int igemm_plan_set_pool(IgemmPlan* p, int ksz, int stride)
+{
+    if (ksz == 0) {                       // back to the unfused form
+        if (p->pool_rows > 0) p->tiles_m = p->tiles_m_unpooled;
+        p->pool_rows = p->tiles_per_image = p->poolP = p->poolQ = 0;
+        return BODA_OK;
+    }
+    const int rows = halo_pool_rows(p, ksz, stride);
+    if (rows <= 0) return BODA_ERR_UNSUPPORTED;
+    if (p->pool_rows == 0) p->tiles_m_unpooled = p->tiles_m;
+    p->pool_rows = rows;
+    p->poolP = (p->d.P - 3) / 2 + 1;
+    p->poolQ = (p->d.Q - 3) / 2 + 1;
+    p->tiles_per_image = (p->poolP + rows - 1) / rows;
+    p->tiles_m = p->d.N * p->tiles_per_image;
+    return BODA_OK;
+}
+
+void igemm_plan_pooled_dims(const IgemmPlan* p, int* P, int* Q)
+{
+    if (p->pool_rows > 0) { *P = p->poolP; *Q = p->poolQ; } else { *P = p->d.P; *Q = p->d.Q; }
+}
+
 int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
     if (in_packed && (p->s2d || p->nacc < 0)) return BODA_ERR_UNSUPPORTED;
     if ((in_packed || out_packed) && p->terms == 3) return BODA_ERR_UNSUPPORTED;
     if (out_packed && p->nacc == -2) return BODA_ERR_UNSUPPORTED;        // that kernel's tiles follow images: NCHW output only
-    if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < p->d.P || oWp < p->d.Q)) return BODA_ERR_INVALID_ARG;
+    const int outP = p->pool_rows > 0 ? p->poolP : p->d.P, outQ = p->pool_rows > 0 ? p->poolQ : p->d.Q;
+    if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < outP || oWp < outQ)) return BODA_ERR_INVALID_ARG;
     p->in_packed = in_packed != 0;
     p->out_packed = out_packed ? 1 : 0;
     p->oHp = oHp; p->oWp = oWp; p->oCp = oCp;
@@ -1430,6 +1478,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
         hp.bias = bias; hp.o = make_out_spec(p, out); hp.tx_extra = p->tx_extra;
         hp.status = p->d_status;
+        hp.pool_rows = p->pool_rows; hp.tiles_per_image = p->tiles_per_image;
         switch (p->BN * 10 + p->nacc) {
             case 641: return launch_halo<64, 1>(p, hp, stream);
             case 1281: return launch_halo<128, 1>(p, hp, stream);

@@ -39,6 +39,13 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
 bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp);
 int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp);
 
+// Fused ReLU -> 3x3 / stride-2 max-pooling in the epilogue (halo tiles with 2 or 4 accumulators, no split): the plan
+// then writes the POOLED tensor (out_packed geometry and NCHW extents refer to it).  set_pool(p, 0, 0) undoes it.
+// Call set_pool before set_io.
+bool igemm_plan_can_fuse_pool(const IgemmPlan* p, int ksz, int stride);
+int igemm_plan_set_pool(IgemmPlan* p, int ksz, int stride);
+void igemm_plan_pooled_dims(const IgemmPlan* p, int* P, int* Q);
+
 // Scratch-in-a-caller-region form (allocates nothing): bytes needed at least, and the run itself.
 size_t igemm_region_min_bytes(const ConvDims& d);
 int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const float* filt, const float* bias,

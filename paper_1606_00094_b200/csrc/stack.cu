@@ -30,6 +30,9 @@ struct boda_stack {
         int oHp = 0, oWp = 0, oCp = 0;
         bool in_packed = false;             // = out_packed of the previous op
         int iHp = 0, iWp = 0, iCp = 0;
+        // a 3x3 / stride-2 max-pool that follows a convolution may run inside that convolution's epilogue: the
+        // convolution is then `fused_pool` and writes the pool op's activation; the pool op is `skipped`
+        bool fused_pool = false, skipped = false;
     };
     std::vector<Op> ops;
     int device = 0;
@@ -62,7 +65,12 @@ int run_ops(boda_stack* s, const float* in, float* out, cudaStream_t stream, cud
     const int n = (int)s->ops.size();
     for (int i = 0; i < n; ++i) {
         boda_stack::Op& op = s->ops[i];
-        float* dst = (i == n - 1) ? out : op.out;
+        if (op.skipped) {                    // ran inside the preceding convolution
+            if (events) for (int e = 0; e < 3; ++e) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + e], stream));
+            continue;
+        }
+        const int w = op.fused_pool ? i + 1 : i;            // the op whose activation this launch writes
+        float* dst = (w == n - 1) ? out : s->ops[w].out;
         if (events) BODA_CUDA_TRY(cudaEventRecord(events[3 * i + 0], stream));
         int rc;
         if (op.kind == 0) {
@@ -198,11 +206,31 @@ int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_op
     // (a tensor-core convolution, or a pool whose own input is staged) and the consumer can read it (a tensor-core
     // convolution that is not a space-to-depth view, or a pool); NCHW otherwise.  The chain's input and output are NCHW.
     const bool chain_layouts = !std::getenv("BODA_STACK_NCHW");
+    const bool fuse_pools = !std::getenv("BODA_STACK_NO_POOL_FUSION");
     auto assign_layouts = [&]() {
-        for (auto& op : s->ops) { op.in_packed = op.out_packed = false; op.oHp = op.oWp = op.oCp = op.iHp = op.iWp = op.iCp = 0; }
-        for (int i = 0; i + 1 < (int)s->ops.size(); ++i) {
+        const int n = (int)s->ops.size();
+        for (auto& op : s->ops) {
+            op.in_packed = op.out_packed = op.fused_pool = op.skipped = false;
+            op.oHp = op.oWp = op.oCp = op.iHp = op.iWp = op.iCp = 0;
+            if (op.kind == BODA_STACK_CONV && op.plan) (void)conv_plan_set_pool(op.plan, 0, 0);
+        }
+        // which pools run inside the preceding convolution's epilogue
+        for (int i = 0; i + 1 < n; ++i) {
+            boda_stack::Op& conv = s->ops[i];
+            boda_stack::Op& pool = s->ops[i + 1];
+            if (fuse_pools && conv.kind == BODA_STACK_CONV && pool.kind == BODA_STACK_MAXPOOL &&
+                conv_plan_can_fuse_pool(conv.plan, pool.ksz, pool.stride) && conv_plan_set_pool(conv.plan, pool.ksz, pool.stride) == BODA_OK) {
+                conv.fused_pool = true;
+                pool.skipped = true;
+            }
+        }
+        // hand-over between the ops that run
+        for (int i = 0; i + 1 < n; ++i) {
             boda_stack::Op& prod = s->ops[i];
-            boda_stack::Op& cons = s->ops[i + 1];
+            if (prod.skipped) continue;
+            const int w = prod.fused_pool ? i + 1 : i;       // the op whose activation the producer writes
+            if (w + 1 >= n) break;
+            boda_stack::Op& cons = s->ops[w + 1];
             const bool can_write = prod.kind == BODA_STACK_CONV ? conv_plan_can_write_packed(prod.plan) : prod.in_packed;
             int Hp = cons.H, Wp = cons.W, Cp = ((cons.C + 31) / 32) * 32;
             bool can_read = true;
@@ -210,6 +238,7 @@ int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_op
             if (chain_layouts && can_write && can_read) {
                 prod.out_packed = true; prod.oHp = Hp; prod.oWp = Wp; prod.oCp = Cp;
                 cons.in_packed = true; cons.iHp = Hp; cons.iWp = Wp; cons.iCp = Cp;
+                if (prod.fused_pool) { boda_stack::Op& pl = s->ops[w]; pl.out_packed = true; pl.oHp = Hp; pl.oWp = Wp; pl.oCp = Cp; }
             }
         }
     };
@@ -223,7 +252,9 @@ int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_op
         boda_stack::Op& op = s->ops[i];
         if (op.kind != BODA_STACK_CONV || !per_op_opts[i].tune || per_op_opts[i].tile_id >= 0) continue;
         boda_conv_plan* tuned = nullptr;
-        rc = conv_plan_create_chained(&op.conv, &per_op_opts[i], op.in_packed, op.out_packed, &tuned);
+        const bool pool_next = fuse_pools && i + 1 < (int)s->ops.size() && s->ops[i + 1].kind == BODA_STACK_MAXPOOL;
+        rc = conv_plan_create_chained(&op.conv, &per_op_opts[i], op.in_packed, op.out_packed || (op.fused_pool && s->ops[i + 1].out_packed),
+                                      pool_next ? s->ops[i + 1].ksz : 0, pool_next ? s->ops[i + 1].stride : 0, &tuned);
         if (rc != BODA_OK) break;
         boda_conv_plan_destroy(op.plan);
         op.plan = tuned;
@@ -238,7 +269,7 @@ int boda_stack_create_ex(const boda_stack_op* ops, int n_ops, const boda_plan_op
             rc = conv_plan_set_io(op.plan, op.in_packed ? 1 : 0, op.out_packed ? 1 : 0, op.oHp, op.oWp, op.oCp);
             if (rc != BODA_OK) break;
         }
-        if (i + 1 < (int)s->ops.size()) {
+        if (i + 1 < (int)s->ops.size() && !op.fused_pool) {   // a convolution with a fused pool writes the pool op's activation
             const size_t elems = op.out_packed ? (size_t)op.N * op.oHp * op.oWp * op.oCp : op.out_elems;
             cudaError_t e = cudaMalloc(&op.out, elems * sizeof(float));
             if (e == cudaSuccess) e = cudaMemset(op.out, 0, elems * sizeof(float));   // staged layouts: the padding stays zero
@@ -284,6 +315,7 @@ int boda_stack_copy_layer_output(const boda_stack* s, int op_index, float* dst_n
 {
     if (!s || op_index < 0 || op_index >= (int)s->ops.size() - 1 || !dst_nchw) return BODA_ERR_INVALID_ARG;
     const boda_stack::Op& op = s->ops[op_index];
+    if (op.fused_pool) return BODA_ERR_UNSUPPORTED;      // never materialised: only its pooled form exists
     if (op.out_packed)
         return unpack_to_nchw_launch(op.out, dst_nchw, op.N, op.oC, op.oH, op.oW, op.oHp, op.oWp, op.oCp, (cudaStream_t)stream);
     BODA_CUDA_TRY(cudaMemcpyAsync(dst_nchw, op.out, op.out_elems * sizeof(float), cudaMemcpyDeviceToDevice, (cudaStream_t)stream));
@@ -299,7 +331,8 @@ int boda_stack_describe(const boda_stack* s, int op_index, char* buf, size_t n)
         const int rc = boda_conv_plan_describe(op.plan, tmp, sizeof(tmp));
         if (rc != BODA_OK) return rc;
     } else {
-        std::snprintf(tmp, sizeof(tmp), "maxpool %dx%d stride %d", op.ksz, op.ksz, op.stride);
+        std::snprintf(tmp, sizeof(tmp), "maxpool %dx%d stride %d%s", op.ksz, op.ksz, op.stride,
+                      op.skipped ? " (fused into the preceding convolution's epilogue)" : "");
     }
     std::snprintf(buf, n, "%s in=%s out=%s", tmp, op.in_packed ? "staged" : "nchw", op.out_packed ? "staged" : "nchw");
     return BODA_OK;
@@ -333,8 +366,10 @@ int boda_stack_run_op(boda_stack* s, int op_index, const float* in, float* out, 
     if (!s || op_index < 0 || op_index >= (int)s->ops.size()) return BODA_ERR_INVALID_ARG;
     const int n = (int)s->ops.size();
     boda_stack::Op& op = s->ops[op_index];
+    if (op.skipped) return BODA_OK;                      // runs inside the preceding convolution
     const float* src = op_index == 0 ? in : s->ops[op_index - 1].out;
-    float* dst = op_index == n - 1 ? out : op.out;
+    const int w = op.fused_pool ? op_index + 1 : op_index;
+    float* dst = w == n - 1 ? out : s->ops[w].out;
     if (!src || !dst) return BODA_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
     if (op.kind == BODA_STACK_CONV) {
@@ -437,7 +472,7 @@ int boda_stack_kernels_per_fwd(const boda_stack* s)
 {
     if (!s) return 0;
     int n = 0;
-    for (const auto& op : s->ops) n += op.kind == BODA_STACK_CONV ? boda_conv_plan_kernels_per_call(op.plan) : 1;
+    for (const auto& op : s->ops) n += op.kind == BODA_STACK_CONV ? boda_conv_plan_kernels_per_call(op.plan) : op.skipped ? 0 : 1;
     return n;
 }
 

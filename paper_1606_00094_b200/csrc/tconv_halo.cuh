@@ -45,6 +45,11 @@ struct HaloParams {
     OutSpec o;                   // output tensor, layout and activation
     int* status;
     int tx_extra;                // test hook: bytes added to the first stage's expected transfer size of CTA (0,0,0)
+    // fused 3x3 / stride-2 max-pooling of the output (pool_rows > 0): a tile then covers output rows
+    // 2*pool_rows*j .. 2*pool_rows*j + 2*pool_rows of ONE image (j = tile index within the image) and stores the
+    // pool_rows pooled rows they contain; `o` describes the POOLED tensor (o.P, o.Q = pooled extent)
+    int pool_rows;
+    int tiles_per_image;
 };
 
 // output location of flat position f = (n*Hp + p)*Wp + q; positions with p >= P or q >= Q are dropped
@@ -74,6 +79,93 @@ struct HaloCfg {
     static constexpr int ISSUERS = NACC >= 4 ? 4 : NACC >= 2 ? 2 : 1;
 };
 
+// ---- fused ReLU -> max-pool epilogue (3x3 window, stride 2, no padding, floor extent).
+// The paper fuses the activation into the convolution (Section 2) and names fusion as what a BLAS call cannot do
+// (Section 3); here the pooling that follows the activation is fused as well, so that the convolution's output -
+// four times the bytes of the pooled tensor - is never written.  The tile's rows are whole output rows of one image
+// (see HaloParams::pool_rows), so every pooling window of the pooled rows it owns lies inside the tile.
+// 32 channels at a time: all accumulators' columns [32c, 32c+32) go, with bias and ReLU applied, into a shared-memory
+// block [128*NACC positions][32 channels] (16-byte pieces XOR-swizzled by the position, so that thread-per-position
+// writes and the window reads below are free of bank conflicts); after a barrier of the 256 epilogue threads every
+// thread takes pooled (row, column, 4 channels) items, reads the nine window positions and writes the maximum,
+// rounded to TF32, into the pooled tile [pool_rows * Q][BN] (or straight to an NCHW tensor).  Two blocks alternate,
+// so filling block c+1 overlaps pooling block c.  At the end each pooled position leaves as one bulk copy.
+template <int BN, int NACC>
+__device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32_t smem_base, uint32_t tmem_acc, const float* s_bias,
+                                                     int k0, int group, int quarter, int lane, int etid)
+{
+    static_assert(NACC == 2 || NACC == 4, "the two epilogue groups take alternate accumulators");
+    constexpr int NCH = BN / 32;
+    constexpr uint32_t BLOCK_BYTES = (uint32_t)NACC * 128u * 128u;
+    const uint32_t pooled = smem_base + 2u * BLOCK_BYTES;
+    const int n = (int)blockIdx.x / p.tiles_per_image;
+    const int j = (int)blockIdx.x - n * p.tiles_per_image;
+    const int prow0 = p.pool_rows * j;                                  // first pooled row of this tile
+    const int prows = min(p.pool_rows, p.o.P - prow0);                  // pooled rows this tile owns
+    const int items = prows * p.o.Q * 8;                                // (pooled position, 4 channels)
+    const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+#pragma unroll 1
+    for (int c = 0; c < NCH; ++c) {
+        const uint32_t block = smem_base + (uint32_t)(c & 1) * BLOCK_BYTES;
+#pragma unroll 1
+        for (int acc = group; acc < NACC; acc += 2) {
+            const int pos = acc * 128 + quarter * 32 + lane;
+            uint32_t v[32];
+            tmem_ld_32cols(trow + acc * BN + 32 * c, v);
+            tmem_ld_wait();
+            float y[32];
+            bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
+            const uint32_t a = block + (uint32_t)pos * 128u;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+                st_shared_v4(a + (uint32_t)((g ^ (pos & 7)) << 4), y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
+        }
+        // every thread is past its pooling of block c-1 when it arrives here, so block (c+1)&1 may be refilled after it
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+#pragma unroll 1
+        for (int item = etid; item < items; item += 256) {
+            const int g = item & 7, t = item >> 3;
+            const int pr = t / p.o.Q, pq = t - pr * p.o.Q;
+            const int pos0 = 2 * pr * p.Wp + 2 * pq;
+            float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+            for (int dr = 0; dr < 3; ++dr)
+#pragma unroll
+                for (int ds = 0; ds < 3; ++ds) {
+                    const int pos = pos0 + dr * p.Wp + ds;
+                    const float4 x = ld_shared_v4(block + (uint32_t)pos * 128u + (uint32_t)((g ^ (pos & 7)) << 4));
+                    if (dr == 0 && ds == 0) m = x;
+                    else { m.x = fmaxf(m.x, x.x); m.y = fmaxf(m.y, x.y); m.z = fmaxf(m.z, x.z); m.w = fmaxf(m.w, x.w); }
+                }
+            if (p.o.packed) {
+                st_shared_v4(pooled + (uint32_t)(t * BN + 32 * c + 4 * g) * 4u, round_to_tf32(m.x), round_to_tf32(m.y),
+                             round_to_tf32(m.z), round_to_tf32(m.w));
+            } else {
+                const int k = k0 + 32 * c + 4 * g;
+                float* dst = p.o.out + ((size_t)(n * p.o.K + k) * p.o.P + prow0 + pr) * p.o.Q + pq;
+                const float mv[4] = {m.x, m.y, m.z, m.w};
+#pragma unroll
+                for (int e = 0; e < 4; ++e)
+                    if (k + e < p.o.K) dst[(size_t)e * p.o.PQ] = mv[e];
+            }
+        }
+    }
+    if (p.o.packed) {
+        fence_proxy_async_smem();
+        asm volatile("bar.sync 1, 256;" ::: "memory");
+        const int w = min(BN, p.o.Cp - k0);
+        if (w > 0) {
+            for (int t = etid; t < prows * p.o.Q; t += 256) {
+                const int pr = t / p.o.Q, pq = t - pr * p.o.Q;
+                float* dst = p.o.out + ((size_t)(n * p.o.Hp + prow0 + pr) * p.o.Wp + pq) * (size_t)p.o.Cp + k0;
+                bulk_store_global(dst, pooled + (uint32_t)(t * BN) * 4u, (uint32_t)w * 4u);
+            }
+        }
+        bulk_commit();
+        bulk_wait_all();
+    }
+}
+
 template <int BN, int NACC>
 __global__ void __launch_bounds__(kThreads, 1)
 tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
@@ -94,7 +186,11 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     const int warp = threadIdx.x >> 5;
     const int lane = threadIdx.x & 31;
-    const int f0 = blockIdx.x * (128 * NACC);
+    int f0 = blockIdx.x * (128 * NACC);
+    if (p.pool_rows > 0) {          // tiles of whole output rows of one image (fused pooling)
+        const int n = (int)blockIdx.x / p.tiles_per_image;
+        f0 = n * p.HpWp + 2 * p.pool_rows * ((int)blockIdx.x - n * p.tiles_per_image) * p.Wp;
+    }
     const int k0 = blockIdx.y * BN;
     const int it_begin = blockIdx.z * p.iters_per_split;
     const int it_end = min(it_begin + p.iters_per_split, p.iters_total);
@@ -229,7 +325,9 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         const bool ok = (s_abort == 0);
         tc_fence_after();
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-        if (ok && p.splits == 1) {
+        if (ok && p.pool_rows > 0) {
+            if constexpr (NACC >= 2) halo_pooled_epilogue<BN, NACC>(p, smem_base, tmem_acc, s_bias, k0, group, quarter, lane, etid);
+        } else if (ok && p.splits == 1) {
             constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
             const int c_begin = (NACC == 1 && group) ? HALF : 0, c_end = (NACC == 1 && !group) ? HALF : NCH;
             // Staged layout: rows go through shared memory (the operand buffers are idle now) and leave as bulk

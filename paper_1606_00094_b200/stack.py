@@ -88,13 +88,19 @@ class ConvStack:
         """Host buffers in and out (pinned for asynchronous copies); returns after the result has landed."""
         B.boda_stack_fwd_host(self.handle, x_host, out_host)
 
-    def layer_output(self, i: int) -> torch.Tensor:
-        """NCHW copy of the activation op i wrote during the last forward pass."""
+    def layer_output(self, i: int) -> Optional[torch.Tensor]:
+        """NCHW copy of the activation op i wrote during the last forward pass; None for a convolution whose
+        max-pool runs inside its epilogue (its own output is never materialised, only the pooled one)."""
         if i == len(self.ops) - 1:
             return self.out.clone()
         shape = B.boda_stack_out_dims(self.handle, i)
         dst = torch.empty(shape, dtype=torch.float32, device=self.out.device)
-        B.boda_stack_copy_layer_output(self.handle, i, dst)
+        try:
+            B.boda_stack_copy_layer_output(self.handle, i, dst)
+        except B.BodaError as e:
+            if e.status == B.BODA_ERR_UNSUPPORTED:
+                return None
+            raise
         torch.cuda.synchronize()
         return dst
 

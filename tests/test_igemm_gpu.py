@@ -311,11 +311,11 @@ def test_tuned_choice_is_remembered_in_the_cache_file(tmp_path, monkeypatch):
     t0 = time.time(); second = B.ConvPlan(shape, tune=1); t_second = time.time() - t0
     try:
         lines = cache.read_text().strip().splitlines()
-        assert len(lines) == 1 and lines[0].startswith("t3:2,64,12,12,96,3,3,1,1,")       # one entry, keyed by tile-table version and shape
+        assert len(lines) == 1 and lines[0].startswith("t4:2,64,12,12,96,3,3,1,1,")       # one entry, keyed by tile-table version and shape
         assert second.describe() == first.describe()
         assert t_second < t_first                                                          # no candidates were timed again
         # an entry written for other tile tables is ignored, not misread
-        cache.write_text(lines[0].replace("t3:", "t2:", 1) + "\n")
+        cache.write_text(lines[0].replace("t4:", "t2:", 1) + "\n")
         third = B.ConvPlan(shape, tune=1)
         third.close()
         assert len(cache.read_text().strip().splitlines()) == 2

@@ -66,8 +66,11 @@ def _run_chain_exact(ops, per_op, seed, expect):
         assert B.boda_query_status() == 0
         assert torch.equal(out, out2)
         for i, r in enumerate(ref):
-            got = stack.layer_output(i).cpu().numpy().astype(np.float64)
-            np.testing.assert_array_equal(got, r, err_msg=f"op {i}: {descs[i]}")
+            got = stack.layer_output(i)
+            if got is None:                 # a convolution whose pool runs in its epilogue: only the pooled tensor exists
+                assert "fused" in descs[i + 1]
+                continue
+            np.testing.assert_array_equal(got.cpu().numpy().astype(np.float64), r, err_msg=f"op {i}: {descs[i]}")
     finally:
         stack.close()
 
@@ -106,7 +109,8 @@ CONV_POOL = [
 
 
 @pytest.mark.parametrize("prod,cons", CONV_POOL)
-def test_conv_pool_conv_pool_staged_is_exact(prod, cons):
+def test_conv_pool_conv_pool_staged_is_exact(prod, cons, monkeypatch):
+    monkeypatch.setenv("BODA_STACK_NO_POOL_FUSION", "1")          # the pooling kernels themselves are under test here
     ops = [StackOp("conv", ConvShape(2, 24, 19, 19, 40, 3, 3, 1, 1, False)),
            StackOp("pool"),                                                            # 19 -> 9
            StackOp("conv", ConvShape(2, 40, 9, 9, 72, 3, 3, 1, 1, True)),
@@ -115,6 +119,30 @@ def test_conv_pool_conv_pool_staged_is_exact(prod, cons):
               {"variant": 2, "tile_id": cons[0], "split_k": cons[1]}, {}]
     _run_chain_exact(ops, per_op, 1200, {0: ["out=staged"], 1: ["in=staged", "out=staged"], 2: ["in=staged", "out=staged"],
                                          3: ["in=staged", "out=nchw"]})
+
+
+# The same chain with the pools run inside the convolutions' epilogues (halo tiles of 256 or 512 positions, no split):
+# tiles then follow whole output rows of one image, and the pooled tensor is written in the consumer's staged layout
+# (first pool) or as NCHW (last pool).  19 x 19 -> 9 x 9 pooled: tiles of 256 positions hold 4 pooled rows (ragged
+# last tile), of 512 positions all 9.
+FUSED = [
+    ((HALO_256x96, 1), (HALO_256x128, 1)),
+    ((HALO_512x96, 1), (HALO_512x64, 1)),
+    ((HALO_256x128, 1), (IM2COL_128, 1)),          # the consumer's pool stays a kernel of its own (im2col tile)
+]
+
+
+@pytest.mark.parametrize("prod,cons", FUSED)
+def test_fused_pool_epilogue_is_exact(prod, cons):
+    ops = [StackOp("conv", ConvShape(2, 24, 19, 19, 40, 3, 3, 1, 1, True)),
+           StackOp("pool"),
+           StackOp("conv", ConvShape(2, 40, 9, 9, 72, 3, 3, 1, 1, True)),
+           StackOp("pool")]
+    per_op = [{"variant": 2, "tile_id": prod[0], "split_k": prod[1]}, {},
+              {"variant": 2, "tile_id": cons[0], "split_k": cons[1]}, {}]
+    halo_cons = cons[0] >= 5
+    _run_chain_exact(ops, per_op, 1300, {0: ["+maxpool3x3s2"], 1: ["fused"], 2: ["in=staged"] + (["+maxpool3x3s2"] if halo_cons else []),
+                                         3: ["fused"] if halo_cons else ["in=staged", "out=nchw"]})
 
 
 # a first layer on 3 channels with a strided window through its space-to-depth view (NCHW in, halo tile, staged
@@ -126,7 +154,7 @@ def test_space_to_depth_first_layer_pool_conv_is_exact(first, second):
            StackOp("conv", ConvShape(2, 80, 7, 7, 48, 5, 5, 1, 2, True))]
     per_op = [{"variant": 2, "tile_id": first[0], "split_k": first[1], "s2d": 1}, {},
               {"variant": 2, "tile_id": second[0], "split_k": second[1]}]
-    _run_chain_exact(ops, per_op, 1500, {0: ["s2d", "in=nchw", "out=staged"], 1: ["in=staged", "out=staged"], 2: ["in=staged"]})
+    _run_chain_exact(ops, per_op, 1500, {0: ["s2d", "in=nchw", "out=staged", "+maxpool3x3s2"], 1: ["fused"], 2: ["in=staged"]})
 
 
 def test_default_plans_chain_is_exact():
