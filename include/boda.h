@@ -63,6 +63,16 @@ enum { BODA_MATH_AUTO = 0,       /* TF32 tensor cores where a tensor-core varian
                                     the next step (Sections 2 and 6); this is the mode for callers who need FP32
                                     accuracy from the tensor cores.  NCHW in and out only; K1CONV and TCONV (im2col
                                     kernel); where no tensor-core variant is legal the FP32 kernel runs instead. */
+enum { BODA_MATH_F16 = 4 };      /* reduced-precision STORAGE (Section 2 of the paper notes that 16-bit storage suffices for
+                                    inference; Section 6 lists it as the next step): input and filters are rounded to
+                                    fp16 (nearest even) when they are staged, products are exact and accumulate in
+                                    fp32 on the tensor cores (kind::f16, 16 channels per MMA instead of 8), output is
+                                    fp32.  A precision class of its own, never chosen automatically: fp16 keeps TF32's
+                                    10 mantissa bits, so the relative L2 error against the fp64 result stays <= 5e-3
+                                    for operands inside fp16's range (|x| < 65504; larger values overflow to infinity,
+                                    values below 6e-8 flush to zero), and <= 1e-5 against the fp64 result computed
+                                    from the fp16-rounded operands.  NCHW in and out only; K1CONV and TCONV (im2col
+                                    kernel); where no tensor-core variant is legal the FP32 kernel runs instead. */
 
 typedef struct boda_conv_shape {
     int N, C, H, W;              /* input  [N][C][H][W] */

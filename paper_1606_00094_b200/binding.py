@@ -28,7 +28,7 @@ BODA_ERR_DEVICE_TIMEOUT = 4
 BODA_ERR_NOMEM = 5
 BODA_ERR_TOO_LARGE = 6
 BODA_VARIANT_AUTO, BODA_VARIANT_DIRECT, BODA_VARIANT_K1CONV, BODA_VARIANT_TCONV = -1, 0, 1, 2
-BODA_MATH_AUTO, BODA_MATH_FP32, BODA_MATH_TF32, BODA_MATH_TF32X3 = 0, 1, 2, 3
+BODA_MATH_AUTO, BODA_MATH_FP32, BODA_MATH_TF32, BODA_MATH_TF32X3, BODA_MATH_F16 = 0, 1, 2, 3, 4
 VARIANT_NAMES = {0: "direct", 1: "k1conv", 2: "tconv"}
 
 

@@ -172,7 +172,7 @@ bool conv_plan_input_geometry(const boda_conv_plan* p, int* Hp, int* Wp, int* Cp
     return p->ig ? igemm_plan_input_geometry(p->ig, Hp, Wp, Cp) : false;
 }
 
-bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && p->math != BODA_MATH_TF32X3 && igemm_plan_writes_packed(p->ig); }
+bool conv_plan_can_write_packed(const boda_conv_plan* p) { return p->ig != nullptr && igemm_plan_writes_packed(p->ig); }
 
 bool conv_plan_can_fuse_pool(const boda_conv_plan* p, int ksz, int stride)
 {
@@ -265,9 +265,9 @@ static int plan_build(const boda_conv_shape& shape, const boda_plan_opts& o, Dev
         }
         p->ws_bytes = 0;
     } else {
-        p->math = o.math == BODA_MATH_TF32X3 ? BODA_MATH_TF32X3 : BODA_MATH_TF32;
-        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig, o.math == BODA_MATH_TF32X3,
-                               o.max_workspace);
+        p->math = o.math == BODA_MATH_TF32X3 ? BODA_MATH_TF32X3 : o.math == BODA_MATH_F16 ? BODA_MATH_F16 : BODA_MATH_TF32;
+        rc = igemm_plan_create(p->d, variant, tile_id, split_k, o.s2d, ctx->d_status, &p->ig,
+                               o.math == BODA_MATH_TF32X3 ? 1 : o.math == BODA_MATH_F16 ? 2 : 0, o.max_workspace);
         if (rc == BODA_OK) { p->tile_id = igemm_plan_tile(p->ig); p->ws_bytes = igemm_plan_workspace_bytes(p->ig); }
     }
     if (rc != BODA_OK) { boda_conv_plan_destroy(p); return rc; }
@@ -296,7 +296,7 @@ int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan
     boda_plan_opts o;
     boda_plan_opts_default(&o);
     if (opts) o = *opts;
-    if (o.math < BODA_MATH_AUTO || o.math > BODA_MATH_TF32X3) return BODA_ERR_INVALID_ARG;
+    if (o.math < BODA_MATH_AUTO || o.math > BODA_MATH_F16) return BODA_ERR_INVALID_ARG;
     if (o.variant < BODA_VARIANT_AUTO || o.variant > BODA_VARIANT_TCONV) return BODA_ERR_INVALID_ARG;
 
     std::lock_guard<std::mutex> lock(g_mutex);
@@ -315,8 +315,8 @@ int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan
     int variant = o.variant;
     if (variant == BODA_VARIANT_AUTO) {
         if (o.math == BODA_MATH_FP32) variant = BODA_VARIANT_DIRECT;
-        else if (o.math == BODA_MATH_TF32X3 && d.K >= 16 && (k1_legal || t_legal) && o.s2d <= 0)
-            variant = k1_legal ? BODA_VARIANT_K1CONV : BODA_VARIANT_TCONV;   // FP32-accurate either way: the tensor cores if legal
+        else if ((o.math == BODA_MATH_TF32X3 || o.math == BODA_MATH_F16) && d.K >= 16 && (k1_legal || t_legal) && o.s2d <= 0)
+            variant = k1_legal ? BODA_VARIANT_K1CONV : BODA_VARIANT_TCONV;   // the mode is the caller's choice: the tensor cores if legal
         else if (k1_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_K1CONV;
         else if (t_legal && igemm_variant_profitable(d)) variant = BODA_VARIANT_TCONV;
         else variant = BODA_VARIANT_DIRECT;
@@ -331,7 +331,7 @@ int boda::conv_plan_create_chained(const boda_conv_shape* shape, const boda_plan
         rc = plan_build(*shape, o, ctx, variant, o.tile_id, o.split_k, plan);
         // the workspace limit ruled out every tensor-core tile: the FP32 kernel needs no workspace
         if (rc == BODA_ERR_NOMEM && o.max_workspace > 0 && o.variant == BODA_VARIANT_AUTO && o.tile_id < 0 &&
-            (o.math == BODA_MATH_AUTO || o.math == BODA_MATH_TF32X3))
+            (o.math == BODA_MATH_AUTO || o.math == BODA_MATH_TF32X3 || o.math == BODA_MATH_F16))
             rc = plan_build(*shape, o, ctx, BODA_VARIANT_DIRECT, -1, 0, plan);
     } else {
         // Automated tuning: the rule above names a variant; timing confirms or overturns it.  Every tile and split
@@ -419,7 +419,7 @@ int boda_conv_plan_describe(const boda_conv_plan* p, char* buf, size_t n)
         char tmp[160];
         igemm_plan_describe(p->ig, tmp, sizeof(tmp));
         std::snprintf(buf, n, "variant=%s %s math=%s workspace=%zu", vn[p->variant], tmp,
-                      p->math == BODA_MATH_TF32X3 ? "tf32x3" : "tf32", p->ws_bytes);
+                      p->math == BODA_MATH_TF32X3 ? "tf32x3" : p->math == BODA_MATH_F16 ? "f16" : "tf32", p->ws_bytes);
     }
     return BODA_OK;
 }

@@ -19,6 +19,7 @@
 // Every wait is bounded (4e9 SM cycles, about two seconds): on expiry the kernel records BODA_ERR_DEVICE_TIMEOUT in the
 // status word, all roles leave their loops, tensor memory is released and the CTA returns.
 #include <cuda.h>
+#include <cuda_fp16.h>
 
 #include <algorithm>
 #include <cstdio>
@@ -94,13 +95,17 @@ __device__ __forceinline__ RowDst igemm_row_dst(const IgemmParams& p, int m)
 }
 
 // ------------------------------------------------------------------------------------------------
-// X3: the error-compensated mode (three reduction steps per channel chunk); a compile-time switch because the
-// producers' loops set the pace of the main loop and every instruction in them shows in the layer's time.
-template <int BN, bool X3>
+// MODE 1: the error-compensated mode (three reduction steps per channel chunk).  MODE 2: fp16 operands (a 128-byte
+// row of a stage holds 64 channels, one MMA covers 16 of them; fp32 accumulation all the same).  A compile-time switch
+// because the producers' loops set the pace of the main loop and every instruction in them shows in the layer's time.
+enum { MODE_TF32 = 0, MODE_X3 = 1, MODE_F16 = 2 };
+template <int BN, int MODE>
 __global__ void __launch_bounds__(kIgemmThreads, 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
                   const IgemmParams p)
 {
+    constexpr bool X3 = MODE == MODE_X3;
+    constexpr int CH = MODE == MODE_F16 ? 64 : BKC;      // channels per reduction chunk (128 bytes)
     using Cfg = TileCfg<BN>;
     constexpr int STAGES = Cfg::STAGES;
     extern __shared__ uint8_t smem_raw[];
@@ -163,8 +168,8 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             const int chunk0 = it_begin / terms;
             int term = it_begin - chunk0 * terms;
             int tap = chunk0 / p.cchunks;
-            int cx = (chunk0 - tap * p.cchunks) * BKC;                 // first channel of the chunk
-            const int cend = p.cchunks * BKC;
+            int cx = (chunk0 - tap * p.cchunks) * CH;                  // first channel of the chunk
+            const int cend = p.cchunks * CH;
             uint32_t stage = 0, par = 1;
             // full barrier of local reduction step i: [stage][i & 1] with two issuers, [stage][0] with one
             constexpr uint32_t FLIP = Cfg::ISSUERS == 2 ? 8u : 0u;
@@ -190,7 +195,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     else { fb += 16; eb += 8; dst += A_STAGE_BYTES; }
                     if (!X3 || ++term == terms) {
                         term = 0;
-                        cx += BKC;
+                        cx += CH;
                         if (cx == cend) { cx = 0; if (++s == S) { s = 0; ++r; } }
                     }
                 }
@@ -206,7 +211,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     else { fb += 16; eb += 8; dst += Cfg::B_STAGE_BYTES; }
                     if (!X3 || ++term == terms) {
                         term = 0;
-                        cx += BKC;
+                        cx += CH;
                         if (cx == cend) { cx = 0; ++tap; }
                     }
                 }
@@ -231,7 +236,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             // BN <= 192 - so with two issuers one issues while the other's MMAs run.  Each issuer accumulates into its
             // own TMEM accumulator (columns [0, BN) and [BN, 2*BN)); the epilogue adds the two, so the summation
             // order - and with it every output bit - is the same in every run.
-            constexpr uint32_t idesc = instr_desc_tf32<BN>();
+            constexpr uint32_t idesc = MODE == MODE_F16 ? instr_desc_f16<BN>() : instr_desc_tf32<BN>();
             constexpr int STEP = Cfg::ISSUERS;                          // stages between two steps of one issuer
             // an issuer returns to a barrier after CYCLE of its own steps: then the barrier's phase has advanced
             constexpr int CYCLE = (STEP == 2 && STAGES % 2 == 0) ? STAGES / 2 : STAGES;
@@ -248,8 +253,10 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (!ok) break;
                 tc_fence_after();
 #pragma unroll
-                for (int k = 0; k < BKC / 8; ++k)       // 8 TF32 values = 32 bytes = 2 descriptor units per step
-                    umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
+                for (int k = 0; k < BKC / 8; ++k) {     // 8 TF32 (16 fp16) values = 32 bytes = 2 descriptor units per step
+                    if constexpr (MODE == MODE_F16) umma_f16(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
+                    else umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, k == 0 ? accumulate : 1u);
+                }
                 accumulate = 1u;
                 tc_commit(eb);                          // frees the stage once these MMAs have read it
                 stage += STEP;
@@ -680,7 +687,10 @@ struct IgemmPlan {
     int BN = 128;
     int Cp = 0;
     int terms = 1;                   // 3: error-compensated TF32, staged operands hold hi and lo parts (2*Cp channels)
+    bool half = false;               // fp16 operands: staged tensors hold __half, Cp is a multiple of 64
     int Cs() const { return terms == 3 ? 2 * Cp : Cp; }
+    int esize() const { return half ? 2 : 4; }            // bytes per staged operand element
+    int chunk() const { return half ? 64 : BKC; }         // channels per 128-byte reduction chunk
     int splits = 1;
     int iters_total = 0, iters_per_split = 0;
     int tiles_m = 0, tiles_n = 0;
@@ -976,14 +986,14 @@ int encode_map_a_halo(IgemmPlan* p, const void* xs)
     return BODA_OK;
 }
 
-template <int BN, bool X3>
+template <int BN, int MODE>
 int launch_bn_mode(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 {
     using Cfg = TileCfg<BN>;
     static DeviceSmemLimit limit;
-    BODA_CUDA_TRY(limit.ensure(igemm_tf32_kernel<BN, X3>, Cfg::SMEM_BYTES));
+    BODA_CUDA_TRY(limit.ensure(igemm_tf32_kernel<BN, MODE>, Cfg::SMEM_BYTES));
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
-    BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN, X3>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
+    BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN, MODE>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
                                 p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
@@ -991,20 +1001,22 @@ int launch_bn_mode(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 template <int BN>
 int launch_bn(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
 {
-    return prm.terms == 3 ? launch_bn_mode<BN, true>(p, prm, stream) : launch_bn_mode<BN, false>(p, prm, stream);
+    if (p->half) return launch_bn_mode<BN, MODE_F16>(p, prm, stream);
+    return prm.terms == 3 ? launch_bn_mode<BN, MODE_X3>(p, prm, stream) : launch_bn_mode<BN, MODE_TF32>(p, prm, stream);
 }
 
 int encode_map_a(IgemmPlan* p, const void* xp)
 {
     const ConvDims& d = p->d;
-    const cuuint64_t Cs = (cuuint64_t)p->Cs();
+    const cuuint64_t Cs = (cuuint64_t)p->Cs(), es = (cuuint64_t)p->esize();
+    const CUtensorMapDataType dtype = p->half ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32;
     const cuuint64_t dims[4] = {Cs, (cuuint64_t)d.W, (cuuint64_t)d.H, (cuuint64_t)d.N};
-    const cuuint64_t strides[3] = {Cs * 4, (cuuint64_t)d.W * Cs * 4, (cuuint64_t)d.H * d.W * Cs * 4};
+    const cuuint64_t strides[3] = {Cs * es, (cuuint64_t)d.W * Cs * es, (cuuint64_t)d.H * d.W * Cs * es};
     const int lower[2] = {-d.pad, -d.pad};                                 // W, H
     const int upper[2] = {d.pad - (d.S - 1), d.pad - (d.R - 1)};
     const cuuint32_t estr[4] = {1, (cuuint32_t)d.stride, (cuuint32_t)d.stride, 1};
-    CUresult r = g_encode_im2col(&p->map_a, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 4, const_cast<void*>(xp), dims, strides,
-                                 lower, upper, BKC, BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+    CUresult r = g_encode_im2col(&p->map_a, dtype, 4, const_cast<void*>(xp), dims, strides,
+                                 lower, upper, (cuuint32_t)p->chunk(), BM, estr, CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                  CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
         char msg[96];
@@ -1034,12 +1046,12 @@ int encode_map_b(IgemmPlan* p)
         }
         return BODA_OK;
     }
-    const cuuint64_t Cs = (cuuint64_t)p->Cs();
+    const cuuint64_t Cs = (cuuint64_t)p->Cs(), es = (cuuint64_t)p->esize();
     const cuuint64_t dims[3] = {Cs, (cuuint64_t)d.K, (cuuint64_t)(d.R * d.S)};
-    const cuuint64_t strides[2] = {Cs * 4, (cuuint64_t)d.K * Cs * 4};
-    const cuuint32_t box[3] = {BKC, (cuuint32_t)p->BN, 1};
+    const cuuint64_t strides[2] = {Cs * es, (cuuint64_t)d.K * Cs * es};
+    const cuuint32_t box[3] = {(cuuint32_t)p->chunk(), (cuuint32_t)p->BN, 1};
     const cuuint32_t estr[3] = {1, 1, 1};
-    CUresult r = g_encode_tiled(&p->map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, dims, strides, box, estr,
+    CUresult r = g_encode_tiled(&p->map_b, p->half ? CU_TENSOR_MAP_DATA_TYPE_FLOAT16 : CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, dims, strides, box, estr,
                                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
                                 CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
     if (r != CUDA_SUCCESS) {
@@ -1052,9 +1064,11 @@ int encode_map_b(IgemmPlan* p)
 
 }  // namespace
 
-int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out, bool x3,
+int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out, int mode,
                       size_t max_ws)
 {
+    // mode 1 (error-compensated TF32) and mode 2 (fp16 operands) run on the im2col kernel only, NCHW in and out
+    const bool x3 = mode != 0;
     if (!igemm_variant_legal(d_in, variant)) return BODA_ERR_UNSUPPORTED;
     // strided tconv layers may run as their stride-1 space-to-depth view
     ConvDims d = d_in;
@@ -1093,9 +1107,10 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     }
     p->variant = variant;
     p->d_status = d_status;
-    p->Cp = ((d.C + BKC - 1) / BKC) * BKC;
-    p->terms = x3 ? 3 : 1;
-    p->iters_total = d.R * d.S * (p->Cp / BKC) * p->terms;
+    p->half = mode == 2;
+    p->Cp = ((d.C + p->chunk() - 1) / p->chunk()) * p->chunk();
+    p->terms = mode == 1 ? 3 : 1;
+    p->iters_total = d.R * d.S * (p->Cp / p->chunk()) * p->terms;
     // tile and split: forced, or the minimum of the cost model
     double best = 1e300;
     int best_t = 2, best_s = 1;
@@ -1125,7 +1140,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         if (max_ws > 0) {
             // staged input of this tile's kernel (see xp_bytes below)
             const size_t rows = nacc > 0 ? (size_t)d.N * (d.H + d.pad) * (d.W + d.pad) : (size_t)d.N * d.H * d.W;
-            if (((rows * p->Cs() * 4 + 1023) & ~(size_t)1023) > max_ws) continue;
+            if (((rows * p->Cs() * p->esize() + 1023) & ~(size_t)1023) > max_ws) continue;
         }
         for (int s : kSplitCandidates) {
             if (split_k > 0 && s != split_k) continue;
@@ -1133,7 +1148,7 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
             // the input staging kernel these tiles need and the gather tiles do not: a launch, or the time to read
             // the input and write its staged copy (about 3000 bytes per clock measured on staging kernels)
             const double staging = std::max(6000.0, ((double)d_in.N * d_in.C * d_in.H * d_in.W + (double)d.N * d.H * d.W * p->Cp) * 4.0 / 3000.0);
-            const double c = staging + (nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms, kTileBN[t], s));
+            const double c = staging + (nacc > 0 ? model_cost_halo(d, p->Cp, kTileBN[t], nacc, s) : model_cost(d, p->Cp * p->terms / (p->half ? 2 : 1), kTileBN[t], s));
             if (c < best) { best = c; best_t = t; best_s = s; }
         }
     }
@@ -1206,12 +1221,12 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     } else {
         p->tiles_m = (d.M + BM - 1) / BM;
-        p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cs() * 4) + 1023) & ~(size_t)1023;
+        p->xp_bytes = (((size_t)d.N * d.H * d.W * p->Cs() * p->esize()) + 1023) & ~(size_t)1023;
         p->partial_bytes = 0;   // split partial sums stay in shared memory (cluster reduction)
     }
 
     if (max_ws > 0 && p->xp_bytes > max_ws) { delete p; return BODA_ERR_NOMEM; }
-    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cs() * 4);
+    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cs() * p->esize());
     if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
     rc = encode_map_b(p);
     if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -1228,7 +1243,7 @@ void igemm_plan_destroy(IgemmPlan* p)
 }
 
 int igemm_plan_tile(const IgemmPlan* p) { return p->tile_id; }
-bool igemm_plan_writes_packed(const IgemmPlan* p) { return p->nacc != -2 && p->terms != 3; }
+bool igemm_plan_writes_packed(const IgemmPlan* p) { return p->nacc != -2 && p->terms != 3 && !p->half; }
 int igemm_plan_splits(const IgemmPlan* p) { return p->splits; }
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->partial_bytes; }
 
@@ -1254,10 +1269,52 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
                       p->tile_id, p->slab_rows, p->b_stages, p->splits, p->tiles_m, p->tiles_n, p->splits, pool);
         return;
     }
-    std::snprintf(buf, n, "%s%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->terms == 3 ? "x3 " : "", p->BN, p->tile_id,
+    std::snprintf(buf, n, "%s%stile=igemm_128x%d(id %d) stages=%d split_k=%d grid=%dx%dx%d", view, p->half ? "f16 " : p->terms == 3 ? "x3 " : "", p->BN, p->tile_id,
                   p->BN == 64 ? TileCfg<64>::STAGES : p->BN == 96 ? TileCfg<96>::STAGES : p->BN == 128 ? TileCfg<128>::STAGES
                   : p->BN == 192 ? TileCfg<192>::STAGES : TileCfg<256>::STAGES,
                   p->splits, p->tiles_m, p->tiles_n, p->splits);
+}
+
+// fp16 operand staging (reduced-precision storage, the paper's Section 2 remark on 16-bit storage): the same two
+// re-layouts with the values rounded to fp16 (nearest even) and channels padded to a multiple of 64
+__global__ void __launch_bounds__(256)
+pack_input_nhwc_half_kernel(const float* __restrict__ in, __half* __restrict__ xp, int C, int Cp, int HW)
+{
+    __shared__ float tile[32][33];
+    pdl_launch_dependents();
+    pdl_wait();
+    const int n = blockIdx.z;
+    const int hw0 = blockIdx.x * 32, c0 = blockIdx.y * 32;
+    const int tx = threadIdx.x & 31, ty = threadIdx.x >> 5;
+    const float* src = in + (size_t)n * C * HW;
+    __half* dst = xp + (size_t)n * HW * Cp;
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int c = c0 + ty + 8 * i, hw = hw0 + tx;
+        tile[ty + 8 * i][tx] = (c < C && hw < HW) ? __ldg(src + (size_t)c * HW + hw) : 0.f;
+    }
+    __syncthreads();
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int hw = hw0 + ty + 8 * i, c = c0 + tx;
+        if (hw < HW) dst[(size_t)hw * Cp + c] = __float2half_rn(tile[tx][ty + 8 * i]);
+    }
+}
+
+__global__ void __launch_bounds__(256)
+pack_filters_half_kernel(const float* __restrict__ filt, __half* __restrict__ wp, int K, int C, int Cp, int RS)
+{
+    pdl_launch_dependents();
+    pdl_wait();
+    const long long total = (long long)RS * K * Cp;
+    for (long long idx = (long long)blockIdx.x * blockDim.x + threadIdx.x; idx < total;
+         idx += (long long)gridDim.x * blockDim.x) {
+        const int c = (int)(idx % Cp);
+        const long long t = idx / Cp;
+        const int k = (int)(t % K);
+        const int tap = (int)(t / K);
+        wp[idx] = __float2half_rn(c < C ? __ldg(filt + ((size_t)k * C + c) * RS + tap) : 0.f);
+    }
 }
 
 // 1x1 filters with C a multiple of 4 are already [K][C] rows: the staging is a rounding copy, 16 bytes per thread
@@ -1285,7 +1342,10 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const ConvDims& d = p->d;
     const long long total = (long long)d.R * d.S * d.K * p->Cp;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
-    if (p->nacc == -1) {
+    if (p->half) {
+        BODA_CUDA_TRY(launch_kernel(pack_filters_half_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, reinterpret_cast<__half*>(p->d_wp),
+                                    d.K, d.C, p->Cp, d.R * d.S));
+    } else if (p->nacc == -1) {
         const int Kp = p->gather_chunks * 32;
         const int gblocks = (int)std::min<long long>(((long long)d.K * Kp + 255) / 256, 148 * 8);
         BODA_CUDA_TRY(launch_kernel(pack_filters_flat_kernel, dim3(gblocks), dim3(256), 0, stream, 1, filt, p->d_wp, d.K, d.Kred, Kp));
@@ -1333,7 +1393,7 @@ static OutSpec make_out_spec(const IgemmPlan* p, float* out)
 
 bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 {
-    if (p->s2d || p->terms == 3 || p->nacc < 0) return false;   // space-to-depth staging, the hi/lo operand split and the gather kernel read NCHW only
+    if (p->s2d || p->terms == 3 || p->half || p->nacc < 0) return false;   // space-to-depth staging, the hi/lo split, fp16 operands and the gather kernel read NCHW only
     if (p->nacc > 0) { *Hp = p->Hp; *Wp = p->Wp; } else { *Hp = p->d.H; *Wp = p->d.W; }
     *Cp = p->Cp;
     return true;
@@ -1383,7 +1443,7 @@ void igemm_plan_pooled_dims(const IgemmPlan* p, int* P, int* Q)
 int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int oWp, int oCp)
 {
     if (in_packed && (p->s2d || p->nacc < 0)) return BODA_ERR_UNSUPPORTED;
-    if ((in_packed || out_packed) && p->terms == 3) return BODA_ERR_UNSUPPORTED;
+    if ((in_packed || out_packed) && (p->terms == 3 || p->half)) return BODA_ERR_UNSUPPORTED;
     if (out_packed && p->nacc == -2) return BODA_ERR_UNSUPPORTED;        // that kernel's tiles follow images: NCHW output only
     const int outP = p->pool_rows > 0 ? p->poolP : p->d.P, outQ = p->pool_rows > 0 ? p->poolQ : p->d.Q;
     if (out_packed && (oCp % 32 != 0 || oCp < p->d.K || oHp < outP || oWp < outQ)) return BODA_ERR_INVALID_ARG;
@@ -1497,7 +1557,10 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     if (!p->s2d && !p->in_packed) {
         const int HW = d.H * d.W;
         dim3 grid((HW + 31) / 32, p->Cp / 32, d.N);
-        BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW, p->terms == 3 ? 1 : 0));
+        if (p->half)
+            BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_half_kernel, grid, dim3(256), 0, stream, 1, in, reinterpret_cast<__half*>(xp), d.C, p->Cp, HW));
+        else
+            BODA_CUDA_TRY(launch_kernel(pack_input_nhwc_kernel, grid, dim3(256), 0, stream, 1, in, xp, d.C, p->Cp, HW, p->terms == 3 ? 1 : 0));
         count_launch();
     }
     if (p->map_a_base != xp) {
@@ -1507,7 +1570,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
     IgemmParams prm;
     prm.M = d.M; prm.stride = d.stride; prm.pad = d.pad; prm.S = d.S;
-    prm.cchunks = p->Cp / BKC;
+    prm.cchunks = p->Cp / p->chunk();
     prm.terms = p->terms;
     prm.lo_off = p->Cp;
     prm.iters_total = p->iters_total;

@@ -15,10 +15,11 @@ int igemm_num_split_candidates();
 int igemm_split_candidate(int i);
 
 // s2d: -1 automatic, 0 never, 1 force the space-to-depth view of a strided tconv layer.
-// x3: error-compensated TF32 (three tensor-core products per FP32 product; im2col kernel only, NCHW in and out).
+// mode: 0 TF32; 1 error-compensated TF32 (three tensor-core products per FP32 product); 2 fp16 operands (fp32
+// accumulate).  Modes 1 and 2: im2col kernel only, NCHW in and out.
 // max_ws: 0, or the largest workspace (staged input) the caller accepts; BODA_ERR_NOMEM if no tile fits it.
 int igemm_plan_create(const ConvDims& d, int variant, int tile_id, int split_k, int s2d, int* d_status, IgemmPlan** out,
-                      bool x3 = false, size_t max_ws = 0);
+                      int mode = 0, size_t max_ws = 0);
 bool igemm_s2d_applicable(const ConvDims& d);
 void igemm_plan_destroy(IgemmPlan* p);
 int igemm_plan_tile(const IgemmPlan* p);

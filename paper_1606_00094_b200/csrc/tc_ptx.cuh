@@ -143,6 +143,15 @@ __device__ __forceinline__ void umma_tf32(uint32_t tmem_d, uint64_t desc_a, uint
         "tcgen05.mma.cta_group::1.kind::tf32 [%0], %1, %2, %3, p;\n\t}"
         :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
 }
+// the same with fp16 operands: 128 x N x 16 per instruction
+__device__ __forceinline__ void umma_f16(uint32_t tmem_d, uint64_t desc_a, uint64_t desc_b, uint32_t idesc, uint32_t accumulate)
+{
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::f16 [%0], %1, %2, %3, p;\n\t}"
+        :: "r"(tmem_d), "l"(desc_a), "l"(desc_b), "r"(idesc), "r"(accumulate) : "memory");
+}
 __device__ __forceinline__ void tmem_ld_32cols(uint32_t taddr, uint32_t (&v)[32])
 {
     asm volatile(
@@ -423,7 +432,16 @@ __host__ __device__ constexpr uint32_t instr_desc_tf32()
          | ((uint32_t)(BN >> 3) << 17) // N
          | ((uint32_t)(128 >> 4) << 24);// M = 128
 }
-
+// fp16 operands (kind::f16), fp32 accumulator
+template <int BN>
+__host__ __device__ constexpr uint32_t instr_desc_f16()
+{
+    return (1u << 4)                   // accumulator format: fp32
+         | (0u << 7) | (0u << 10)      // A and B format: fp16
+         | (0u << 15) | (0u << 16)     // A and B are K-major
+         | ((uint32_t)(BN >> 3) << 17) // N
+         | ((uint32_t)(128 >> 4) << 24);// M = 128
+}
 
 }  // namespace tc
 }  // namespace boda
