@@ -224,8 +224,18 @@ def single_layer_configs(B, wl, torch, peaks, flush):
         us_x3 = _graph_us(torch, lambda: plan3(x, w, b, out=y))
         desc_x3 = plan3.describe()
         plan3.close()
+        # and with fp16 operand storage (a precision class of its own: an extra row, never the headline)
+        plan16 = B.ConvPlan(s.as_tuple(), math=B.BODA_MATH_F16, tune=1)
+        plan16.bind_filters(w)
+        for _ in range(3):
+            plan16(x, w, b, out=y)
+        torch.cuda.synchronize()
+        us_f16 = _graph_us(torch, lambda: plan16(x, w, b, out=y))
+        desc_f16 = plan16.describe()
+        plan16.close()
         tf = s.flops / us / 1e6
-        out.append({"config": cid, "us_tf32x3": round(us_x3, 2), "plan_tf32x3": desc_x3, "name": cfg.name, "us_per_call": round(us, 2), "us_l2_cold": round(cold_us, 2),
+        out.append({"config": cid, "us_f16_storage": round(us_f16, 2), "plan_f16_storage": desc_f16,
+                    "us_tf32x3": round(us_x3, 2), "plan_tf32x3": desc_x3, "name": cfg.name, "us_per_call": round(us, 2), "us_l2_cold": round(cold_us, 2),
                     "us_unbound_filters": round(us_unbound, 2), "gflops": round(tf * 1e3, 1),
                     "algorithmic_gbs": round(s.min_bytes / us / 1e3, 1),
                     "frac_of_hbm_peak_l2_cold": round(s.min_bytes / cold_us / 1e3 / peaks["hbm_gbs"], 4),
@@ -270,6 +280,50 @@ def large_batch_rows(B, wl, torch, peaks, flush):
                     "frac_of_hbm_peak": round(nbytes / us / 1e3 / peaks["hbm_gbs"], 4),
                     "frac_of_tf32_peak": round(flops / us / 1e6 / (0.5 * peaks["bf16_tflops"]), 4), "plan": plan.describe()})
         plan.close()
+    return out
+
+
+SWEEP_SHAPES = [
+    # (N, C, H, W, K, R, S, stride, pad): a SYNTHETIC grid over window, stride, channel counts, extent and batch -
+    # not the paper's benchmark list (which it does not print)
+    (1, 3, 224, 224, 64, 7, 7, 2, 3), (5, 3, 227, 227, 96, 11, 11, 4, 0), (20, 3, 64, 64, 16, 5, 5, 1, 2),
+    (5, 16, 56, 56, 64, 3, 3, 1, 1), (20, 64, 56, 56, 64, 1, 1, 1, 0), (1, 64, 56, 56, 256, 1, 1, 1, 0),
+    (5, 96, 27, 27, 256, 5, 5, 1, 2), (20, 96, 27, 27, 256, 5, 5, 1, 2), (1, 256, 13, 13, 384, 3, 3, 1, 1),
+    (5, 256, 13, 13, 384, 3, 3, 1, 1), (20, 384, 13, 13, 256, 3, 3, 1, 1), (5, 384, 6, 6, 384, 3, 3, 1, 1),
+    (20, 256, 28, 28, 96, 3, 3, 2, 1), (5, 64, 28, 28, 96, 7, 7, 2, 3), (20, 16, 32, 32, 16, 3, 3, 1, 1),
+    (1, 96, 6, 6, 16, 1, 1, 1, 0),
+]
+
+
+def synthetic_shape_sweep(B, torch, peaks):
+    """EXTRA, synthetic: per shape the time of the plan the rules pick (no timing at plan time) against the plan the
+    tuner picks after timing every tile, split and variant - the regret of the cost model on shapes it was not fitted
+    to - with GFLOP/s and the two roofline fractions.  L2-warm, 20 launches per captured graph, filters bound."""
+    out = []
+    for (N, C, H, W, K, R, S, st, pad) in SWEEP_SHAPES:
+        shape = (N, C, H, W, K, R, S, st, pad, 1)
+        P, Q = (H + 2 * pad - R) // st + 1, (W + 2 * pad - S) // st + 1
+        x = torch.rand((N, C, H, W), dtype=torch.float32, device="cuda")
+        w = torch.randn((K, C, R, S), dtype=torch.float32, device="cuda") * (2.0 / (C * R * S)) ** 0.5
+        b = torch.zeros((K,), dtype=torch.float32, device="cuda")
+        row = {"shape": "N%d C%d %dx%d K%d %dx%d s%d p%d" % (N, C, H, W, K, R, S, st, pad)}
+        for label, tune in (("rule", 0), ("tuned", 1)):
+            plan = B.ConvPlan(shape, tune=tune)
+            y = torch.empty(plan.out_shape, dtype=torch.float32, device="cuda")
+            plan.bind_filters(w)
+            for _ in range(3):
+                plan(x, w, b, out=y)
+            torch.cuda.synchronize()
+            row["us_" + label] = round(_graph_us(torch, lambda: plan(x, w, b, out=y)), 2)
+            row["plan_" + label] = plan.describe().split(" math=")[0]
+            plan.close()
+        flops = 2.0 * N * K * P * Q * C * R * S
+        nbytes = 4.0 * (N * C * H * W + K * C * R * S + K + N * K * P * Q)
+        best = min(row["us_rule"], row["us_tuned"])
+        row.update({"regret_of_rule": round(row["us_rule"] / best, 3), "gflops": round(flops / best / 1e3, 1),
+                    "frac_of_tf32_peak": round(flops / best / 1e6 / (0.5 * peaks["bf16_tflops"]), 4),
+                    "frac_of_hbm_peak_l2_warm": round(nbytes / best / 1e3 / peaks["hbm_gbs"], 4)})
+        out.append(row)
     return out
 
 
@@ -398,7 +452,11 @@ def run_ours(args):
     # cost nor gaps count), the graph replayed several times between events
     dom_reps = 2 if args.stack_only else 20
     inplace_ms = []
+    descs_all = stack.describe()
     for i in range(n_ops):
+        if "fused into" in descs_all[i]:                # a pool that runs inside the preceding convolution: no launch
+            inplace_ms.append(0.0)
+            continue
         g = torch.cuda.CUDAGraph()
         with torch.cuda.graph(g):
             for _ in range(dom_reps):
@@ -415,7 +473,6 @@ def run_ours(args):
         inplace_ms.append(sum(a.elapsed_time(b) for a, b in evs) / (len(evs) * dom_reps))
         del g
     conv_ops = [i for i, op in enumerate(ops) if op.kind == "conv"]
-    descs_all = stack.describe()
     # the dominant KERNEL: among the conv ops that are a single kernel launch (input already staged, or DIRECT)
     single = [i for i in conv_ops if "in=staged" in descs_all[i] or "variant=direct" in descs_all[i]] or conv_ops
     dom = max(single, key=lambda i: inplace_ms[i])
@@ -461,7 +518,10 @@ def run_ours(args):
                                "inplace_ms": round(inplace_ms[i], 5),
                                "gflops": round(gf, 1), "plan": descs[i]})
             else:
-                layers.append({"op": "pool", "ms": round(layer_ms[i], 5), "inplace_ms": round(inplace_ms[i], 5)})
+                if "fused" in descs[i]:
+                    layers.append({"op": "pool", "fused_into_previous_conv": True, "ms": 0.0, "inplace_ms": 0.0})
+                else:
+                    layers.append({"op": "pool", "ms": round(layer_ms[i], 5), "inplace_ms": round(inplace_ms[i], 5)})
         # dominant kernel: the main kernel of the conv layer that takes the most time in the step (timed above)
         dom_tf = ops[dom].shape.flops / (dom_ms * 1e-3) / 1e12
         tensor_path = "variant=direct" not in descs[dom]
@@ -482,6 +542,7 @@ def run_ours(args):
         per_config = [] if args.stack_only else single_layer_configs(B, wl, torch, peaks, flush)
         sgemm_rows = [] if args.stack_only else sgemm_table1(B, torch, peaks)
         extra_rows = [] if args.stack_only else large_batch_rows(B, wl, torch, peaks, flush)
+        sweep_rows = [] if args.stack_only else synthetic_shape_sweep(B, torch, peaks)
         cpu_v, cpu_t, cpu_threads = time_oracle(BATCH, 2) if not args.no_cpu_baseline else (None, None, 0)
         cpu1_v, cpu1_t, _ = time_oracle_one_thread(2) if not args.no_cpu_baseline else (None, None, 0)
         line = {
@@ -506,6 +567,7 @@ def run_ours(args):
             "single_layer_configs": per_config,
             "sgemm_table1": sgemm_rows,
             "extra_not_baseline_batch256": extra_rows,
+            "extra_synthetic_shape_sweep": sweep_rows,
             "frac_of_tf32_peak_whole_step": round(value / 1e3 / (0.5 * peaks["bf16_tflops"]) / world, 4),
         }
         print(json.dumps(line))
