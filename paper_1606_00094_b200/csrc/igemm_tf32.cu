@@ -912,11 +912,16 @@ bool k1n_legal(const ConvDims& d, int variant, bool x3)
 
 // One kernel, no staging: about 380 clocks per 32-channel step (or the MMAs' 2*BN), 3500 of prologue and tail,
 // 32 per output channel of epilogue; tiles follow images, so an image of HW points costs ceil(HW/128) tiles.
-double model_cost_k1n(const ConvDims& d, int BN, int sm_count)
+double model_cost_k1n(const ConvDims& d, int BN, int sm_count, int splits = 1)
 {
     const long long tiles = (long long)d.N * ((d.H * d.W + BM - 1) / BM) * ((d.K + BN - 1) / BN);
-    const double per_cta = (double)((tiles + sm_count - 1) / sm_count);       // persistent: epilogues hide under the next tile
     const int steps = (d.C + BKC - 1) / BKC;
+    if (splits > 1) {
+        // one tile per CTA, clusters of `splits` CTAs; the sum through remote reads costs about 60 clocks per channel and peer
+        const int ips = (steps + splits - 1) / splits;
+        return wave_count((double)tiles, splits) * (ips * std::max(2.0 * BN, 410.0) + 3500.0 + epilogue_cost(BN, splits, false));
+    }
+    const double per_cta = (double)((tiles + sm_count - 1) / sm_count);       // persistent: epilogues hide under the next tile
     return per_cta * steps * std::max(2.0 * BN, 410.0) + 3500.0 + 32.0 * BN;
 }
 
@@ -948,7 +953,8 @@ int launch_k1n(IgemmPlan* p, const k1n::K1nParams& prm, cudaStream_t stream)
     static DeviceSmemLimit limit;
     BODA_CUDA_TRY(limit.ensure(k1n::k1nchw_tf32_kernel<BN>, C::SMEM_BYTES));
     dim3 grid(std::min(prm.tiles_total, p->sm_count));
-    BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, 1,
+    if (prm.splits > 1) grid = dim3(prm.tiles_total, 1, prm.splits);          // one tile per CTA, a cluster per tile
+    BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, prm.splits,
                                 p->map_a, p->map_b, prm));
     count_launch();
     return BODA_OK;
@@ -1124,9 +1130,13 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         if (tile_id >= 0 && t != tile_id) continue;
         const int nacc = kTileNacc[t];
         if (nacc == -2) {
-            if (!k1n_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) continue;
-            const double c = model_cost_k1n(d_in, kTileBN[t], p->sm_count);
-            if (c < best) { best = c; best_t = t; best_s = 1; }
+            if (!k1n_legal(d_in, variant, x3) || s2d > 0) continue;
+            for (int s : kSplitCandidates) {
+                if (split_k > 0 && s != split_k) continue;
+                if (s > (d_in.C + BKC - 1) / BKC) continue;
+                const double c = model_cost_k1n(d_in, kTileBN[t], p->sm_count, s);
+                if (c < best) { best = c; best_t = t; best_s = s; }
+            }
             continue;
         }
         if (nacc < 0) {
@@ -1160,12 +1170,16 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->nacc = kTileNacc[best_t];
     if (p->nacc == -2) {
         // ---- 1x1 from NCHW: no staged input; filters [K][Cp] as for the im2col kernel
-        if (!k1n_legal(d_in, variant, x3) || s2d > 0 || split_k > 1) { delete p; return BODA_ERR_UNSUPPORTED; }
+        if (!k1n_legal(d_in, variant, x3) || s2d > 0) { delete p; return BODA_ERR_UNSUPPORTED; }
         p->d = d_in;
         p->s2d = false;
         p->Cp = ((d_in.C + BKC - 1) / BKC) * BKC;
-        p->splits = 1;
-        p->iters_total = p->iters_per_split = p->Cp / BKC;
+        p->iters_total = p->Cp / BKC;
+        {
+            const int want = std::max(1, std::min(split_k > 0 ? split_k : best_s, p->iters_total));
+            p->iters_per_split = (p->iters_total + want - 1) / want;
+            p->splits = (p->iters_total + p->iters_per_split - 1) / p->iters_per_split;       // no empty split
+        }
         p->tiles_m = d_in.N * ((d_in.H * d_in.W + BM - 1) / BM);
         p->tiles_n = (d_in.K + p->BN - 1) / p->BN;
         p->xp_bytes = 0;
@@ -1251,9 +1265,10 @@ void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
     const char* view = p->s2d ? "s2d " : "";
     if (p->nacc == -2) {
-        std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=1 grid=%dx1x1 tiles=%d", p->BN, p->tile_id,
-                      p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES,
-                      std::min(p->tiles_m * p->tiles_n, p->sm_count), p->tiles_m * p->tiles_n);
+        std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=%d grid=%dx1x%d tiles=%d", p->BN, p->tile_id,
+                      p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES, p->splits,
+                      p->splits > 1 ? p->tiles_m * p->tiles_n : std::min(p->tiles_m * p->tiles_n, p->sm_count), p->splits,
+                      p->tiles_m * p->tiles_n);
         return;
     }
     if (p->nacc < 0) {
@@ -1481,6 +1496,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         kp.status = p->d_status;
         kp.tx_extra = p->tx_extra;
         kp.b_early = (filt == p->bound_filt) ? 1 : 0;
+        kp.splits = p->splits; kp.chunks_per_split = p->iters_per_split;
         switch (p->BN) {
             case 64: return launch_k1n<64>(p, kp, stream);
             case 128: return launch_k1n<128>(p, kp, stream);

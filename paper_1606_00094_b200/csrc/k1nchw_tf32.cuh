@@ -40,6 +40,9 @@ struct K1nParams {
     int* status;
     int tx_extra;                // test hook: bytes added to the expected size of the first stage of CTA (0, 0)
     int b_early;                 // bound filters: the filter tiles' loads need not wait for the preceding kernel
+    // reduction split over the CTAs of a cluster (grid.z = splits > 1: one tile per CTA, grid.x = tiles_total): CTA z
+    // takes channel chunks [z*chunks_per_split, ...) and the partial sums are added through distributed shared memory
+    int splits, chunks_per_split;
 };
 
 template <int BN> struct Cfg {
@@ -86,7 +89,8 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     const int lane = threadIdx.x & 31;
     // persistent: this CTA walks tiles blockIdx.x, blockIdx.x + gridDim.x, ...; tile = (image, point tile) * tiles_n + channel tile
     const int my_tiles = ((int)blockIdx.x < p.tiles_total) ? (p.tiles_total - 1 - (int)blockIdx.x) / (int)gridDim.x + 1 : 0;
-    const int steps = p.cchunks;
+    const int i_begin = p.splits > 1 ? (int)blockIdx.z * p.chunks_per_split : 0;
+    const int steps = p.splits > 1 ? min(p.cchunks, i_begin + p.chunks_per_split) - i_begin : p.cchunks;
 
     pdl_launch_dependents();
     if (threadIdx.x == 0) {
@@ -131,8 +135,8 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     ok = mbar_wait(empty_bar + 8 * stage, par, &s_abort, p.status, 41);
                     if (!ok) break;
                     const uint32_t dst = smem_a + stage * A_STAGE_BYTES + (uint32_t)half * A_BOX_BYTES;
-                    tma_load_3d(dst, &map_a, full_bar + 8 * stage, hw0 + 32 * half, 32 * i, n);
-                    tma_load_3d(dst + A_BOX_BYTES, &map_a, full_bar + 8 * stage, hw0 + 32 * half + 32, 32 * i, n);
+                    tma_load_3d(dst, &map_a, full_bar + 8 * stage, hw0 + 32 * half, 32 * (i_begin + i), n);
+                    tma_load_3d(dst + A_BOX_BYTES, &map_a, full_bar + 8 * stage, hw0 + 32 * half + 32, 32 * (i_begin + i), n);
                     if (++stage == (uint32_t)kStages) { stage = 0; par ^= 1u; }
                 }
             }
@@ -150,7 +154,7 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
                     if (!ok) break;
                     mbar_expect_tx(full_bar + 8 * stage, bytes);
                     bytes = C::STAGE_BYTES;
-                    tma_load_3d(smem_b + stage * C::B_STAGE_BYTES, &map_b, full_bar + 8 * stage, 32 * i, k0, 0);
+                    tma_load_3d(smem_b + stage * C::B_STAGE_BYTES, &map_b, full_bar + 8 * stage, 32 * (i_begin + i), k0, 0);
                     if (++stage == (uint32_t)kStages) { stage = 0; par ^= 1u; }
                 }
             }
@@ -204,6 +208,18 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
             const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16) + slot * (uint32_t)BN;
             const int hw = hw0 + row;
             const RowDst d = row_dst(p.o, hw < p.HW, n, 0, hw);
+            if (p.splits > 1) {
+                // split reduction, step 1: park the partial accumulator in this CTA's shared memory (the stages are idle:
+                // a split CTA has one tile); the cluster-wide sum follows after the role branches
+#pragma unroll 1
+                for (int c = 0; c < BN / 32; ++c) {
+                    uint32_t v[32];
+                    tmem_ld_32cols(trow + 32 * c, v);
+                    tmem_ld_wait();
+                    stash_row32<BN>(smem_base, row, 32 * c, v);
+                }
+                break;
+            }
 #pragma unroll 1
             for (int c = 0; c < BN / 32; ++c) {
                 uint32_t v[32];
@@ -221,6 +237,17 @@ k1nchw_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_const
     }
     tc_fence_before();
     __syncthreads();
+    if (p.splits > 1) {
+        // step 2: every CTA of the cluster sums its share of the channels over all peers' parked accumulators in rank
+        // order (the result does not depend on which CTA sums), adds the bias, applies ReLU and stores
+        cluster_sync_all();
+        if (warp >= 4 && s_abort == 0) {
+            const int row = (warp & 3) * 32 + lane;
+            const int hw = hw0 + row;
+            cluster_reduce_store<BN>(smem_base, row, cluster_cta_rank(), p.splits, row_dst(p.o, hw < p.HW, n, 0, hw), p.o, k0, s_bias);
+        }
+        cluster_sync_all();          // nobody leaves while a peer may still read its shared memory
+    }
     if (warp == 1) {
         tc_fence_after();
         tmem_dealloc(tmem_acc, tmem_cols);

@@ -275,11 +275,25 @@ K1N_SHAPES = [
 
 @pytest.mark.parametrize("shape", K1N_SHAPES)
 @pytest.mark.parametrize("tile", [20, 21, 22])
-def test_k1conv_from_nchw_exact(shape, tile):
+@pytest.mark.parametrize("split", [0, 2, 4])          # 0: the cost model's choice; otherwise a cluster of that many CTAs per tile
+def test_k1conv_from_nchw_exact(shape, tile, split):
     x, w, b = _int_tensors(shape, 1800)
-    got, desc = run_planned(shape, x, w, b, variant=K1, tile_id=tile)
+    got, desc = run_planned(shape, x, w, b, variant=K1, tile_id=tile, split_k=split)
     assert "k1nchw_128x" in desc and f"id {tile}" in desc
+    if split and shape[1] >= 32 * split:
+        assert f"split_k={split}" in desc
     np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_k1conv_from_nchw_split_runs_twice_bitwise_equal():
+    """The cluster sum adds the partial accumulators in rank order: two runs must agree bit for bit."""
+    shape = (5, 480, 14, 14, 192, 1, 1, 1, 0, 1)
+    x, w, b = _real_tensors(shape, 1850)
+    a, desc = run_planned(shape, x, w, b, variant=K1, tile_id=20, split_k=4)
+    c, _ = run_planned(shape, x, w, b, variant=K1, tile_id=20, split_k=4)
+    assert "split_k=4" in desc
+    np.testing.assert_array_equal(a, c)
+    assert_parity(a, oracle_out(shape, x, w, b), TF32_TOL, desc)
 
 
 def test_k1conv_from_nchw_on_real_values_is_the_choice_for_configuration_3_and_refuses_what_it_cannot_address():
