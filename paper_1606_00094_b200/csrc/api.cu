@@ -430,7 +430,7 @@ int boda_conv_plan_kernels_per_call(const boda_conv_plan* p)
 {
     if (!p) return 0;
     if (p->variant == BODA_VARIANT_DIRECT) return 1;
-    return p->in_packed ? 1 : 2;                           // tensor-core variants: input staging + main kernel
+    return igemm_plan_kernels_per_call(p->ig);             // tensor-core variants: input staging (where needed) + main kernel
 }
 
 int boda_conv_plan_bind_filters(boda_conv_plan* p, const float* filt, void* stream)

@@ -33,6 +33,7 @@
 #include "tconv_halo.cuh"
 #include "gconv_tf32.cuh"
 #include "k1nchw_tf32.cuh"
+#include "tconv_first_layer.cuh"
 
 namespace boda {
 namespace {
@@ -667,9 +668,10 @@ int load_driver_entry_points()
 // with NACC accumulators of 128 rows each (ids 5..8: 1, 9..12: 2, 13..15: 4).
 // accumulators per tile: 0 = im2col kernel, 1 / 2 / 4 = halo kernel, -1 = gather kernel (gconv_tf32.cuh)
 // Ids 20..22: 1x1 layers by TMA straight from NCHW (k1nchw_tf32.cuh), accumulator code -2.
+// Ids 23..25: first-layer kernel (tconv_first_layer.cuh; 3 channels, stride 4, straight from NCHW), accumulator code -3.
 constexpr int kTileBN[] = {64, 96, 128, 192, 256, /*halo*/ 64, 128, 192, 256, 96, 128, 192, 256, 64, 96, 128, /*gather*/ 64, 96, 128, 192,
-                           /*1x1 from NCHW*/ 64, 128, 192};
-constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1, -1, -2, -2, -2};
+                           /*1x1 from NCHW*/ 64, 128, 192, /*first layer*/ 64, 96, 128};
+constexpr int kTileNacc[] = {0, 0, 0, 0, 0, 1, 1, 1, 1, 2, 2, 2, 2, 4, 4, 4, -1, -1, -1, -1, -2, -2, -2, -3, -3, -3};
 constexpr int kFirstK1nTile = 20;
 constexpr int kFirstGatherTile = 16;
 constexpr int kNumIgemmTiles = sizeof(kTileBN) / sizeof(kTileBN[0]);
@@ -715,6 +717,9 @@ struct IgemmPlan {
     // fused 3x3 / stride-2 max-pooling of the output (halo kernel with 2 or 4 accumulators, no split)
     int pool_rows = 0, tiles_per_image = 0, poolP = 0, poolQ = 0;
     int tiles_m_unpooled = 0;
+    // first-layer kernel only (nacc == -3): view taps, tile geometry, second filter map (chunk 1: 16 channels, 64-byte rows)
+    int fl_Rb = 0, fl_Sb = 0, fl_rows_per_tile = 0, fl_raw_rows = 0, fl_raw_buf = 0, fl_slab_rows = 0, fl_tiles_unpooled = 0;
+    CUtensorMap map_b1;
 };
 
 // Geometry of the halo kernel for a shape and tile; false if the shape does not fit it.
@@ -900,6 +905,45 @@ int launch_gather(IgemmPlan* p, const gconv::GconvParams& prm, cudaStream_t stre
     return BODA_OK;
 }
 
+// First-layer kernel: 3 channels, stride 4, no padding, a window of at most 12 x 12 (3 x 3 block taps); tiles of 512
+// flat positions of the space-to-depth view start every 2*pr output rows of an image (pr = pooled rows a tile would own).
+bool first_layer_geometry(const ConvDims& d, int variant, bool restricted, int BN, IgemmPlan* p)
+{
+    if (variant != BODA_VARIANT_TCONV || restricted) return false;
+    if (d.C != first::kChannels || d.stride != first::kStride || d.pad != 0 || d.R * d.S < 2 || d.R > 12 || d.S > 12) return false;
+    const int Rb = (d.R + 3) / 4, Sb = (d.S + 3) / 4;
+    const int Hb = d.P - 1 + Rb, Wb = d.Q - 1 + Sb;
+    const int pr = (512 - d.Q) / (2 * Wb);
+    if (pr < 1 || d.K < 8) return false;
+    const int rows_per_tile = 2 * pr;
+    const int raw_rows = (rows_per_tile + Rb) * 4;
+    const int slab_rows = ((512 + (Rb - 1) * Wb + (Sb - 1)) + 7) & ~7;
+    const long long raw_need = (long long)raw_rows * d.W * 4 + 32;
+    const int raw_buf = (int)((std::max<long long>(raw_need, (long long)slab_rows * 64) + 1023) & ~1023LL);
+    const long long fixed = (long long)slab_rows * 128 + 2LL * raw_buf + 1024 + 512;
+    int b_stages = (int)((232448 - fixed) / (BN * 128));
+    if (b_stages > halo::kMaxBStages) b_stages = halo::kMaxBStages;
+    if (b_stages < 2) return false;
+    if ((long long)d.N * Hb * Wb > 0x3fffffffLL || (long long)d.N * d.C * d.H * d.W > 0x7fffffffLL) return false;
+    if (p) {
+        p->fl_Rb = Rb; p->fl_Sb = Sb; p->Hp = Hb; p->Wp = Wb; p->fl_rows_per_tile = rows_per_tile; p->fl_raw_rows = raw_rows;
+        p->fl_raw_buf = raw_buf; p->fl_slab_rows = slab_rows; p->b_stages = b_stages;
+        p->fl_tiles_unpooled = d.N * ((d.P + rows_per_tile - 1) / rows_per_tile);
+    }
+    return true;
+}
+
+// One kernel, nothing staged: per tap and accumulator 4 + 2 MMAs of about 57 clocks (four issuers keep the pipe busy),
+// about 4000 clocks to fetch the raw rows and build the first slab, 9000 of prologue, tail and epilogue.
+double model_cost_first_layer(const ConvDims& d, int BN, int sm_count)
+{
+    const int Rb = (d.R + 3) / 4, Sb = (d.S + 3) / 4, Wb = d.Q - 1 + Sb;
+    const int pr = std::max(1, (512 - d.Q) / (2 * Wb));
+    const long long tiles = (long long)d.N * ((d.P + 2 * pr - 1) / (2 * pr)) * ((d.K + BN - 1) / BN);
+    const double waves = (double)((tiles + sm_count - 1) / sm_count);
+    return waves * (Rb * Sb * 24.0 * std::max(57.0, 0.6 * BN) + 4000.0 + 9000.0);
+}
+
 // 1x1 from NCHW: stride 1, no padding, rows of HW floats that TMA can address (16-byte multiples), and the staged
 // output layout is not offered (tiles follow images, not the flat output-point index of a consumer's tiles - the
 // stores themselves would work).
@@ -956,6 +1000,19 @@ int launch_k1n(IgemmPlan* p, const k1n::K1nParams& prm, cudaStream_t stream)
     if (prm.splits > 1) grid = dim3(prm.tiles_total, 1, prm.splits);          // one tile per CTA, a cluster per tile
     BODA_CUDA_TRY(launch_kernel(k1n::k1nchw_tf32_kernel<BN>, grid, dim3(k1n::kThreads), (size_t)C::SMEM_BYTES, stream, prm.splits,
                                 p->map_a, p->map_b, prm));
+    count_launch();
+    return BODA_OK;
+}
+
+template <int BN>
+int launch_first_layer(IgemmPlan* p, const first::FirstParams& prm, cudaStream_t stream)
+{
+    const int smem = p->fl_slab_rows * 128 + 2 * p->fl_raw_buf + p->b_stages * BN * 128 + 1024 + 512;
+    static DeviceSmemLimit limit;
+    BODA_CUDA_TRY(limit.ensure(first::tconv_first_layer_kernel<BN>, (size_t)smem));
+    dim3 grid(p->tiles_m, p->tiles_n, 1);
+    BODA_CUDA_TRY(launch_kernel(first::tconv_first_layer_kernel<BN>, grid, dim3(first::kThreads), (size_t)smem, stream, 1,
+                                p->map_b, p->map_b1, prm));
     count_launch();
     return BODA_OK;
 }
@@ -1036,6 +1093,26 @@ int encode_map_a(IgemmPlan* p, const void* xp)
 int encode_map_b(IgemmPlan* p)
 {
     const ConvDims& d = p->d;
+    if (p->nacc == -3) {
+        // filters [Rb*Sb][K][48]: chunk 0 = channels 0..31 as 128-byte rows, chunk 1 = channels 32..47 as 64-byte rows
+        const cuuint64_t fdims[3] = {(cuuint64_t)first::kViewChannels, (cuuint64_t)d.K, (cuuint64_t)(p->fl_Rb * p->fl_Sb)};
+        const cuuint64_t fstrides[2] = {(cuuint64_t)first::kViewChannels * 4, (cuuint64_t)d.K * first::kViewChannels * 4};
+        const cuuint32_t festr[3] = {1, 1, 1};
+        const cuuint32_t box0[3] = {32, (cuuint32_t)p->BN, 1}, box1[3] = {16, (cuuint32_t)p->BN, 1};
+        CUresult fr = g_encode_tiled(&p->map_b, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, fdims, fstrides, box0, festr,
+                                     CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                     CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (fr == CUDA_SUCCESS)
+            fr = g_encode_tiled(&p->map_b1, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 3, p->d_wp, fdims, fstrides, box1, festr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_64B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+        if (fr != CUDA_SUCCESS) {
+            char msg[96];
+            std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (first-layer filters) failed with CUresult %d", (int)fr);
+            return record_cuda_error(cudaErrorInvalidValue, msg);
+        }
+        return BODA_OK;
+    }
     if (p->nacc == -1) {
         const cuuint64_t Kp = (cuuint64_t)p->gather_chunks * 32;
         const cuuint64_t gdims[2] = {Kp, (cuuint64_t)d.K};
@@ -1129,6 +1206,12 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     for (int t = 0; t < kNumIgemmTiles; ++t) {
         if (tile_id >= 0 && t != tile_id) continue;
         const int nacc = kTileNacc[t];
+        if (nacc == -3) {
+            if (s2d == 0 || split_k > 1 || !first_layer_geometry(d_in, variant, x3, kTileBN[t], nullptr)) continue;
+            const double c = model_cost_first_layer(d_in, kTileBN[t], p->sm_count);
+            if (c < best) { best = c; best_t = t; best_s = 1; }
+            continue;
+        }
         if (nacc == -2) {
             if (!k1n_legal(d_in, variant, x3) || s2d > 0) continue;
             for (int s : kSplitCandidates) {
@@ -1168,6 +1251,25 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     p->tile_id = best_t;
     p->BN = kTileBN[best_t];
     p->nacc = kTileNacc[best_t];
+    if (p->nacc == -3) {
+        // ---- first-layer kernel: no staged input; filters [Rb*Sb][K][48]
+        p->d = d_in;
+        p->s2d = false;
+        if (s2d == 0 || split_k > 1 || !first_layer_geometry(d_in, variant, x3, p->BN, p)) { delete p; return BODA_ERR_UNSUPPORTED; }
+        p->Cp = 64;
+        p->splits = 1;
+        p->iters_total = p->iters_per_split = 2 * p->fl_Rb * p->fl_Sb;
+        p->tiles_m = p->fl_tiles_unpooled;
+        p->tiles_n = (d_in.K + p->BN - 1) / p->BN;
+        p->xp_bytes = 0;
+        p->partial_bytes = 0;
+        cudaError_t fe = cudaMalloc(&p->d_wp, (size_t)p->fl_Rb * p->fl_Sb * d_in.K * first::kViewChannels * 4);
+        if (fe != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(fe, "plan allocation"); }
+        rc = encode_map_b(p);
+        if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
+        *out = p;
+        return BODA_OK;
+    }
     if (p->nacc == -2) {
         // ---- 1x1 from NCHW: no staged input; filters [K][Cp] as for the im2col kernel
         if (!k1n_legal(d_in, variant, x3) || s2d > 0) { delete p; return BODA_ERR_UNSUPPORTED; }
@@ -1258,12 +1360,20 @@ void igemm_plan_destroy(IgemmPlan* p)
 
 int igemm_plan_tile(const IgemmPlan* p) { return p->tile_id; }
 bool igemm_plan_writes_packed(const IgemmPlan* p) { return p->nacc != -2 && p->terms != 3 && !p->half; }
+int igemm_plan_kernels_per_call(const IgemmPlan* p) { return (p->nacc < 0 || p->in_packed) ? 1 : 2; }
 int igemm_plan_splits(const IgemmPlan* p) { return p->splits; }
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p) { return p->xp_bytes + p->partial_bytes; }
 
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n)
 {
     const char* view = p->s2d ? "s2d " : "";
+    if (p->nacc == -3) {
+        char pool[48] = "";
+        if (p->pool_rows > 0) std::snprintf(pool, sizeof(pool), " +maxpool3x3s2(%d rows/tile)", p->pool_rows);
+        std::snprintf(buf, n, "s2d tile=first_512x%d(id %d) taps=%dx%d rows/tile=%d stages=%d split_k=1 grid=%dx%dx1%s", p->BN, p->tile_id,
+                      p->fl_Rb, p->fl_Sb, p->fl_rows_per_tile, p->b_stages, p->tiles_m, p->tiles_n, pool);
+        return;
+    }
     if (p->nacc == -2) {
         std::snprintf(buf, n, "tile=k1nchw_128x%d(id %d) stages=%d split_k=%d grid=%dx1x%d tiles=%d", p->BN, p->tile_id,
                       p->BN == 64 ? k1n::Cfg<64>::STAGES : p->BN == 128 ? k1n::Cfg<128>::STAGES : k1n::Cfg<192>::STAGES, p->splits,
@@ -1357,7 +1467,11 @@ static int pack_filters(IgemmPlan* p, const float* filt, cudaStream_t stream)
     const ConvDims& d = p->d;
     const long long total = (long long)d.R * d.S * d.K * p->Cp;
     const int blocks = (int)std::min<long long>((total + 255) / 256, 148 * 8);
-    if (p->half) {
+    if (p->nacc == -3) {
+        const int fblocks = std::min((p->fl_Rb * p->fl_Sb * d.K * first::kViewChannels + 255) / 256, 148 * 8);
+        BODA_CUDA_TRY(launch_kernel(first::pack_filters_first_layer_kernel, dim3(fblocks), dim3(256), 0, stream, 1, filt, p->d_wp,
+                                    d.K, d.R, d.S, p->fl_Rb, p->fl_Sb));
+    } else if (p->half) {
         BODA_CUDA_TRY(launch_kernel(pack_filters_half_kernel, dim3(blocks), dim3(256), 0, stream, 1, filt, reinterpret_cast<__half*>(p->d_wp),
                                     d.K, d.C, p->Cp, d.R * d.S));
     } else if (p->nacc == -1) {
@@ -1420,6 +1534,13 @@ bool igemm_plan_input_geometry(const IgemmPlan* p, int* Hp, int* Wp, int* Cp)
 static int halo_pool_rows(const IgemmPlan* p, int ksz, int stride)
 {
     const ConvDims& d = p->d;
+    if (p->nacc == -3) {
+        // the first-layer kernel's tiles are row-aligned already: a tile owns rows_per_tile / 2 pooled rows
+        if (ksz != 3 || stride != 2 || d.P < 3 || d.Q < 3) return 0;
+        const int rows = p->fl_rows_per_tile / 2, poolQ = (d.Q - 3) / 2 + 1;
+        const long long region = (long long)p->fl_slab_rows * 128 + 2LL * p->fl_raw_buf + (long long)p->b_stages * p->BN * 128;
+        return 2LL * 4 * 128 * 128 + (long long)rows * poolQ * p->BN * 4 <= region ? rows : 0;
+    }
     if (p->nacc != 2 && p->nacc != 4) return 0;
     if (p->splits != 1 || ksz != 3 || stride != 2 || d.P < 3 || d.Q < 3) return 0;
     const int poolP = (d.P - 3) / 2 + 1, poolQ = (d.Q - 3) / 2 + 1;
@@ -1435,7 +1556,7 @@ bool igemm_plan_can_fuse_pool(const IgemmPlan* p, int ksz, int stride) { return 
 int igemm_plan_set_pool(IgemmPlan* p, int ksz, int stride)
 {
     if (ksz == 0) {                       // back to the unfused form
-        if (p->pool_rows > 0) p->tiles_m = p->tiles_m_unpooled;
+        if (p->pool_rows > 0) p->tiles_m = p->nacc == -3 ? p->fl_tiles_unpooled : p->tiles_m_unpooled;
         p->pool_rows = p->tiles_per_image = p->poolP = p->poolQ = 0;
         return BODA_OK;
     }
@@ -1480,6 +1601,28 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         if (!filt) return BODA_ERR_INVALID_ARG;
         int rc = pack_filters(p, filt, stream);       // unbound: re-layout on every call
         if (rc != BODA_OK) return rc;
+    }
+    if (p->nacc == -3) {
+        if (((uintptr_t)in & 15) != 0) return BODA_ERR_INVALID_ARG;       // bulk copies start on 16-byte boundaries
+        if (after_staging) BODA_CUDA_TRY(cudaEventRecord(after_staging, stream));
+        first::FirstParams fp;
+        fp.h.Mflat = d.N * p->Hp * p->Wp; fp.h.HpWp = p->Hp * p->Wp; fp.h.Wp = p->Wp;
+        fp.h.S = p->fl_Sb; fp.h.taps = p->fl_Rb * p->fl_Sb; fp.h.cchunks = 2; fp.h.lead = 0;
+        fp.h.nbox = 0; fp.h.box_rows = 0; fp.h.a_slot_bytes = 0; fp.h.b_stages = p->b_stages;
+        fp.h.iters_total = fp.h.iters_per_split = p->iters_total; fp.h.splits = 1;
+        fp.h.bias = bias; fp.h.o = make_out_spec(p, out); fp.h.status = p->d_status; fp.h.tx_extra = p->tx_extra;
+        fp.h.pool_rows = p->pool_rows; fp.h.tiles_per_image = p->tiles_m / d.N;
+        fp.h.tile_positions = p->fl_rows_per_tile * p->Wp;
+        fp.in = in; fp.H = d.H; fp.W = d.W;
+        fp.rows_per_tile = p->fl_rows_per_tile; fp.raw_rows = p->fl_raw_rows; fp.raw_buf_bytes = p->fl_raw_buf;
+        fp.slab_rows = p->fl_slab_rows; fp.b_stages = p->b_stages;
+        fp.in_floats = (long long)d.N * d.C * d.H * d.W;
+        switch (p->BN) {
+            case 64: return launch_first_layer<64>(p, fp, stream);
+            case 96: return launch_first_layer<96>(p, fp, stream);
+            case 128: return launch_first_layer<128>(p, fp, stream);
+            default: return BODA_ERR_UNSUPPORTED;
+        }
     }
     if (p->nacc == -2) {
         if (p->map_a_base != in) {
@@ -1554,7 +1697,7 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         hp.iters_total = p->iters_total; hp.iters_per_split = p->iters_per_split; hp.splits = p->splits;
         hp.bias = bias; hp.o = make_out_spec(p, out); hp.tx_extra = p->tx_extra;
         hp.status = p->d_status;
-        hp.pool_rows = p->pool_rows; hp.tiles_per_image = p->tiles_per_image;
+        hp.pool_rows = p->pool_rows; hp.tiles_per_image = p->tiles_per_image; hp.tile_positions = 128 * p->nacc;
         switch (p->BN * 10 + p->nacc) {
             case 641: return launch_halo<64, 1>(p, hp, stream);
             case 1281: return launch_halo<128, 1>(p, hp, stream);

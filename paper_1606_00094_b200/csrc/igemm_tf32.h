@@ -24,6 +24,7 @@ bool igemm_s2d_applicable(const ConvDims& d);
 void igemm_plan_destroy(IgemmPlan* p);
 int igemm_plan_tile(const IgemmPlan* p);
 bool igemm_plan_writes_packed(const IgemmPlan* p);       // can the plan write a consumer's staged layout?
+int igemm_plan_kernels_per_call(const IgemmPlan* p);     // 1, or 2 where an input staging kernel runs first
 int igemm_plan_splits(const IgemmPlan* p);
 size_t igemm_plan_workspace_bytes(const IgemmPlan* p);
 void igemm_plan_describe(const IgemmPlan* p, char* buf, size_t n);

@@ -417,7 +417,8 @@ int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, vo
 {
     if (!s || !in_host || !out_host) return BODA_ERR_INVALID_ARG;
     cudaStream_t st = (cudaStream_t)stream;
-    if (!s->staging_in) BODA_CUDA_TRY(cudaMalloc(&s->staging_in, s->in_elems * sizeof(float)));
+    // slices of the batch start on 256-byte boundaries of the staging buffer (kernels want 16-byte aligned tensors)
+    if (!s->staging_in) BODA_CUDA_TRY(cudaMalloc(&s->staging_in, (s->in_elems + 64 * 8) * sizeof(float)));
     if (!s->staging_out) BODA_CUDA_TRY(cudaMalloc(&s->staging_out, s->out_elems * sizeof(float)));
     if (s->host_chunks == 0) prepare_host_slices(s);
     if (s->host_chunks > 1) {
@@ -433,6 +434,7 @@ int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, vo
         }
         const int k = s->host_chunks;
         const size_t in_chunk = s->in_elems / k, out_chunk = s->out_elems / k;
+        const size_t in_pitch = (in_chunk + 63) & ~(size_t)63;            // floats between slice starts in the staging buffer
         // The call is ordered on `stream`: the slices are copied on a second stream, which first waits for everything
         // the caller has queued on `stream` so far (a kernel or copy that fills in_host, for instance).
         BODA_CUDA_TRY(cudaEventRecord(s->entry_event, st));
@@ -441,13 +443,13 @@ int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, vo
         int rc = BODA_OK;
         cudaError_t ce = cudaSuccess;
         for (int i = 0; i < k && ce == cudaSuccess; ++i) {
-            ce = cudaMemcpyAsync(s->staging_in + i * in_chunk, in_host + i * in_chunk, in_chunk * sizeof(float),
+            ce = cudaMemcpyAsync(s->staging_in + i * in_pitch, in_host + i * in_chunk, in_chunk * sizeof(float),
                                  cudaMemcpyHostToDevice, s->copy_stream);
             if (ce == cudaSuccess) ce = cudaEventRecord(s->chunk_events[i], s->copy_stream);
         }
         for (int i = 0; i < k && ce == cudaSuccess && rc == BODA_OK; ++i) {
             ce = cudaStreamWaitEvent(st, s->chunk_events[i], 0);
-            if (ce == cudaSuccess) rc = boda_stack_fwd(s->sub, s->staging_in + i * in_chunk, s->staging_out + i * out_chunk, stream);
+            if (ce == cudaSuccess) rc = boda_stack_fwd(s->sub, s->staging_in + i * in_pitch, s->staging_out + i * out_chunk, stream);
         }
         if (ce == cudaSuccess && rc == BODA_OK)
             ce = cudaMemcpyAsync(out_host, s->staging_out, s->out_elems * sizeof(float), cudaMemcpyDeviceToHost, st);

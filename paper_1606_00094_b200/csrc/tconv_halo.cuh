@@ -50,12 +50,15 @@ struct HaloParams {
     // pool_rows pooled rows they contain; `o` describes the POOLED tensor (o.P, o.Q = pooled extent)
     int pool_rows;
     int tiles_per_image;
+    // flat positions of a tile whose outputs the tile owns (128*NACC for the contiguous tiles of this kernel; fewer
+    // for the row-aligned tiles of the first-layer kernel, whose last rows belong to the next tile)
+    int tile_positions;
 };
 
 // output location of flat position f = (n*Hp + p)*Wp + q; positions with p >= P or q >= Q are dropped
-__device__ __forceinline__ RowDst halo_row_dst(const HaloParams& p, int f)
+__device__ __forceinline__ RowDst halo_row_dst(const HaloParams& p, int f, int f0)
 {
-    bool valid = f < p.Mflat;
+    bool valid = f < p.Mflat && f - f0 < p.tile_positions;
     int n = 0, pp = 0, qq = 0;
     if (valid) {
         n = f / p.HpWp;
@@ -163,6 +166,74 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
         }
         bulk_commit();
         bulk_wait_all();
+    }
+}
+
+// ---- the epilogue of the 8 epilogue warps (2..5 and 7..10) of a CTA that owns NACC accumulators of 128 flat
+// positions x BN channels: bias, ReLU, then either the fused pooling above or the plain store (NCHW, or the staged
+// layout through bulk copies).  `region_bytes`: shared memory from smem_base that the idle operand buffers leave free.
+template <int BN, int NACC>
+__device__ __forceinline__ void halo_epilogue(const HaloParams& p, uint32_t smem_base, uint32_t region_bytes, uint32_t tmem_acc,
+                                              float* s_bias, volatile int* s_abort, uint32_t accum_bar, int f0, int k0,
+                                              int warp, int lane)
+{
+    // ---------------- epilogue: 8 warps.  Warp w may read TMEM lanes 32*(w%4) .. +31 only, so warps 2..5 and
+    // 7..10 pair up on the same 32 rows: with several accumulators the two groups take alternate accumulators,
+    // with one they take the two halves of its columns.
+    const int quarter = warp & 3;
+    const int group = warp >= 7 ? 1 : 0;
+    const int row = quarter * 32 + lane;
+    const int etid = threadIdx.x - (group ? 96 : 64);                  // 0 .. 255 over the epilogue threads
+    for (int j = etid; j < BN; j += 256)
+        s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
+    if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, s_abort, p.status, 16);   // one poller per warp
+    __syncwarp();
+    asm volatile("bar.sync 1, 256;" ::: "memory");
+    const bool ok = (*s_abort == 0);
+    tc_fence_after();
+    const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    if (ok && p.pool_rows > 0) {
+        if constexpr (NACC >= 2) halo_pooled_epilogue<BN, NACC>(p, smem_base, tmem_acc, s_bias, k0, group, quarter, lane, etid);
+    } else if (ok && p.splits == 1) {
+        constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
+        const int c_begin = (NACC == 1 && group) ? HALF : 0, c_end = (NACC == 1 && !group) ? HALF : NCH;
+        // Staged layout: rows go through shared memory (the operand buffers are idle now) and leave as bulk
+        // copies; every thread owns the same row slot of each of the `nbuf` tile buffers that fit, so only its
+        // own earlier copy has to have been read before it overwrites a slot.
+        constexpr uint32_t TILE_BYTES = 128u * out_tile_row_bytes<BN>();
+        const int nbuf = (int)(region_bytes / TILE_BYTES);
+        const bool bulk = p.o.packed && nbuf >= (NACC == 1 ? 1 : 2);      // with several accumulators: a buffer per group
+        // Which accumulator and which tile buffer a group takes on its turn.  One accumulator: both groups share
+        // it (column halves) and buffer 0.  Two: one each.  Four: with three buffers group 0 takes accumulators
+        // 0 and 3 through buffer 0 and group 1 takes 1 and 2 through buffers 1 and 2, so that only one of the four
+        // tiles waits for an earlier copy to leave its buffer; with two buffers each group reuses its own.
+        const bool three = NACC == 4 && nbuf >= 3;
+        constexpr int TURNS = NACC == 1 ? 1 : NACC / 2;
+#pragma unroll 1
+        for (int turn = 0; turn < TURNS; ++turn) {
+            const int acc = NACC == 1 ? 0 : !three ? group + 2 * turn : group == 0 ? 3 * turn : 1 + turn;
+            const int buf = NACC == 1 ? 0 : !three ? group : group == 0 ? 0 : 1 + turn;
+            const bool reuse = turn > 0 && !(three && group == 1);
+            const RowDst d = halo_row_dst(p, f0 + acc * 128 + row, f0);
+            const uint32_t row_addr = smem_base + (uint32_t)buf * TILE_BYTES + (uint32_t)row * out_tile_row_bytes<BN>();
+            if (bulk && reuse) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
+#pragma unroll 1
+            for (int c = c_begin; c < c_end; ++c) {
+                uint32_t v[32];
+                tmem_ld_32cols(trow + acc * BN + 32 * c, v);
+                tmem_ld_wait();
+                float y[32];
+                bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
+                if (bulk) out_tile_put32(row_addr, 32 * c, y);
+                else store_row32(p.o, d, k0 + 32 * c, y);
+            }
+            if (bulk) {
+                fence_proxy_async_smem();
+                out_tile_store_row(p.o, d, k0 + 32 * c_begin, 32 * (c_end - c_begin), row_addr + 128u * (uint32_t)c_begin);
+                bulk_commit();
+            }
+        }
+        if (bulk) bulk_wait_all();
     }
 }
 
@@ -310,64 +381,8 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 15);
         }
     } else {
-        // ---------------- epilogue: 8 warps.  Warp w may read TMEM lanes 32*(w%4) .. +31 only, so warps 2..5 and
-        // 7..10 pair up on the same 32 rows: with several accumulators the two groups take alternate accumulators,
-        // with one they take the two halves of its columns.
-        const int quarter = warp & 3;
-        const int group = warp >= 7 ? 1 : 0;
-        const int row = quarter * 32 + lane;
-        const int etid = threadIdx.x - (group ? 96 : 64);                  // 0 .. 255 over the epilogue threads
-        for (int j = etid; j < BN; j += 256)
-            s_bias[j] = (p.bias && k0 + j < p.o.K) ? __ldg(p.bias + k0 + j) : 0.f;
-        if (lane == 0) (void)mbar_wait_relaxed(accum_bar, 0, &s_abort, p.status, 16);   // one poller per warp
-        __syncwarp();
-        asm volatile("bar.sync 1, 256;" ::: "memory");
-        const bool ok = (s_abort == 0);
-        tc_fence_after();
-        const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
-        if (ok && p.pool_rows > 0) {
-            if constexpr (NACC >= 2) halo_pooled_epilogue<BN, NACC>(p, smem_base, tmem_acc, s_bias, k0, group, quarter, lane, etid);
-        } else if (ok && p.splits == 1) {
-            constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
-            const int c_begin = (NACC == 1 && group) ? HALF : 0, c_end = (NACC == 1 && !group) ? HALF : NCH;
-            // Staged layout: rows go through shared memory (the operand buffers are idle now) and leave as bulk
-            // copies; every thread owns the same row slot of each of the `nbuf` tile buffers that fit, so only its
-            // own earlier copy has to have been read before it overwrites a slot.
-            constexpr uint32_t TILE_BYTES = 128u * out_tile_row_bytes<BN>();
-            const int nbuf = (int)((uint32_t)(kASlots * p.a_slot_bytes + p.b_stages * Cfg::B_STAGE_BYTES) / TILE_BYTES);
-            const bool bulk = p.o.packed && nbuf >= (NACC == 1 ? 1 : 2);      // with several accumulators: a buffer per group
-            // Which accumulator and which tile buffer a group takes on its turn.  One accumulator: both groups share
-            // it (column halves) and buffer 0.  Two: one each.  Four: with three buffers group 0 takes accumulators
-            // 0 and 3 through buffer 0 and group 1 takes 1 and 2 through buffers 1 and 2, so that only one of the four
-            // tiles waits for an earlier copy to leave its buffer; with two buffers each group reuses its own.
-            const bool three = NACC == 4 && nbuf >= 3;
-            constexpr int TURNS = NACC == 1 ? 1 : NACC / 2;
-#pragma unroll 1
-            for (int turn = 0; turn < TURNS; ++turn) {
-                const int acc = NACC == 1 ? 0 : !three ? group + 2 * turn : group == 0 ? 3 * turn : 1 + turn;
-                const int buf = NACC == 1 ? 0 : !three ? group : group == 0 ? 0 : 1 + turn;
-                const bool reuse = turn > 0 && !(three && group == 1);
-                const RowDst d = halo_row_dst(p, f0 + acc * 128 + row);
-                const uint32_t row_addr = smem_base + (uint32_t)buf * TILE_BYTES + (uint32_t)row * out_tile_row_bytes<BN>();
-                if (bulk && reuse) asm volatile("cp.async.bulk.wait_group.read 0;" ::: "memory");
-#pragma unroll 1
-                for (int c = c_begin; c < c_end; ++c) {
-                    uint32_t v[32];
-                    tmem_ld_32cols(trow + acc * BN + 32 * c, v);
-                    tmem_ld_wait();
-                    float y[32];
-                    bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
-                    if (bulk) out_tile_put32(row_addr, 32 * c, y);
-                    else store_row32(p.o, d, k0 + 32 * c, y);
-                }
-                if (bulk) {
-                    fence_proxy_async_smem();
-                    out_tile_store_row(p.o, d, k0 + 32 * c_begin, 32 * (c_end - c_begin), row_addr + 128u * (uint32_t)c_begin);
-                    bulk_commit();
-                }
-            }
-            if (bulk) bulk_wait_all();
-        }
+        halo_epilogue<BN, NACC>(p, smem_base, (uint32_t)(kASlots * p.a_slot_bytes + p.b_stages * Cfg::B_STAGE_BYTES), tmem_acc,
+                                s_bias, &s_abort, accum_bar, f0, k0, warp, lane);
         tc_fence_before();
     }
     __syncthreads();
@@ -395,7 +410,7 @@ tconv_halo_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
             cluster_sync_all();
             if (warp >= 2 && warp <= 5 && ok)
-                cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row), p.o, k0, s_bias);
+                cluster_reduce_store<BN>(smem_base, row, rank, p.splits, halo_row_dst(p, f0 + acc * 128 + row, f0), p.o, k0, s_bias);
             cluster_sync_all();      // peers are done with this CTA's shared memory
         }
     }

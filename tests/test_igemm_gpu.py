@@ -169,6 +169,44 @@ def test_space_to_depth_exact(shape, tile):
     np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
 
 
+# ---- the first-layer kernel (tiles 23..25): 3 channels, stride 4, no padding, read straight from NCHW by bulk copies
+# and re-laid-out in shared memory (second channel chunk as 64-byte rows)
+FIRST_SHAPES = [
+    (1, 3, 227, 227, 96, 11, 11, 4, 0, 1),       # configuration 2: the tensor's last floats are not a whole 16-byte piece
+    (3, 3, 227, 227, 96, 11, 11, 4, 0, 1),       # images start at odd float offsets
+    (2, 3, 67, 67, 80, 11, 11, 4, 0, 0),         # one tile per image, K ragged against every tile, no ReLU
+    (4, 3, 99, 83, 40, 9, 11, 4, 0, 1),          # R != S, non-square image, several tiles per image
+    (2, 3, 61, 50, 24, 7, 5, 4, 0, 1),           # 2 x 2 block taps
+    (5, 3, 35, 35, 16, 8, 8, 4, 0, 1),           # window a multiple of the stride; tiny output (7 x 7)
+    (1, 3, 131, 259, 32, 11, 11, 4, 0, 1),       # wide rows
+]
+
+
+@pytest.mark.parametrize("shape", FIRST_SHAPES)
+@pytest.mark.parametrize("tile", [23, 24, 25])
+def test_first_layer_kernel_exact(shape, tile):
+    x, w, b = _int_tensors(shape, 1350)
+    got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=tile)
+    assert "first_512x" in desc and f"id {tile}" in desc
+    np.testing.assert_array_equal(got.astype(np.float64), oracle_out(shape, x, w, b), err_msg=desc)
+
+
+def test_first_layer_kernel_real_values_bound_filters_and_refusals():
+    from paper_1606_00094_b200 import binding as B
+    shape = (2, 3, 227, 227, 96, 11, 11, 4, 0, 1)
+    x, w, b = _real_tensors(shape, 1360)
+    ref = oracle_out(shape, x, w, b)
+    for bind in (False, True):
+        got, desc = run_planned(shape, x, w, b, variant=TC, tile_id=24, bind=bind)
+        assert_parity(got, ref, TF32_TOL, desc)
+    for bad in [(2, 4, 67, 67, 32, 11, 11, 4, 0, 1),      # 4 channels
+                (2, 3, 67, 67, 32, 11, 11, 2, 0, 1),      # stride 2
+                (2, 3, 67, 67, 32, 11, 11, 4, 1, 1),      # padding
+                (2, 3, 67, 67, 32, 13, 13, 4, 0, 1)]:     # 4 x 4 block taps
+        with pytest.raises(B.BodaError):
+            B.ConvPlan(bad, variant=TC, tile_id=24)
+
+
 def test_space_to_depth_off_and_auto_agree_with_oracle():
     shape = (2, 3, 99, 99, 96, 11, 11, 4, 0, 1)
     x, w, b = _real_tensors(shape, 1400)

@@ -147,7 +147,11 @@ def test_fused_pool_epilogue_is_exact(prod, cons):
 
 # a first layer on 3 channels with a strided window through its space-to-depth view (NCHW in, halo tile, staged
 # out), pooled, then a 5x5 layer: the shape of the AlexNet-shaped stack's first three ops, small
-@pytest.mark.parametrize("first,second", [((HALO_512x96, 1), (IM2COL_128, 1)), ((HALO_256x96, 1), (HALO_128x128, 1))])
+FIRST_512x64, FIRST_512x96 = 23, 24       # the first-layer kernel: no staged input at all
+
+
+@pytest.mark.parametrize("first,second", [((HALO_512x96, 1), (IM2COL_128, 1)), ((HALO_256x96, 1), (HALO_128x128, 1)),
+                                          ((FIRST_512x96, 1), (IM2COL_128, 1)), ((FIRST_512x64, 1), (HALO_128x128, 1))])
 def test_space_to_depth_first_layer_pool_conv_is_exact(first, second):
     ops = [StackOp("conv", ConvShape(2, 3, 67, 67, 80, 11, 11, 4, 0, True)),           # -> 15 x 15
            StackOp("pool"),                                                            # -> 7 x 7
