@@ -1539,7 +1539,7 @@ static int halo_pool_rows(const IgemmPlan* p, int ksz, int stride)
         if (ksz != 3 || stride != 2 || d.P < 3 || d.Q < 3) return 0;
         const int rows = p->fl_rows_per_tile / 2, poolQ = (d.Q - 3) / 2 + 1;
         const long long region = (long long)p->fl_slab_rows * 128 + 2LL * p->fl_raw_buf + (long long)p->b_stages * p->BN * 128;
-        return 2LL * 4 * 128 * 128 + (long long)rows * poolQ * p->BN * 4 <= region ? rows : 0;
+        return halo::pooled_epilogue_bytes(4, rows * poolQ, p->BN) <= region ? rows : 0;
     }
     if (p->nacc != 2 && p->nacc != 4) return 0;
     if (p->splits != 1 || ksz != 3 || stride != 2 || d.P < 3 || d.Q < 3) return 0;
@@ -1547,7 +1547,7 @@ static int halo_pool_rows(const IgemmPlan* p, int ksz, int stride)
     int rows = (128 * p->nacc - d.Q) / (2 * p->Wp);
     if (rows > poolP) rows = poolP;
     const long long region = (long long)halo::kASlots * p->a_slot_bytes + (long long)p->b_stages * p->BN * 128;
-    while (rows >= 1 && 2LL * p->nacc * 128 * 128 + (long long)rows * poolQ * p->BN * 4 > region) --rows;
+    while (rows >= 1 && halo::pooled_epilogue_bytes(p->nacc, rows * poolQ, p->BN) > region) --rows;
     return rows < 1 ? 0 : rows;
 }
 
@@ -1749,6 +1749,13 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
         default: return BODA_ERR_UNSUPPORTED;
     }
 }
+
+#ifdef BODA_FL_PROF
+extern "C" int boda_debug_fl_prof(long long* out16)
+{
+    return cudaMemcpyFromSymbol(out16, halo::g_fl_prof, sizeof(long long) * 16) == cudaSuccess ? 0 : 3;
+}
+#endif
 
 // ------------------------------------------------------------------------------------------------
 // The same convolution with every piece of scratch (status word, re-laid-out filters and

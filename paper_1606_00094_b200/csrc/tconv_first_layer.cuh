@@ -99,6 +99,7 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
     const int taps = p.h.taps;
 
     pdl_launch_dependents();
+    if (threadIdx.x == 64) FL_STAMP(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int c = 0; c < 3; ++c) mbar_init(raw_full + 8 * c, 1);
@@ -144,7 +145,7 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
             bool ok = mbar_wait(slab_full, 0, &s_abort, p.h.status, 53);
             for (int i = 0; ok && i < 2 * taps; ++i) {
                 const bool second = i >= taps;
-                if (i == taps) { ok = mbar_wait(slab_full + 8, 0, &s_abort, p.h.status, 54); if (!ok) break; }
+                if (i == taps) { if (acc == 0) FL_STAMP(1); ok = mbar_wait(slab_full + 8, 0, &s_abort, p.h.status, 54); if (!ok) break; }
                 ok = mbar_wait(b_full + 8 * stage, par, &s_abort, p.h.status, 55);
                 if (!ok) break;
                 tc_fence_after();
@@ -165,6 +166,7 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
                 if (++stage == (uint32_t)p.b_stages) { stage = 0; par ^= 1u; }
             }
             tc_commit(accum_bar);
+            if (acc == 0) FL_STAMP(6);
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.h.status, 56);
         }
     } else {
@@ -215,27 +217,31 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
                 const int yl0 = kStride * ybl;
                 if (chunk == 0) {
                     const uint32_t dst = slab0 + (uint32_t)i * 128u + (uint32_t)dx * 4u;
+                    float v[8];
 #pragma unroll
-                    for (int jj = 0; jj < 8; ++jj) {
+                    for (int jj = 0; jj < 8; ++jj) {                       // all eight loads first: their latencies overlap
                         const int c = jj >> 2, dy = jj & 3;                // literals after unrolling
                         const int yl = yl0 + dy;
                         const bool ok = xok && yl < rows_avail;
                         const uint32_t src = (c ? raw1 : raw0) + (uint32_t)((c ? mis1 : mis0) + yl * W + x) * 4u;
-                        float v = 0.f;
-                        if (ok) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(src));
-                        st_shared_f32(dst + (uint32_t)((jj ^ (i & 7)) << 4), round_to_tf32(v));
+                        v[jj] = 0.f;
+                        if (ok) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[jj]) : "r"(src));
                     }
+#pragma unroll
+                    for (int jj = 0; jj < 8; ++jj) st_shared_f32(dst + (uint32_t)((jj ^ (i & 7)) << 4), round_to_tf32(v[jj]));
                 } else {
                     const uint32_t dst = slab1 + (uint32_t)i * 64u + (uint32_t)dx * 4u;
+                    float v[4];
 #pragma unroll
                     for (int dy = 0; dy < 4; ++dy) {
                         const int yl = yl0 + dy;
                         const bool ok = xok && yl < rows_avail;
                         const uint32_t src = raw0 + (uint32_t)(mis0 + yl * W + x) * 4u;
-                        float v = 0.f;
-                        if (ok) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v) : "r"(src));
-                        st_shared_f32(dst + (uint32_t)((dy ^ ((i >> 1) & 3)) << 4), round_to_tf32(v));
+                        v[dy] = 0.f;
+                        if (ok) asm volatile("ld.shared.f32 %0, [%1];" : "=f"(v[dy]) : "r"(src));
                     }
+#pragma unroll
+                    for (int dy = 0; dy < 4; ++dy) st_shared_f32(dst + (uint32_t)((dy ^ ((i >> 1) & 3)) << 4), round_to_tf32(v[dy]));
                 }
             }
         };
@@ -255,10 +261,12 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
             if (tail1) patch_tail(1, raw1);
             asm volatile("bar.sync 2, 256;" ::: "memory");
         }
+        if (etid == 0) FL_STAMP(2);
         if (ok) build(0, mis_c0, mis_c1);
         fence_proxy_async_smem();                               // the tensor core reads the slab through the asynchronous proxy
         asm volatile("bar.sync 2, 256;" ::: "memory");       // every builder is done with both raw buffers
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(slab_full) : "memory");
+        if (etid == 0) FL_STAMP(3);
         if (etid == 0) load_raw(2, raw0, raw_full + 16);
         if (lane == 0) ok = ok && mbar_wait(raw_full + 16, 0, &s_abort, p.h.status, 59);
         ok = __shfl_sync(0xffffffffu, ok ? 1 : 0, 0) != 0;
@@ -267,15 +275,18 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
             patch_tail(2, raw0);
             asm volatile("bar.sync 2, 256;" ::: "memory");
         }
+        if (etid == 0) FL_STAMP(4);
         if (ok) build(1, mis_c2, 0);
         fence_proxy_async_smem();
         __syncwarp();
         if (lane == 0) asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" :: "r"(slab_full + 8) : "memory");
+        if (etid == 0) FL_STAMP(5);
         const uint32_t region = (uint32_t)p.slab_rows * 128u + 2u * (uint32_t)p.raw_buf_bytes + (uint32_t)p.b_stages * B_STAGE_BYTES;
         // the tile owns rows_per_tile output rows, but never positions of the next image (a small image ends inside the tile)
         halo::HaloParams h = p.h;
         h.tile_positions = min(p.h.tile_positions, p.h.HpWp - row_first * p.h.Wp);
         halo::halo_epilogue<BN, NACC>(h, smem_base, region, tmem_acc, s_bias, &s_abort, accum_bar, f0, k0, warp, lane);
+        if (etid == 0) FL_STAMP(7);
         tc_fence_before();
     }
     __syncthreads();

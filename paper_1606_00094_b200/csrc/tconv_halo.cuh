@@ -82,6 +82,14 @@ struct HaloCfg {
     static constexpr int ISSUERS = NACC >= 4 ? 4 : NACC >= 2 ? 2 : 1;
 };
 
+#ifdef BODA_FL_PROF
+// development aid (off unless the library is built with -DBODA_FL_PROF): clock stamps of CTA (0, 0)
+__device__ long long g_fl_prof[16];
+#define FL_STAMP(i) do { if ((blockIdx.x | blockIdx.y) == 0) ::boda::halo::g_fl_prof[i] = clock64(); } while (0)
+#else
+#define FL_STAMP(i) do { } while (0)
+#endif
+
 // ---- fused ReLU -> max-pool epilogue (3x3 window, stride 2, no padding, floor extent).
 // The paper fuses the activation into the convolution (Section 2) and names fusion as what a BLAS call cannot do
 // (Section 3); here the pooling that follows the activation is fused as well, so that the convolution's output -
@@ -93,20 +101,33 @@ struct HaloCfg {
 // thread takes pooled (row, column, 4 channels) items, reads the nine window positions and writes the maximum,
 // rounded to TF32, into the pooled tile [pool_rows * Q][BN] (or straight to an NCHW tensor).  Two blocks alternate,
 // so filling block c+1 overlaps pooling block c.  At the end each pooled position leaves as one bulk copy.
+// bytes of one position's 32 channels in a pooling block: 128 of data + 16 of padding, which keeps thread-per-position
+// 16-byte stores and piece-per-thread window loads free of bank conflicts without any address swizzling
+constexpr uint32_t kPoolRowBytes = 144;
+// shared memory the fused pooling needs: two blocks and the pooled tile
+__host__ __device__ constexpr long long pooled_epilogue_bytes(int nacc, int pooled_positions, int BN)
+{
+    return 2LL * nacc * 128 * kPoolRowBytes + (long long)pooled_positions * BN * 4;
+}
+
 template <int BN, int NACC>
 __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32_t smem_base, uint32_t tmem_acc, const float* s_bias,
                                                      int k0, int group, int quarter, int lane, int etid)
 {
     static_assert(NACC == 2 || NACC == 4, "the two epilogue groups take alternate accumulators");
     constexpr int NCH = BN / 32;
-    constexpr uint32_t BLOCK_BYTES = (uint32_t)NACC * 128u * 128u;
+    constexpr uint32_t BLOCK_BYTES = (uint32_t)NACC * 128u * kPoolRowBytes;
     const uint32_t pooled = smem_base + 2u * BLOCK_BYTES;
     const int n = (int)blockIdx.x / p.tiles_per_image;
     const int j = (int)blockIdx.x - n * p.tiles_per_image;
     const int prow0 = p.pool_rows * j;                                  // first pooled row of this tile
     const int prows = min(p.pool_rows, p.o.P - prow0);                  // pooled rows this tile owns
-    const int items = prows * p.o.Q * 8;                                // (pooled position, 4 channels)
+    const int npos = prows * p.o.Q;                                     // pooled positions this tile owns
     const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
+    // a thread pools one 16-byte piece (4 channels) g of pooled positions t0, t0 + 32, ...: everything that depends on g
+    // and on the window geometry is computed once
+    const int g = etid & 7, t0 = etid >> 3;
+    const uint32_t row_pitch = (uint32_t)p.Wp * kPoolRowBytes;
 #pragma unroll 1
     for (int c = 0; c < NCH; ++c) {
         const uint32_t block = smem_base + (uint32_t)(c & 1) * BLOCK_BYTES;
@@ -118,27 +139,26 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
             tmem_ld_wait();
             float y[32];
             bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
-            const uint32_t a = block + (uint32_t)pos * 128u;
+            const uint32_t a = block + (uint32_t)pos * kPoolRowBytes;
 #pragma unroll
-            for (int g = 0; g < 8; ++g)
-                st_shared_v4(a + (uint32_t)((g ^ (pos & 7)) << 4), y[4 * g], y[4 * g + 1], y[4 * g + 2], y[4 * g + 3]);
+            for (int q = 0; q < 8; ++q) st_shared_v4(a + 16u * q, y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
         }
+        if (etid == 0 && c == 0) FL_STAMP(8);
         // every thread is past its pooling of block c-1 when it arrives here, so block (c+1)&1 may be refilled after it
         asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (etid == 0 && c == 0) FL_STAMP(9);
+        int pr = t0 / p.o.Q, pq = t0 - pr * p.o.Q;
 #pragma unroll 1
-        for (int item = etid; item < items; item += 256) {
-            const int g = item & 7, t = item >> 3;
-            const int pr = t / p.o.Q, pq = t - pr * p.o.Q;
-            const int pos0 = 2 * pr * p.Wp + 2 * pq;
-            float4 m = make_float4(0.f, 0.f, 0.f, 0.f);
+        for (int t = t0; t < npos; t += 32) {
+            const uint32_t w0 = block + (uint32_t)(2 * pr * p.Wp + 2 * pq) * kPoolRowBytes + 16u * (uint32_t)g;
+            float4 m = ld_shared_v4(w0);
 #pragma unroll
             for (int dr = 0; dr < 3; ++dr)
 #pragma unroll
                 for (int ds = 0; ds < 3; ++ds) {
-                    const int pos = pos0 + dr * p.Wp + ds;
-                    const float4 x = ld_shared_v4(block + (uint32_t)pos * 128u + (uint32_t)((g ^ (pos & 7)) << 4));
-                    if (dr == 0 && ds == 0) m = x;
-                    else { m.x = fmaxf(m.x, x.x); m.y = fmaxf(m.y, x.y); m.z = fmaxf(m.z, x.z); m.w = fmaxf(m.w, x.w); }
+                    if (dr == 0 && ds == 0) continue;
+                    const float4 x = ld_shared_v4(w0 + (uint32_t)dr * row_pitch + (uint32_t)ds * kPoolRowBytes);
+                    m.x = fmaxf(m.x, x.x); m.y = fmaxf(m.y, x.y); m.z = fmaxf(m.z, x.z); m.w = fmaxf(m.w, x.w);
                 }
             if (p.o.packed) {
                 st_shared_v4(pooled + (uint32_t)(t * BN + 32 * c + 4 * g) * 4u, round_to_tf32(m.x), round_to_tf32(m.y),
@@ -151,21 +171,50 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
                 for (int e = 0; e < 4; ++e)
                     if (k + e < p.o.K) dst[(size_t)e * p.o.PQ] = mv[e];
             }
+            // position t + 32 without a division
+            pq += 32;
+            while (pq >= p.o.Q) { pq -= p.o.Q; ++pr; }
         }
+        if (etid == 0 && c == 0) FL_STAMP(10);
     }
+    if (etid == 0) FL_STAMP(11);
     if (p.o.packed) {
         fence_proxy_async_smem();
         asm volatile("bar.sync 1, 256;" ::: "memory");
+        if (etid == 0) FL_STAMP(12);
         const int w = min(BN, p.o.Cp - k0);
         if (w > 0) {
-            for (int t = etid; t < prows * p.o.Q; t += 256) {
-                const int pr = t / p.o.Q, pq = t - pr * p.o.Q;
-                float* dst = p.o.out + ((size_t)(n * p.o.Hp + prow0 + pr) * p.o.Wp + pq) * (size_t)p.o.Cp + k0;
-                bulk_store_global(dst, pooled + (uint32_t)(t * BN) * 4u, (uint32_t)w * 4u);
+            // One thread issues one bulk copy, and the lanes of a warp issue theirs one after the other: copy whole
+            // pooled rows where they are contiguous on both sides (the tile spans all the consumer's channels), so that
+            // a tile leaves in a handful of copies instead of one per position.
+            const bool rows_contiguous = w == BN && p.o.Cp == BN;
+            if (rows_contiguous) {
+                const bool all_contiguous = p.o.Wp == p.o.Q;
+                if (all_contiguous) {
+                    if (etid == 0) {
+                        float* dst = p.o.out + ((size_t)(n * p.o.Hp + prow0) * p.o.Wp) * (size_t)p.o.Cp;
+                        bulk_store_global(dst, pooled, (uint32_t)npos * (uint32_t)BN * 4u);
+                    }
+                } else if ((etid & 31) == 0 || prows > 8) {
+                    // lane 0 of each of the eight warps takes rows warp, warp + 8, ...; many rows: every thread takes some
+                    const int first_row = prows > 8 ? etid : etid >> 5, step = prows > 8 ? 256 : 8;
+                    for (int r = first_row; r < prows; r += step) {
+                        float* dst = p.o.out + ((size_t)(n * p.o.Hp + prow0 + r) * p.o.Wp) * (size_t)p.o.Cp;
+                        bulk_store_global(dst, pooled + (uint32_t)(r * p.o.Q * BN) * 4u, (uint32_t)p.o.Q * (uint32_t)BN * 4u);
+                    }
+                }
+            } else {
+                for (int t = etid; t < npos; t += 256) {
+                    const int pr2 = t / p.o.Q, pq2 = t - pr2 * p.o.Q;
+                    float* dst = p.o.out + ((size_t)(n * p.o.Hp + prow0 + pr2) * p.o.Wp + pq2) * (size_t)p.o.Cp + k0;
+                    bulk_store_global(dst, pooled + (uint32_t)(t * BN) * 4u, (uint32_t)w * 4u);
+                }
             }
         }
         bulk_commit();
+        if (etid == 0) FL_STAMP(13);
         bulk_wait_all();
+        if (etid == 0) FL_STAMP(14);
     }
 }
 
@@ -191,6 +240,7 @@ __device__ __forceinline__ void halo_epilogue(const HaloParams& p, uint32_t smem
     asm volatile("bar.sync 1, 256;" ::: "memory");
     const bool ok = (*s_abort == 0);
     tc_fence_after();
+    if (etid == 0) FL_STAMP(15);
     const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
     if (ok && p.pool_rows > 0) {
         if constexpr (NACC >= 2) halo_pooled_epilogue<BN, NACC>(p, smem_base, tmem_acc, s_bias, k0, group, quarter, lane, etid);
