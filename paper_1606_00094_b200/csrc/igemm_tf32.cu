@@ -132,6 +132,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     const bool exchange = split_exchange_fits(BN, p.splits, STAGES * Cfg::STAGE_BYTES);   // the same in every CTA
 
     pdl_launch_dependents();
+    if (threadIdx.x == 0 && blockIdx.z == 0) FL_STAMP(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 16 * s, 1); mbar_init(full_bar + 16 * s + 8, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -153,6 +154,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
     // tiles are not its results: with bound filters their producer and the byte counts start at once, so the first
     // filter tiles (HBM-cold after a long pause) are on their way while the input is still being written.
     if (!(p.b_early && (warp == 11 || warp == 12))) pdl_wait();
+    if (threadIdx.x == 0 && blockIdx.z == 0) FL_STAMP(1);
 
     if (warp == 0 || warp >= 11) {
         if (lane == 0) {
@@ -252,6 +254,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             for (int i = me; i < my_iters; i += STEP) {
                 ok = mbar_wait(fb, par, &s_abort, p.status, 2);
                 if (!ok) break;
+                if (i == 0 && blockIdx.z == 0) FL_STAMP(2);
                 tc_fence_after();
 #pragma unroll
                 for (int k = 0; k < BKC / 8; ++k) {     // 8 TF32 (16 fp16) values = 32 bytes = 2 descriptor units per step
@@ -272,6 +275,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 if (++visited == CYCLE) { visited = 0; par ^= 1u; }
             }
             tc_commit(accum_bar);                       // this issuer's MMAs have drained
+            if (me == 0 && blockIdx.z == 0) FL_STAMP(3);
             if (!ok) (void)mbar_wait(accum_bar, 0, &s_abort, p.status, 3);
         }
     } else {
@@ -298,6 +302,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                      : "=r"(stop) : "r"((uint32_t)s_abort) : "memory");
         const bool ok = stop == 0;
         tc_fence_after();
+        if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(4);
         const uint32_t trow = tmem_acc + ((uint32_t)(quarter * 32) << 16);
         const bool two_acc = Cfg::ISSUERS == 2 && my_iters >= 2;   // a single reduction step never reaches the second issuer
         // 32 accumulator columns of this thread's row (the sum of the two issuers' accumulators)
@@ -372,7 +377,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                         fence_proxy_async_smem();
                         if (group) asm volatile("bar.sync 3, 128;" ::: "memory"); else asm volatile("bar.sync 2, 128;" ::: "memory");
                         if (push_warp) {
-                            if (!waited) { cluster_wait(); waited = true; }
+                            if (!waited) { cluster_wait(); waited = true; if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(6); }
                             if (lane == 0)
                                 bulk_push_cluster(map_to_cta(slot + 16384u * (uint32_t)c, (uint32_t)dst), block + 16384u * (uint32_t)c, 16384u,
                                               map_to_cta(recv_bar + 8 * c, (uint32_t)dst));
@@ -380,12 +385,14 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     }
                 }
             }
+            if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(7);
             if (!waited) cluster_wait();           // every thread takes the second half of the barrier exactly once
             if (ok && my_w > 0) {
                 const RowDst d = igemm_row_dst(p, m);
 #pragma unroll 1
                 for (int c = group; 32 * c < my_w; c += 2) {
                     if (!mbar_wait(recv_bar + 8 * c, 0, &s_abort, p.status, 5)) break;
+                    if (threadIdx.x == 64 && blockIdx.z == 0 && c == 0) FL_STAMP(8);
                     uint32_t v[32];
                     load32(rank * per + 32 * c, v);
                     float y[32];
@@ -398,6 +405,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                     bias_relu32(v, s_bias + rank * per + 32 * c, p.o.relu != 0, y);
                     store_row32(p.o, d, k0 + rank * per + 32 * c, y);
                 }
+                if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(9);
             }
         } else if (ok) {
             // split reduction through remote reads (the exchange blocks do not fit), step 1: park this CTA's partial
@@ -427,6 +435,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
             }
         }
         cluster_sync_all();          // nobody leaves while a peer may still read or write its shared memory
+        if (threadIdx.x == 0 && blockIdx.z == 0) FL_STAMP(10);
     }
     if (warp == 1) {
         __syncwarp();
@@ -698,6 +707,7 @@ struct IgemmPlan {
     int tiles_m = 0, tiles_n = 0;
     int* d_status = nullptr;
     float* d_wp = nullptr;           // packed filters [RS][K][Cp]
+    size_t wp_bytes = 0;
     const float* bound_filt = nullptr;
     size_t xp_bytes = 0, partial_bytes = 0;
     CUtensorMap map_b;
@@ -1263,7 +1273,8 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         p->tiles_n = (d_in.K + p->BN - 1) / p->BN;
         p->xp_bytes = 0;
         p->partial_bytes = 0;
-        cudaError_t fe = cudaMalloc(&p->d_wp, (size_t)p->fl_Rb * p->fl_Sb * d_in.K * first::kViewChannels * 4);
+        p->wp_bytes = (size_t)p->fl_Rb * p->fl_Sb * d_in.K * first::kViewChannels * 4;
+        cudaError_t fe = cudaMalloc(&p->d_wp, p->wp_bytes);
         if (fe != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(fe, "plan allocation"); }
         rc = encode_map_b(p);
         if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -1286,7 +1297,8 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         p->tiles_n = (d_in.K + p->BN - 1) / p->BN;
         p->xp_bytes = 0;
         p->partial_bytes = 0;
-        cudaError_t ke = cudaMalloc(&p->d_wp, (size_t)d_in.K * p->Cp * 4);
+        p->wp_bytes = (size_t)d_in.K * p->Cp * 4;
+        cudaError_t ke = cudaMalloc(&p->d_wp, p->wp_bytes);
         if (ke != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(ke, "plan allocation"); }
         rc = encode_map_b(p);
         if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -1319,7 +1331,8 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
         }
         cudaError_t ge = cudaMalloc(&p->d_tab, (size_t)Kp * sizeof(int2));
         if (ge == cudaSuccess) ge = cudaMemcpy(p->d_tab, tab.data(), (size_t)Kp * sizeof(int2), cudaMemcpyHostToDevice);
-        if (ge == cudaSuccess) ge = cudaMalloc(&p->d_wp, (size_t)g.K * Kp * 4);
+        p->wp_bytes = (size_t)g.K * Kp * 4;
+        if (ge == cudaSuccess) ge = cudaMalloc(&p->d_wp, p->wp_bytes);
         if (ge != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(ge, "gather plan allocation"); }
         rc = encode_map_b(p);
         if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
@@ -1342,7 +1355,8 @@ int igemm_plan_create(const ConvDims& d_in, int variant, int tile_id, int split_
     }
 
     if (max_ws > 0 && p->xp_bytes > max_ws) { delete p; return BODA_ERR_NOMEM; }
-    cudaError_t e = cudaMalloc(&p->d_wp, (size_t)d.R * d.S * d.K * p->Cs() * p->esize());
+    p->wp_bytes = (size_t)d.R * d.S * d.K * p->Cs() * p->esize();
+    cudaError_t e = cudaMalloc(&p->d_wp, p->wp_bytes);
     if (e != cudaSuccess) { igemm_plan_destroy(p); return record_cuda_error(e, "igemm plan allocation"); }
     rc = encode_map_b(p);
     if (rc != BODA_OK) { igemm_plan_destroy(p); return rc; }
