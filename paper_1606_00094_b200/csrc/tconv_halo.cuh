@@ -131,49 +131,67 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
 #pragma unroll 1
     for (int c = 0; c < NCH; ++c) {
         const uint32_t block = smem_base + (uint32_t)(c & 1) * BLOCK_BYTES;
-#pragma unroll 1
-        for (int acc = group; acc < NACC; acc += 2) {
-            const int pos = acc * 128 + quarter * 32 + lane;
-            uint32_t v[32];
-            tmem_ld_32cols(trow + acc * BN + 32 * c, v);
-            tmem_ld_wait();
+        auto put = [&](int acc, const uint32_t (&v)[32]) {
             float y[32];
             bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
-            const uint32_t a = block + (uint32_t)pos * kPoolRowBytes;
+            const uint32_t a = block + (uint32_t)(acc * 128 + quarter * 32 + lane) * kPoolRowBytes;
 #pragma unroll
             for (int q = 0; q < 8; ++q) st_shared_v4(a + 16u * q, y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+        };
+        if constexpr (NACC == 4) {
+            // both of this group's accumulators are read from tensor memory before either is used: one load latency per block
+            uint32_t v0[32], v1[32];
+            tmem_ld_32cols(trow + group * BN + 32 * c, v0);
+            tmem_ld_32cols(trow + (group + 2) * BN + 32 * c, v1);
+            tmem_ld_wait();
+            put(group, v0);
+            put(group + 2, v1);
+        } else {
+            uint32_t v[32];
+            tmem_ld_32cols(trow + group * BN + 32 * c, v);
+            tmem_ld_wait();
+            put(group, v);
         }
         if (etid == 0 && c == 0) FL_STAMP(8);
         // every thread is past its pooling of block c-1 when it arrives here, so block (c+1)&1 may be refilled after it
         asm volatile("bar.sync 1, 256;" ::: "memory");
         if (etid == 0 && c == 0) FL_STAMP(9);
-        int pr = t0 / p.o.Q, pq = t0 - pr * p.o.Q;
+        // A thread pools piece g of ONE pooled column pq for all the pooled rows of the tile, walking down the 2*prows + 1
+        // output rows once: per row the maximum of the three columns 2pq .. 2pq+2, and every pooled row is the maximum of
+        // three consecutive row maxima (rows 2r, 2r+1, 2r+2; row 2r+2 is also row 2(r+1) of the next pooled row).  That
+        // is 3 * (2*prows + 1) window loads for prows outputs instead of 9 * prows: the pooling is bound by the
+        // bandwidth of shared memory.
+        for (int pq = t0; pq < p.o.Q; pq += 32) {
+            uint32_t w = block + (uint32_t)(2 * pq) * kPoolRowBytes + 16u * (uint32_t)g;
+            auto row_max = [&](uint32_t a) {
+                float4 m = ld_shared_v4(a);
+                const float4 x1 = ld_shared_v4(a + kPoolRowBytes), x2 = ld_shared_v4(a + 2u * kPoolRowBytes);
+                m.x = fmaxf(m.x, fmaxf(x1.x, x2.x)); m.y = fmaxf(m.y, fmaxf(x1.y, x2.y));
+                m.z = fmaxf(m.z, fmaxf(x1.z, x2.z)); m.w = fmaxf(m.w, fmaxf(x1.w, x2.w));
+                return m;
+            };
+            float4 top = row_max(w);                                       // output row 2*pr
 #pragma unroll 1
-        for (int t = t0; t < npos; t += 32) {
-            const uint32_t w0 = block + (uint32_t)(2 * pr * p.Wp + 2 * pq) * kPoolRowBytes + 16u * (uint32_t)g;
-            float4 m = ld_shared_v4(w0);
+            for (int pr = 0; pr < prows; ++pr) {
+                const float4 mid = row_max(w + row_pitch), bot = row_max(w + 2u * row_pitch);
+                float4 m;
+                m.x = fmaxf(top.x, fmaxf(mid.x, bot.x)); m.y = fmaxf(top.y, fmaxf(mid.y, bot.y));
+                m.z = fmaxf(top.z, fmaxf(mid.z, bot.z)); m.w = fmaxf(top.w, fmaxf(mid.w, bot.w));
+                const int t = pr * p.o.Q + pq;
+                if (p.o.packed) {
+                    st_shared_v4(pooled + (uint32_t)(t * BN + 32 * c + 4 * g) * 4u, round_to_tf32(m.x), round_to_tf32(m.y),
+                                 round_to_tf32(m.z), round_to_tf32(m.w));
+                } else {
+                    const int k = k0 + 32 * c + 4 * g;
+                    float* dst = p.o.out + ((size_t)(n * p.o.K + k) * p.o.P + prow0 + pr) * p.o.Q + pq;
+                    const float mv[4] = {m.x, m.y, m.z, m.w};
 #pragma unroll
-            for (int dr = 0; dr < 3; ++dr)
-#pragma unroll
-                for (int ds = 0; ds < 3; ++ds) {
-                    if (dr == 0 && ds == 0) continue;
-                    const float4 x = ld_shared_v4(w0 + (uint32_t)dr * row_pitch + (uint32_t)ds * kPoolRowBytes);
-                    m.x = fmaxf(m.x, x.x); m.y = fmaxf(m.y, x.y); m.z = fmaxf(m.z, x.z); m.w = fmaxf(m.w, x.w);
+                    for (int e = 0; e < 4; ++e)
+                        if (k + e < p.o.K) dst[(size_t)e * p.o.PQ] = mv[e];
                 }
-            if (p.o.packed) {
-                st_shared_v4(pooled + (uint32_t)(t * BN + 32 * c + 4 * g) * 4u, round_to_tf32(m.x), round_to_tf32(m.y),
-                             round_to_tf32(m.z), round_to_tf32(m.w));
-            } else {
-                const int k = k0 + 32 * c + 4 * g;
-                float* dst = p.o.out + ((size_t)(n * p.o.K + k) * p.o.P + prow0 + pr) * p.o.Q + pq;
-                const float mv[4] = {m.x, m.y, m.z, m.w};
-#pragma unroll
-                for (int e = 0; e < 4; ++e)
-                    if (k + e < p.o.K) dst[(size_t)e * p.o.PQ] = mv[e];
+                top = bot;
+                w += 2u * row_pitch;
             }
-            // position t + 32 without a division
-            pq += 32;
-            while (pq >= p.o.Q) { pq -= p.o.Q; ++pr; }
         }
         if (etid == 0 && c == 0) FL_STAMP(10);
     }
