@@ -799,12 +799,17 @@ bool igemm_variant_profitable(const ConvDims& d)
 {
     // Channels are padded to 32 per reduction chunk and pixels to 128 per tile: tiny C (first layers) and tiny
     // layers stay on the FP32 kernel.
-    if (d.K < 16 || (long long)d.M * d.K < 128 * 64) return false;
+    if (d.K < 16) return false;
+    // tiny layers stay on the FP32 kernel (one 3 us launch beats the tensor-core kernels' fixed costs) unless the
+    // reduction is long: measured on a 1x1 layer with 96 channels on 6x6 points, 16 filters: 3.7 us on the NCHW 1x1
+    // kernel against 8.3 us for the FP32 kernel, whose loop over the reduction is bound by latency
+    if ((long long)d.M * d.K < 128 * 64 && !(d.R * d.S == 1 && d.Kred >= 64)) return false;
     const int Cp = ((d.C + BKC - 1) / BKC) * BKC;
     // measured: staged input with C = 8 of 32 channels wins, C = 3 of 32 loses; the gather kernel needs no staged input
-    // (tiny layers stay on the FP32 kernel: one 3 us launch beats the tensor-core kernel's fixed costs)
+    // but its narrowest tile has 64 columns: with 16 filters the run-time compiled FP32 kernel wins (5x5 on 3 channels,
+    // 64x64, batch 20: 12.6 against 19.1 us), so the gather rule asks for at least 32 filters
     return std::max((double)d.C / Cp, s2d_efficiency(d)) >= 0.2 ||
-           (d.R * d.S >= 2 && ((d.Kred + 31) / 32) * 32 <= gconv::kMaxKred && (long long)d.M * d.K >= 128 * 256);
+           (d.R * d.S >= 2 && d.K >= 32 && ((d.Kred + 31) / 32) * 32 <= gconv::kMaxKred && (long long)d.M * d.K >= 128 * 256);
 }
 
 int igemm_num_tiles() { return kNumIgemmTiles; }
