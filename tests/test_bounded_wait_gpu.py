@@ -48,7 +48,8 @@ def test_expired_wait_sets_status_and_context_survives(tile, split):
     assert_parity(got, oracle_out(shape, x, w, b), TF32_TOL)
 
 
-def test_expired_wait_in_the_nchw_1x1_kernel():
+@pytest.mark.parametrize("split", [1, 2])          # persistent form, and one tile per CTA with a cluster split over the channels
+def test_expired_wait_in_the_nchw_1x1_kernel(split):
     import torch
     from paper_1606_00094_b200 import binding as B
     shape = (3, 64, 12, 12, 200, 1, 1, 1, 0, 1)
@@ -61,7 +62,7 @@ def test_expired_wait_in_the_nchw_1x1_kernel():
     os.environ["BODA_TEST_TX_MISMATCH"] = "1"
     os.environ["BODA_WAIT_LIMIT_CYCLES"] = "100000000"
     try:
-        plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20)
+        plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20, split_k=split)
     finally:
         del os.environ["BODA_TEST_TX_MISMATCH"]
         del os.environ["BODA_WAIT_LIMIT_CYCLES"]
@@ -70,7 +71,37 @@ def test_expired_wait_in_the_nchw_1x1_kernel():
     assert B.boda_query_status() == B.BODA_ERR_DEVICE_TIMEOUT
     assert B.boda_query_status() == 0
     plan.close()
-    plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20)
+    plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_K1CONV, tile_id=20, split_k=split)
+    got = plan(dx, dw, db).cpu().numpy()
+    torch.cuda.synchronize()
+    assert B.boda_query_status() == 0
+    plan.close()
+    assert_parity(got, oracle_out(shape, x, w, b), TF32_TOL)
+
+
+def test_expired_wait_in_the_first_layer_kernel():
+    import torch
+    from paper_1606_00094_b200 import binding as B
+    shape = (2, 3, 67, 67, 80, 11, 11, 4, 0, 1)
+    N, C, H, W, K, R, S, st, pad, relu = shape
+    x = wl.half_normal(7, (N, C, H, W))
+    w = wl.normal(8, (K, C, R, S), 0, (2.0 / (C * R * S)) ** 0.5)
+    b = wl.normal(9, (K,), 0, 0.01)
+    dx, dw, db = (torch.from_numpy(t).cuda() for t in (x, w, b))
+    assert B.boda_query_status() == 0
+    os.environ["BODA_TEST_TX_MISMATCH"] = "1"
+    os.environ["BODA_WAIT_LIMIT_CYCLES"] = "100000000"
+    try:
+        plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_TCONV, tile_id=24)
+    finally:
+        del os.environ["BODA_TEST_TX_MISMATCH"]
+        del os.environ["BODA_WAIT_LIMIT_CYCLES"]
+    plan(dx, dw, db)
+    torch.cuda.synchronize()
+    assert B.boda_query_status() == B.BODA_ERR_DEVICE_TIMEOUT
+    assert B.boda_query_status() == 0
+    plan.close()
+    plan = B.ConvPlan(shape, variant=B.BODA_VARIANT_TCONV, tile_id=24)
     got = plan(dx, dw, db).cpu().numpy()
     torch.cuda.synchronize()
     assert B.boda_query_status() == 0
