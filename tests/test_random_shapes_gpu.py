@@ -115,3 +115,72 @@ def test_degenerate_shapes_exact_on_integers(shape):
         np.testing.assert_array_equal(got.astype(np.float64), ref, err_msg=f"{shape} {desc}")
         ran += 1
     assert ran >= 2
+
+
+# ---- seeded random CHAINS conv -> pool -> conv: whatever the stack decides (staged hand-off, pool in the epilogue or as a
+# kernel, first-layer kernel) must reproduce the fp64 oracle chain EXACTLY on operands from {-1, 0, 1}
+def _chains(seed, count):
+    r = wl.uniform01(seed, count * 10).reshape(count, 10)
+    out = []
+    for u in r:
+        pick = lambda a, lst: lst[min(int(a * len(lst)), len(lst) - 1)]
+        first_layer = u[0] < 0.4
+        N = pick(u[1], [1, 2, 3])
+        if first_layer:            # 3 channels, stride 4, no padding: legal for the first-layer kernel
+            R = pick(u[2], [5, 7, 8, 9, 11]); S = R if u[3] < 0.6 else pick(u[3], [5, 7, 9, 11])
+            P = pick(u[4], [7, 9, 12, 15, 21]); Q = pick(u[5], [7, 10, 13, 15, 22])
+            c1 = wl.ConvShape(N, 3, 4 * (P - 1) + R, 4 * (Q - 1) + S, pick(u[6], [16, 40, 64, 96]), R, S, 4, 0, True)
+        else:
+            R = pick(u[2], [2, 3, 3, 5]); pad = pick(u[3], [0, 1, 1, 2]); pad = min(pad, R - 1)
+            H = pick(u[4], [7, 9, 13, 16, 19]); W = pick(u[5], [7, 10, 13, 17, 20])
+            c1 = wl.ConvShape(N, pick(u[6], [8, 24, 40, 64]), H, W, pick(u[7], [16, 40, 72, 96]), R, R, 1, pad, True)
+        if c1.P < 3 or c1.Q < 3:
+            continue
+        pP, pQ = (c1.P - 3) // 2 + 1, (c1.Q - 3) // 2 + 1
+        R2 = pick(u[8], [1, 3, 3, 5]); pad2 = R2 // 2
+        c2 = wl.ConvShape(N, c1.K, pP, pQ, pick(u[9], [16, 48, 80]), R2, R2, 1, pad2, False)
+        out.append((c1, c2, first_layer))
+    return out
+
+
+CHAINS = _chains(0xC4A1, 40)
+
+
+@pytest.mark.parametrize("idx", range(len(CHAINS)))
+@pytest.mark.parametrize("forced", [False, True])
+def test_random_chain_exact(idx, forced):
+    """forced: the first convolution on a tile that can run the pool in its epilogue (a halo tile, or the first-layer
+    kernel), where the library accepts it for the shape; otherwise the rules choose."""
+    import torch
+    from oracle import conv_oracle as orc
+    from paper_1606_00094_b200 import binding as B
+    from paper_1606_00094_b200.stack import ConvStack
+    c1, c2, first_layer = CHAINS[idx]
+    ops = [wl.StackOp("conv", c1), wl.StackOp("pool"), wl.StackOp("conv", c2)]
+    tern = lambda seed, shape: wl.integers(seed, shape, -1, 1)
+    x = tern(9000 + idx, (c1.N, c1.C, c1.H, c1.W))
+    # sparse second-layer filters keep every sum far below 2^24; the first layer's sums are at most C*R*S <= 2048
+    w2 = (tern(9300 + idx, (c2.K, c2.C, c2.R, c2.S)) * (wl.uniform01(9400 + idx, c2.K * c2.C * c2.R * c2.S).reshape(c2.K, c2.C, c2.R, c2.S) < 0.2)).astype(np.float32)
+    params = [(tern(9100 + idx, (c1.K, c1.C, c1.R, c1.S)), tern(9200 + idx, (c1.K,))), (w2, tern(9500 + idx, (c2.K,)))]
+    assert c1.C * c1.R * c1.S + 1 <= 2048
+    a = orc.conv_fwd(x, params[0][0], params[0][1], stride=c1.stride, pad=c1.pad, relu=True)
+    pooled = orc.maxpool_fwd(a, 3, 2)
+    ref = orc.conv_fwd(pooled, params[1][0], params[1][1], stride=1, pad=c2.pad, relu=False)
+    per_op = None
+    if forced:
+        per_op = [{"variant": 2, "tile_id": 24 if first_layer else 10}, {}, {}]
+    try:
+        stack = ConvStack(ops, params, per_op=per_op)
+    except B.BodaError as e:
+        assert forced and e.status == B.BODA_ERR_UNSUPPORTED, f"{c1} {c2}: {e}"
+        pytest.skip("the forced tile does not take this shape")
+    try:
+        descs = stack.describe()
+        out = stack.forward(torch.from_numpy(x).cuda())
+        torch.cuda.synchronize()
+        assert B.boda_query_status() == 0
+        got_pool = stack.layer_output(1)
+        np.testing.assert_array_equal(got_pool.cpu().numpy().astype(np.float64), pooled, err_msg=str(descs))
+        np.testing.assert_array_equal(out.cpu().numpy().astype(np.float64), ref, err_msg=str(descs))
+    finally:
+        stack.close()
