@@ -96,7 +96,10 @@ typedef struct boda_plan_opts {
                                     5..15 halo_128/256/512xBN (TCONV stride 1 or space-to-depth view: shared-memory
                                     reuse of the input across taps), 16..19 gconv_128x64/96/128/192 (input gathered
                                     from NCHW, nothing staged; short reductions and 1x1), 20..22 k1nchw_128x64/128/192
-                                    (K1CONV by TMA straight from NCHW).  A tile that cannot run the shape is refused
+                                    (K1CONV by TMA straight from NCHW; split_k > 1: a cluster split over the input
+                                    channels), 23..25 first_512x64/96/128 (TCONV for 3 input channels, stride 4, no
+                                    padding, windows up to 11x11: the space-to-depth view built in shared memory
+                                    straight from NCHW, nothing staged).  A tile that cannot run the shape is refused
                                     with BODA_ERR_UNSUPPORTED. */
     int split_k;                 /* 0: automatic; otherwise the number of reduction splits of a tensor-core variant */
     int device;                  /* CUDA device ordinal; -1: the current device */
@@ -145,8 +148,9 @@ int boda_conv_plan_describe(const boda_conv_plan* plan, char* buf, size_t buf_by
  * the re-laid-out input (the "input transformation" that the paper's k1conv and tconv apply, Section 5). */
 size_t boda_conv_plan_workspace_bytes(const boda_conv_plan* plan);
 
-/* Kernels one boda_conv_fwd_planned call launches when the filters are bound (1 for DIRECT; 2 for the
- * tensor-core variants: input staging and the main kernel). */
+/* Kernels one boda_conv_fwd_planned call launches when the filters are bound: 1 for DIRECT and for the tensor-core
+ * kernels that read NCHW themselves (gather, NCHW 1x1, first-layer kernel), 2 for the others (input staging and the
+ * main kernel). */
 int boda_conv_plan_kernels_per_call(const boda_conv_plan* plan);
 
 /*
@@ -278,6 +282,12 @@ int boda_softmax_fwd(const float* in, float* out, int rows, int cols, void* stre
  * benchmark uses.  (The paper's framework runs a whole compute graph, Section 4 and Figure "Boda flow"; this is
  * the minimal form of it: a linear chain.)  The stack owns its plans, the activations between layers, one
  * workspace and a CUDA graph of the chain, so that boda_stack_fwd is one graph launch.
+ * Fusion (the paper's argument for writing convolution kernels instead of calling a BLAS, Section 3): a 3x3 / stride-2
+ * max-pool that follows a convolution whose kernel works on whole output rows (halo tiles of 256 or 512 positions, the
+ * first-layer kernel) runs inside that kernel's epilogue; the convolution's own output is then never written, the pool
+ * op launches nothing, and boda_stack_copy_layer_output returns BODA_ERR_UNSUPPORTED for that convolution.
+ * BODA_STACK_NO_POOL_FUSION=1 in the environment keeps every pool a kernel of its own.  With opts->tune the layers are
+ * tuned the way the chain runs them (staged input and output, the pool that follows included).
  */
 enum { BODA_STACK_CONV = 0, BODA_STACK_MAXPOOL = 1 };
 typedef struct boda_stack_op {
