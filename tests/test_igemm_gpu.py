@@ -373,3 +373,30 @@ def test_tuned_choice_is_remembered_in_the_cache_file(tmp_path, monkeypatch):
         assert len(cache.read_text().strip().splitlines()) == 2
     finally:
         first.close(); second.close()
+
+
+def test_workspace_limit_steers_the_plan():
+    """opts.max_workspace: tiles whose staged input does not fit are not considered; automatic selection then lands on
+    a kernel that stages nothing (or the FP32 kernel), a forced tile that needs more is refused with BODA_ERR_NOMEM."""
+    from paper_1606_00094_b200 import binding as B
+    shape = (4, 64, 13, 13, 96, 3, 3, 1, 1, 1)
+    x, w, b = _real_tensors(shape, 3100)
+    ref = oracle_out(shape, x, w, b)
+    free = B.ConvPlan(shape)
+    need = B.boda_conv_plan_workspace_bytes(free.handle)
+    free.close()
+    assert need > 0                                           # the unconstrained choice stages its input
+    roomy = B.ConvPlan(shape, max_workspace=need)
+    assert B.boda_conv_plan_workspace_bytes(roomy.handle) <= need
+    roomy.close()
+    tight = B.ConvPlan(shape, max_workspace=1024)
+    try:
+        assert B.boda_conv_plan_workspace_bytes(tight.handle) <= 1024, tight.describe()
+        import torch
+        got = tight(torch.from_numpy(x).cuda(), torch.from_numpy(w).cuda(), torch.from_numpy(b).cuda()).cpu().numpy()
+        assert_parity(got, ref, TF32_TOL, tight.describe())
+    finally:
+        tight.close()
+    with pytest.raises(B.BodaError) as e:
+        B.ConvPlan(shape, variant=TC, tile_id=2, max_workspace=1024)
+    assert e.value.status == B.BODA_ERR_NOMEM
