@@ -133,6 +133,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 
     pdl_launch_dependents();
     if (threadIdx.x == 0 && blockIdx.z == 0) FL_STAMP(0);
+    if (threadIdx.x == 0) FL_CTA_TIME(0);
     if (threadIdx.x == 0) {
         s_abort = 0;
         for (int s = 0; s < STAGES; ++s) { mbar_init(full_bar + 16 * s, 1); mbar_init(full_bar + 16 * s + 8, 1); mbar_init(empty_bar + 8 * s, 1); }
@@ -437,6 +438,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         cluster_sync_all();          // nobody leaves while a peer may still read or write its shared memory
         if (threadIdx.x == 0 && blockIdx.z == 0) FL_STAMP(10);
     }
+    if (threadIdx.x == 0) FL_CTA_TIME(1);
     if (warp == 1) {
         __syncwarp();
         tc_fence_after();
@@ -1770,6 +1772,10 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
 }
 
 #ifdef BODA_FL_PROF
+extern "C" int boda_debug_cta_times(unsigned long long* out1024)
+{
+    return cudaMemcpyFromSymbol(out1024, halo::g_cta_times, sizeof(unsigned long long) * 1024) == cudaSuccess ? 0 : 3;
+}
 extern "C" int boda_debug_fl_prof(long long* out16)
 {
     return cudaMemcpyFromSymbol(out16, halo::g_fl_prof, sizeof(long long) * 16) == cudaSuccess ? 0 : 3;

@@ -85,9 +85,13 @@ struct HaloCfg {
 #ifdef BODA_FL_PROF
 // development aid (off unless the library is built with -DBODA_FL_PROF): clock stamps of CTA (0, 0)
 __device__ long long g_fl_prof[16];
+__device__ unsigned long long g_cta_times[2 * 512];      // per CTA: global timer (ns) at its first and last instruction
+__device__ __forceinline__ unsigned long long fl_globaltimer() { unsigned long long t; asm volatile("mov.u64 %0, %%globaltimer;" : "=l"(t)); return t; }
+#define FL_CTA_TIME(which) do { const unsigned _b = blockIdx.x + gridDim.x * (blockIdx.y + gridDim.y * blockIdx.z); if (_b < 512) ::boda::halo::g_cta_times[2 * _b + (which)] = ::boda::halo::fl_globaltimer(); } while (0)
 #define FL_STAMP(i) do { if ((blockIdx.x | blockIdx.y) == 0) ::boda::halo::g_fl_prof[i] = clock64(); } while (0)
 #else
 #define FL_STAMP(i) do { } while (0)
+#define FL_CTA_TIME(which) do { } while (0)
 #endif
 
 // ---- fused ReLU -> max-pool epilogue (3x3 window, stride 2, no padding, floor extent).
