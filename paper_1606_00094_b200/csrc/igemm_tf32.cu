@@ -59,6 +59,7 @@ struct IgemmParams {
     int* status;
     int tx_extra;                // test hook: bytes added to the first stage's expected transfer size of CTA (0,0,0)
     int b_early;                 // the staged filters were written long before this launch (bound filters): their loads need not wait for the preceding kernel
+    int out_tma;                 // staged output without padding rows or columns: the tile leaves through the output tensor map
 };
 
 
@@ -103,7 +104,7 @@ enum { MODE_TF32 = 0, MODE_X3 = 1, MODE_F16 = 2 };
 template <int BN, int MODE>
 __global__ void __launch_bounds__(kIgemmThreads, 1)
 igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_constant__ CUtensorMap map_b,
-                  const IgemmParams p)
+                  const __grid_constant__ CUtensorMap map_o, const IgemmParams p)
 {
     constexpr bool X3 = MODE == MODE_X3;
     constexpr int CH = MODE == MODE_F16 ? 64 : BKC;      // channels per reduction chunk (128 bytes)
@@ -142,6 +143,7 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
         asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
         prefetch_tensormap(&map_a);
         prefetch_tensormap(&map_b);
+        if (p.out_tma) prefetch_tensormap(&map_o);
     }
     if (warp == 1) {
         tmem_alloc(smem_u32(&s_tmem_base), Cfg::TMEM_COLS);
@@ -319,7 +321,42 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
                 tmem_ld_wait();
             }
         };
-        if (p.splits == 1) {
+        // Staged output whose rows follow one another without padding (the consumer reads it through an im2col map or
+        // is a pooling layer): the tile is a box of the [rows][channels] matrix, so it leaves as tensor stores of
+        // 32 rows x 32 channels (4 KB, 128-byte rows swizzled by the row like the exchange blocks).  A warp hands over
+        // its own 32 rows: no barrier between warps, and 8 times fewer copies than one per half row (the copy engine
+        // moved about 13 bytes per clock with 512-byte copies against 32 with large ones).
+        auto store_box = [&](uint32_t chunk_block, int kc, const float (&y)[32]) {
+            const uint32_t box = chunk_block + 4096u * (uint32_t)quarter;
+            const uint32_t a = box + 128u * (uint32_t)lane;
+#pragma unroll
+            for (int g = 0; g < 8; ++g)
+                st_shared_v4(a + (uint32_t)((g ^ (lane & 7)) << 4), round_to_tf32(y[4 * g]), round_to_tf32(y[4 * g + 1]),
+                             round_to_tf32(y[4 * g + 2]), round_to_tf32(y[4 * g + 3]));
+            fence_proxy_async_smem();
+            __syncwarp();
+            if (lane == 0 && kc < p.o.Cp && m0 + 32 * quarter < p.M) {
+                tma_store_2d(&map_o, box, kc, m0 + 32 * quarter);
+                bulk_commit();
+            }
+        };
+        if (p.splits == 1 && p.out_tma) {
+            if (ok) {
+                constexpr int NCH = BN / 32, HALF = (NCH + 1) / 2;
+                const int c_begin = group ? HALF : 0, c_end = group ? NCH : HALF;
+#pragma unroll 1
+                for (int c = c_begin; c < c_end; ++c) {
+                    uint32_t v[32];
+                    load32(32 * c, v);
+                    float y[32];
+                    bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
+                    store_box(smem_base + 16384u * (uint32_t)c, k0 + 32 * c, y);      // the stage buffers are idle now
+                }
+                if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(5);
+                if (lane == 0) bulk_wait_all();
+                if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(6);
+            }
+        } else if (p.splits == 1) {
             if (ok) {
                 const RowDst d = igemm_row_dst(p, m);
                 const uint32_t row_addr = smem_base + (uint32_t)row * out_tile_row_bytes<BN>();   // the stage buffers are idle now
@@ -404,8 +441,11 @@ igemm_tf32_kernel(const __grid_constant__ CUtensorMap map_a, const __grid_consta
 #pragma unroll
                     for (int j = 0; j < 32; ++j) v[j] = __float_as_uint(y[j]);
                     bias_relu32(v, s_bias + rank * per + 32 * c, p.o.relu != 0, y);
-                    store_row32(p.o, d, k0 + rank * per + 32 * c, y);
+                    // (the finished chunk goes back into the received block it was summed from: same rows, same thread)
+                    if (p.out_tma) store_box(recv_base + 16384u * (uint32_t)c, k0 + rank * per + 32 * c, y);
+                    else store_row32(p.o, d, k0 + rank * per + 32 * c, y);
                 }
+                if (p.out_tma && lane == 0) bulk_wait_all();
                 if (threadIdx.x == 64 && blockIdx.z == 0) FL_STAMP(9);
             }
         } else if (ok) {
@@ -715,6 +755,8 @@ struct IgemmPlan {
     CUtensorMap map_b;
     CUtensorMap map_a;
     const void* map_a_base = nullptr;
+    CUtensorMap map_o{};                  // output as a [rows][channels] matrix (im2col kernel, staged output without padding)
+    const void* map_o_base = nullptr;
     // activation layouts on either side (set by igemm_plan_set_io; NCHW by default)
     int tx_extra = 0;                // test hook (BODA_TEST_TX_MISMATCH): makes one bounded wait of one CTA expire
     bool in_packed = false;          // the input already is this plan's staged layout: skip the staging kernel
@@ -1074,7 +1116,7 @@ int launch_bn_mode(IgemmPlan* p, const IgemmParams& prm, cudaStream_t stream)
     BODA_CUDA_TRY(limit.ensure(igemm_tf32_kernel<BN, MODE>, Cfg::SMEM_BYTES));
     dim3 grid(p->tiles_m, p->tiles_n, p->splits);
     BODA_CUDA_TRY(launch_kernel(igemm_tf32_kernel<BN, MODE>, grid, dim3(kIgemmThreads), (size_t)Cfg::SMEM_BYTES, stream, p->splits,
-                                p->map_a, p->map_b, prm));
+                                p->map_a, p->map_b, p->map_o, prm));
     count_launch();
     return BODA_OK;
 }
@@ -1104,6 +1146,25 @@ int encode_map_a(IgemmPlan* p, const void* xp)
         return record_cuda_error(cudaErrorInvalidValue, msg);
     }
     p->map_a_base = xp;
+    return BODA_OK;
+}
+
+// The staged output as a matrix [N*P*Q rows][oCp channels], boxes of 32 x 32 (what one epilogue warp hands over).
+int encode_map_o(IgemmPlan* p, float* out)
+{
+    const ConvDims& d = p->d;
+    const cuuint64_t dims[2] = {(cuuint64_t)p->oCp, (cuuint64_t)d.M};
+    const cuuint64_t strides[1] = {(cuuint64_t)p->oCp * 4};
+    const cuuint32_t box[2] = {32, 32}, estr[2] = {1, 1};
+    CUresult r = g_encode_tiled(&p->map_o, CU_TENSOR_MAP_DATA_TYPE_FLOAT32, 2, out, dims, strides, box, estr,
+                                CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B,
+                                CU_TENSOR_MAP_L2_PROMOTION_L2_128B, CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE);
+    if (r != CUDA_SUCCESS) {
+        char msg[96];
+        std::snprintf(msg, sizeof(msg), "cuTensorMapEncodeTiled (output) failed with CUresult %d", (int)r);
+        return record_cuda_error(cudaErrorInvalidValue, msg);
+    }
+    p->map_o_base = out;
     return BODA_OK;
 }
 
@@ -1607,6 +1668,7 @@ int igemm_plan_set_io(IgemmPlan* p, int in_packed, int out_packed, int oHp, int 
     p->in_packed = in_packed != 0;
     p->out_packed = out_packed ? 1 : 0;
     p->oHp = oHp; p->oWp = oWp; p->oCp = oCp;
+    p->map_o_base = nullptr;
     return BODA_OK;
 }
 
@@ -1761,6 +1823,11 @@ int igemm_launch(IgemmPlan* p, const float* in, const float* filt, const float* 
     prm.tx_extra = p->tx_extra;
     prm.b_early = (filt == p->bound_filt) ? 1 : 0;
     prm.status = p->d_status;
+    prm.out_tma = (p->out_packed && p->oHp == d.P && p->oWp == d.Q && ((uintptr_t)out & 15) == 0) ? 1 : 0;
+    if (prm.out_tma && p->map_o_base != out) {
+        int rc = encode_map_o(p, out);
+        if (rc != BODA_OK) return rc;
+    }
     switch (p->BN) {
         case 64: return launch_bn<64>(p, prm, stream);
         case 96: return launch_bn<96>(p, prm, stream);
@@ -1863,6 +1930,7 @@ int igemm_run_in_region(const ConvDims& d, int variant, const float* in, const f
     prm.bias = bias;
     prm.o = make_out_spec(p, out);
     prm.b_early = 0;
+    prm.out_tma = 0;
     prm.tx_extra = p->tx_extra;
     prm.status = p->d_status;
     switch (p->BN) {

@@ -234,6 +234,13 @@ __device__ __forceinline__ void bulk_store_global(void* gdst, uint32_t smem_src,
 {
     asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;" :: "l"(gdst), "r"(smem_src), "r"(bytes) : "memory");
 }
+// a box of shared memory (laid out as the map's swizzle says) -> the tensor at (x, y); x * element size must be a
+// multiple of 16 bytes, and elements of the box outside the tensor are not written
+__device__ __forceinline__ void tma_store_2d(const CUtensorMap* map, uint32_t smem_src, int x, int y)
+{
+    asm volatile("cp.async.bulk.tensor.2d.global.shared::cta.bulk_group [%0, {%2, %3}], [%1];"
+                 :: "l"(map), "r"(smem_src), "r"(x), "r"(y) : "memory");
+}
 __device__ __forceinline__ void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
 __device__ __forceinline__ void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
 // shared memory of this CTA -> shared memory of a CTA of the cluster (`dst` and `bar` are cluster addresses from
