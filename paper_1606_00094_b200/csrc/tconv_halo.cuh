@@ -99,11 +99,11 @@ __device__ __forceinline__ unsigned long long fl_globaltimer() { unsigned long l
 // (Section 3); here the pooling that follows the activation is fused as well, so that the convolution's output -
 // four times the bytes of the pooled tensor - is never written.  The tile's rows are whole output rows of one image
 // (see HaloParams::pool_rows), so every pooling window of the pooled rows it owns lies inside the tile.
-// 32 channels at a time: all accumulators' columns [32c, 32c+32) go, with bias and ReLU applied, into a shared-memory
+// 32 channels at a time: all accumulators' columns [32c, 32c+32) go into a shared-memory
 // block [128*NACC positions][32 channels] (16-byte pieces XOR-swizzled by the position, so that thread-per-position
 // writes and the window reads below are free of bank conflicts); after a barrier of the 256 epilogue threads every
-// thread takes pooled (row, column, 4 channels) items, reads the nine window positions and writes the maximum,
-// rounded to TF32, into the pooled tile [pool_rows * Q][BN] (or straight to an NCHW tensor).  Two blocks alternate,
+// thread takes pooled (row, column, 4 channels) items, reads the nine window positions and writes the maximum -
+// plus bias, after ReLU, rounded to TF32 - into the pooled tile [pool_rows * Q][BN] (or straight to an NCHW tensor).  Two blocks alternate,
 // so filling block c+1 overlaps pooling block c.  At the end each pooled position leaves as one bulk copy.
 // bytes of one position's 32 channels in a pooling block: 128 of data + 16 of padding, which keeps thread-per-position
 // 16-byte stores and piece-per-thread window loads free of bank conflicts without any address swizzling
@@ -135,13 +135,18 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
 #pragma unroll 1
     for (int c = 0; c < NCH; ++c) {
         const uint32_t block = smem_base + (uint32_t)(c & 1) * BLOCK_BYTES;
+        // The block takes the RAW accumulators: adding a per-channel bias, ReLU and rounding are all non-decreasing, so
+        // they commute with the maximum and are applied to the pooled values only - a quarter of the arithmetic, which
+        // is what bounds this phase (two epilogue warps per scheduler).
         auto put = [&](int acc, const uint32_t (&v)[32]) {
-            float y[32];
-            bias_relu32(v, s_bias + 32 * c, p.o.relu != 0, y);
             const uint32_t a = block + (uint32_t)(acc * 128 + quarter * 32 + lane) * kPoolRowBytes;
 #pragma unroll
-            for (int q = 0; q < 8; ++q) st_shared_v4(a + 16u * q, y[4 * q], y[4 * q + 1], y[4 * q + 2], y[4 * q + 3]);
+            for (int q = 0; q < 8; ++q)
+                st_shared_v4(a + 16u * q, __uint_as_float(v[4 * q]), __uint_as_float(v[4 * q + 1]), __uint_as_float(v[4 * q + 2]),
+                             __uint_as_float(v[4 * q + 3]));
         };
+        const float4 b4 = *reinterpret_cast<const float4*>(s_bias + 32 * c + 4 * g);
+        const bool relu = p.o.relu != 0;
         if constexpr (NACC == 4) {
             // both of this group's accumulators are read from tensor memory before either is used: one load latency per block
             uint32_t v0[32], v1[32];
@@ -181,6 +186,8 @@ __device__ __forceinline__ void halo_pooled_epilogue(const HaloParams& p, uint32
                 float4 m;
                 m.x = fmaxf(top.x, fmaxf(mid.x, bot.x)); m.y = fmaxf(top.y, fmaxf(mid.y, bot.y));
                 m.z = fmaxf(top.z, fmaxf(mid.z, bot.z)); m.w = fmaxf(top.w, fmaxf(mid.w, bot.w));
+                m.x += b4.x; m.y += b4.y; m.z += b4.z; m.w += b4.w;
+                if (relu) { m.x = fmaxf(m.x, 0.f); m.y = fmaxf(m.y, 0.f); m.z = fmaxf(m.z, 0.f); m.w = fmaxf(m.w, 0.f); }
                 const int t = pr * p.o.Q + pq;
                 if (p.o.packed) {
                     st_shared_v4(pooled + (uint32_t)(t * BN + 32 * c + 4 * g) * 4u, round_to_tf32(m.x), round_to_tf32(m.y),
