@@ -450,15 +450,25 @@ int boda_stack_fwd_host(boda_stack* s, const float* in_host, float* out_host, vo
         for (int i = 0; i < k && ce == cudaSuccess && rc == BODA_OK; ++i) {
             ce = cudaStreamWaitEvent(st, s->chunk_events[i], 0);
             if (ce == cudaSuccess) rc = boda_stack_fwd(s->sub, s->staging_in + i * in_pitch, s->staging_out + i * out_chunk, stream);
+            if (ce != cudaSuccess || rc != BODA_OK) break;
+            // a slice's result goes back while the next slice is still computing: on the copy stream (behind the
+            // input copies, which are done by then) for all but the last slice
+            cudaStream_t back = i + 1 < k ? s->copy_stream : st;
+            if (i + 1 < k) {
+                ce = cudaEventRecord(s->chunk_events[i], st);             // the slice's input event has been consumed above
+                if (ce == cudaSuccess) ce = cudaStreamWaitEvent(s->copy_stream, s->chunk_events[i], 0);
+            }
+            if (ce == cudaSuccess)
+                ce = cudaMemcpyAsync(out_host + i * out_chunk, s->staging_out + i * out_chunk, out_chunk * sizeof(float),
+                                     cudaMemcpyDeviceToHost, back);
         }
-        if (ce == cudaSuccess && rc == BODA_OK)
-            ce = cudaMemcpyAsync(out_host, s->staging_out, s->out_elems * sizeof(float), cudaMemcpyDeviceToHost, st);
         if (ce != cudaSuccess || rc != BODA_OK) {
             // no copy may still be writing the staging buffer when the caller gets the error
             (void)cudaStreamSynchronize(s->copy_stream);
             (void)cudaStreamSynchronize(st);
             return rc != BODA_OK ? rc : record_cuda_error(ce, "boda_stack_fwd_host (sliced copies)");
         }
+        BODA_CUDA_TRY(cudaStreamSynchronize(s->copy_stream));
         BODA_CUDA_TRY(cudaStreamSynchronize(st));
         return BODA_OK;
     }
