@@ -142,28 +142,46 @@ tconv_first_layer_kernel(const __grid_constant__ CUtensorMap map_b0, const __gri
             constexpr uint32_t idesc = instr_desc_tf32<BN>();
             const uint32_t my_acc = tmem_acc + (uint32_t)(acc * BN);
             uint32_t stage = 0, par = 0;
+            // Between a stage's barrier and its MMAs the four issuers are all busy with bookkeeping and the tensor pipe
+            // idles, so the loops hold as little of it as possible: one loop per chunk, descriptors advanced by
+            // additions (a descriptor's address field counts 16-byte units: 8 per slab row of chunk 0, 4 of chunk 1).
             bool ok = mbar_wait(slab_full, 0, &s_abort, p.h.status, 53);
-            for (int i = 0; ok && i < 2 * taps; ++i) {
-                const bool second = i >= taps;
-                if (i == taps) { if (acc == 0) FL_STAMP(1); ok = mbar_wait(slab_full + 8, 0, &s_abort, p.h.status, 54); if (!ok) break; }
-                ok = mbar_wait(b_full + 8 * stage, par, &s_abort, p.h.status, 55);
-                if (!ok) break;
-                tc_fence_after();
-                const int tap = second ? i - taps : i;
-                const int r = tap / p.h.S;
-                const uint32_t row = (uint32_t)(acc * 128 + r * p.h.Wp + (tap - r * p.h.S));   // first slab row of this tap's A tile
-                const uint32_t b_addr = smem_b + stage * B_STAGE_BYTES;
-                if (!second) {
-                    const uint64_t da = smem_desc_k_sw128(slab0 + row * 128u), db = smem_desc_k_sw128(b_addr);
+            const uint32_t S = (uint32_t)p.h.S, row_step = (uint32_t)(p.h.Wp - p.h.S + 1);   // slab rows from a tap row's last tap to the next row's first
+            const uint32_t nstages = (uint32_t)p.b_stages;
+            uint32_t b_addr = smem_b;
+            {
+                uint64_t da = smem_desc_k_sw128(slab0 + (uint32_t)(acc * 128) * 128u);
+                uint32_t s = 0;
+                for (int i = 0; ok && i < taps; ++i) {
+                    ok = mbar_wait(b_full + 8 * stage, par, &s_abort, p.h.status, 55);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t db = smem_desc_k_sw128(b_addr);
 #pragma unroll
                     for (int k = 0; k < 4; ++k) umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, (i | k) ? 1u : 0u);
-                } else {
-                    const uint64_t da = smem_desc_k_sw64(slab1 + row * 64u), db = smem_desc_k_sw64(b_addr);
+                    tc_commit(b_empty + 8 * stage);
+                    b_addr += B_STAGE_BYTES;
+                    if (++stage == nstages) { stage = 0; par ^= 1u; b_addr = smem_b; }
+                    if (++s == S) { s = 0; da += 8 * row_step; } else da += 8;
+                }
+            }
+            if (acc == 0) FL_STAMP(1);
+            if (ok) ok = mbar_wait(slab_full + 8, 0, &s_abort, p.h.status, 54);
+            {
+                uint64_t da = smem_desc_k_sw64(slab1 + (uint32_t)(acc * 128) * 64u);
+                uint32_t s = 0;
+                for (int i = 0; ok && i < taps; ++i) {
+                    ok = mbar_wait(b_full + 8 * stage, par, &s_abort, p.h.status, 55);
+                    if (!ok) break;
+                    tc_fence_after();
+                    const uint64_t db = smem_desc_k_sw64(b_addr);
 #pragma unroll
                     for (int k = 0; k < 2; ++k) umma_tf32(my_acc, da + 2 * k, db + 2 * k, idesc, 1u);
+                    tc_commit(b_empty + 8 * stage);
+                    b_addr += B_STAGE_BYTES;
+                    if (++stage == nstages) { stage = 0; par ^= 1u; b_addr = smem_b; }
+                    if (++s == S) { s = 0; da += 4 * row_step; } else da += 4;
                 }
-                tc_commit(b_empty + 8 * stage);
-                if (++stage == (uint32_t)p.b_stages) { stage = 0; par ^= 1u; }
             }
             tc_commit(accum_bar);
             if (acc == 0) FL_STAMP(6);
